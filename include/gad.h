@@ -1,0 +1,183 @@
+/*
+ * gad.h - C boundary of the B200 (sm_100a) library for one training epoch of GAD
+ * (Graph-Augmentation-based Distributed GCN, arXiv 2110.02987).
+ *
+ * What the library computes: K replicas of an L-layer GCN, one per augmented subgraph g'_k produced by
+ * GAD-Partition, all batched on one GPU.  One call of gad_train_epoch is one pass of Algorithm 2 with one
+ * subgraph per processor: forward propagation, loss, backward propagation (Section 3.3), the variance-based
+ * subgraph importance zeta (Section 3.4.1) and the weighted global consensus over the K parameter copies
+ * (Section 3.4.2).  The partition and the replicated-node lists are inputs (they are GAD-Partition's output,
+ * Section 3.2); the library does not compute them.
+ *
+ * Conventions
+ *   - Every function returns an int status: GAD_OK (0) or a negative GAD_ERR_* code.  Nothing throws.
+ *     gad_last_error(ctx) gives a NUL-terminated message that belongs to the context.
+ *   - "host" pointers are ordinary CPU memory owned by the caller; they are only read (or written) during the
+ *     call.  "device" pointers are CUDA device memory of the current device.
+ *   - The library allocates no device memory: the caller passes one device workspace (size from
+ *     gad_workspace_bytes) and a CUDA stream; both must outlive the context.  All kernels of a context run on
+ *     that stream.  A context is not thread-safe.
+ *   - Matrices are row-major.  One replica's parameters are the P floats
+ *       [ W_0 (F_0 x F_1), b_0 (F_1), W_1 (F_1 x F_2), b_1 (F_2), ... ],  P = sum_l (F_l F_{l+1} + F_{l+1}).
+ *   - "store row": the K augmented subgraphs are kept as one block-diagonal matrix.  Subgraph k owns the rows
+ *     sub_off[k] .. sub_off[k+1]-1: first its core nodes in the order given, then its replicated nodes in the
+ *     order given.  N' = sub_off[K], nnz' = stored entries of all A~_k.
+ */
+#ifndef GAD_H
+#define GAD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GAD_OK 0
+#define GAD_ERR_ARG (-1)            /* NULL pointer, non-positive size, bad flag                           */
+#define GAD_ERR_RANGE (-2)          /* node id, column, label or split value out of range                  */
+#define GAD_ERR_UNSORTED (-3)       /* a pointer array (rowptr, core_ptr, halo_ptr) is not non-decreasing   */
+#define GAD_ERR_DUPLICATE (-4)      /* a node listed twice inside one subgraph, or in two core sets         */
+#define GAD_ERR_OOM (-5)            /* workspace too small, or host allocation failed                       */
+#define GAD_ERR_NONFINITE (-6)      /* a loss came out NaN or infinite (reported, never trapped)            */
+#define GAD_ERR_DEVICE_TIMEOUT (-7) /* a bounded device-side wait ran out                                   */
+#define GAD_ERR_CUDA (-8)           /* a CUDA call failed; see gad_last_error                               */
+#define GAD_ERR_UNSUPPORTED (-9)    /* a documented option that this build does not implement               */
+
+typedef struct gad_ctx gad_ctx;
+
+/* The whole graph G = (V, E) in CSR form, host memory.  Columns need not be sorted; parallel edges are summed;
+ * w == NULL means unit weights.  An undirected graph lists every edge in both directions. */
+typedef struct {
+    int32_t n;
+    int64_t nnz;
+    const int64_t* rowptr; /* [n+1] */
+    const int32_t* col;    /* [nnz] */
+    const float* w;        /* [nnz] or NULL */
+} gad_csr;
+
+/* GAD-Partition's output (Definition 1 and Algorithm 1): for subgraph k the core nodes
+ * core_nodes[core_ptr[k] .. core_ptr[k+1]) (disjoint between subgraphs; they need not cover V) and the
+ * replicated nodes halo_nodes[halo_ptr[k] .. halo_ptr[k+1]) (not in the same subgraph's core set; a node may
+ * be replicated into several subgraphs).  Host memory. */
+typedef struct {
+    int32_t K;
+    const int64_t* core_ptr;   /* [K+1] */
+    const int32_t* core_nodes;
+    const int64_t* halo_ptr;   /* [K+1] */
+    const int32_t* halo_nodes;
+} gad_partition;
+
+typedef struct {
+    int32_t L;            /* number of GCN layers, >= 1                                                      */
+    const int32_t* dims;  /* [L+1] host: F_0 (input features) ... F_L (classes)                              */
+    float lr;             /* eta of the update equation (Section 3.3 / 3.4.2)                                 */
+    float dropout;        /* probability of dropping a hidden unit after the ReLU, in [0,1); 0 = none         */
+    uint64_t seed;        /* seed of the dropout mask and of the default initialisation                       */
+    int32_t gemm_mode;    /* 0: fp32-accurate transform (SIMT, or split-TF32 tensor cores);                   *
+                           * 1: bf16 operands with fp32 accumulation on tensor cores                          */
+    int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form (GAD_ERR_UNSUPPORTED)       */
+    float beta;           /* beta of the importance weight (Section 3.4.1); the paper uses 1                  */
+    int32_t weighted;     /* 1: weighted global consensus (Section 3.4.2); 0: plain average (Definition 3)    */
+    int32_t flags;        /* bit 0: force the SIMT transform even where a tensor-core kernel exists           */
+} gad_config;
+
+/* Bytes of device workspace gad_create needs for these inputs.  Host-only; touches no GPU. */
+int gad_workspace_bytes(const gad_csr* g, const gad_partition* part, const gad_config* cfg, size_t* bytes);
+
+/* Builds the block-diagonal store of the augmented subgraphs g'_k = (v_k + v'_k, e_k + e'_k) (Algorithm 1,
+ * last step): every edge of G with both endpoints in v_k + v'_k, a unit self-loop added where a node has none,
+ * A~_k = D~^-1/2 (A'_k + I) D~^-1/2 with the degrees taken inside g'_k (the A~ of the forward equation,
+ * Section 3.3); uploads it with the features, labels and split, and makes K identical parameter copies
+ * (Algorithm 2: every processor starts from the same model).
+ *   X            host [n x dims[0]]
+ *   labels       host [n], values in 0 .. dims[L]-1
+ *   split        host [n]: 0 train, 1 validation, 2 test.  Only core nodes with split 0 carry loss.
+ *   init_params  host [P], or NULL for seeded Glorot-uniform W and zero b
+ *   workspace    device, 256-byte aligned, at least gad_workspace_bytes; owned by the caller
+ *   stream       a cudaStream_t (NULL = the default stream)
+ * Synchronises the stream before returning.  On error *out is NULL. */
+int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const float* X, const int32_t* labels,
+               const uint8_t* split, const gad_config* cfg, const float* init_params, void* workspace,
+               size_t workspace_bytes, void* stream);
+
+/* One pass of Algorithm 2 (one subgraph per processor): for every replica k
+ *   forward   H^(l+1) = sigma(A~_k (H^(l) W_k^(l)) + b_k^(l)), sigma = ReLU (identity on the last layer), with
+ *             the optional dropout after the ReLU                          (Section 3.3, forward equations)
+ *   loss      softmax cross-entropy, mean over the core training nodes     (Section 3.3, loss equation)
+ *   backward  gradients of every W_k^(l), b_k^(l) through A~_k^T           (Section 3.3, gradient equation)
+ *   update    theta_k <- theta_k - eta * grad_k                            (Section 3.3, update equation)
+ * then zeta_k and the weighted consensus theta_k <- sum_j w_j theta_j      (Sections 3.4.1, 3.4.2).
+ * loss_out: host [K+1] = the K subgraph losses, then sum_k |T_k| L_k / sum_k |T_k|, all evaluated before the
+ * update; the call then waits for the stream.  loss_out == NULL: the epoch is only enqueued (no wait, no
+ * copy); read the losses later with gad_get_loss.  Returns GAD_ERR_NONFINITE if a loss is NaN or infinite
+ * (detected when the losses are read). */
+int gad_train_epoch(gad_ctx* ctx, float* loss_out);
+
+/* Losses of the most recent epoch, host [K+1]; waits for the stream. */
+int gad_get_loss(gad_ctx* ctx, float* loss_out);
+
+/* Inference forward (no dropout) of replica k on subgraph k.  logits_out: host [n x dims[L]] in graph-node
+ * order, filled for core nodes; rows that no subgraph owns are zero.  (Section 3.3, forward equations.) */
+int gad_forward(gad_ctx* ctx, float* logits_out);
+
+/* Variance-based importance of every subgraph (Section 3.4.1) and the consensus weights (Section 3.4.2):
+ *   p_i = deg_k(i) / sum_j deg_k(j)  (degree inside g'_k without the self-loop; uniform if there are no edges)
+ *   S_k = sum_{i<j} p_i p_j,   D_k = sqrt( sum_{i<j} p_i p_j |x_i - x_j|^2 / S_k )  on the input features
+ *   zeta_k = S_k / (D_k + beta),   w_k = zeta_k / sum_j zeta_j   (1/K when weighted == 0 or all zeta are 0)
+ * zeta_out, w_out: host [K], either may be NULL. */
+int gad_subgraph_weights(gad_ctx* ctx, float* zeta_out, float* w_out);
+
+/* Weighted global consensus on its own: theta_k <- sum_j w_j theta_j for every k (Section 3.4.2; Definition 3
+ * when weighted == 0).  Enqueued on the stream. */
+int gad_consensus(gad_ctx* ctx);
+
+/* Parameter copy / gradient of replica k, host [P] in the layout above.  Gradients are those of the most recent
+ * epoch (d L_k / d theta_k).  These calls wait for the stream. */
+int gad_get_params(gad_ctx* ctx, int32_t k, float* out);
+int gad_set_params(gad_ctx* ctx, int32_t k, const float* in);
+int gad_get_grads(gad_ctx* ctx, int32_t k, float* out);
+int gad_param_count(const gad_ctx* ctx, int64_t* P);
+
+/* The store as built (for checking the bookkeeping): sizes, then the arrays, all host.
+ *   rowptr int64 [N'+1], col int32 [nnz'] (store-row ids, ascending inside a row), val float [nnz'],
+ *   sub_off int32 [K+1], gid int32 [N'] (graph node of each store row), deg int32 [N'] (local degree without
+ *   the self-loop).  Any array pointer may be NULL. */
+int gad_store_sizes(const gad_ctx* ctx, int64_t* n_prime, int64_t* nnz_prime);
+int gad_get_store(gad_ctx* ctx, int64_t* rowptr, int32_t* col, float* val, int32_t* sub_off, int32_t* gid,
+                  int32_t* deg);
+
+/* Activation H^(l) of the most recent forward pass, l = 0 .. L (l = L: logits), host [N' x dims[l]] in store-row
+ * order.  Waits for the stream. */
+int gad_get_activation(gad_ctx* ctx, int32_t l, float* out);
+
+/* Replaces the node features and/or labels (either may be NULL), host arrays of the shapes given to
+ * gad_create.  The copies are enqueued on the stream from the caller's buffers, which must stay valid until
+ * the stream has passed them (pinned memory makes the copy asynchronous). */
+int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels);
+
+/* Epoch counter (it indexes the dropout mask); set it to resume a run. */
+int gad_get_epoch(const gad_ctx* ctx, int64_t* epoch);
+int gad_set_epoch(gad_ctx* ctx, int64_t epoch);
+
+/* Per-kernel timing with CUDA events on the context's stream.  While enabled, every kernel launch of the
+ * epoch is bracketed by two events.  gad_profile_read waits for the stream and returns, for entry i of
+ * gad_profile_count entries: a name (up to 63 chars + NUL), launches and total milliseconds since the last
+ * gad_profile_reset, and the algorithmic bytes and flops of ONE launch. */
+int gad_profile_enable(gad_ctx* ctx, int32_t on);
+int gad_profile_reset(gad_ctx* ctx);
+int gad_profile_count(const gad_ctx* ctx, int32_t* count);
+int gad_profile_read(gad_ctx* ctx, int32_t i, char* name64, int64_t* launches, double* total_ms,
+                     double* bytes_per_launch, double* flops_per_launch);
+
+/* Message of the context's last error; with ctx == NULL, of the calling thread's last error (e.g. after a failed
+ * gad_create). */
+const char* gad_last_error(const gad_ctx* ctx);
+
+/* Frees the context.  Frees nothing the caller allocated (workspace, stream). */
+void gad_destroy(gad_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GAD_H */

@@ -1,0 +1,305 @@
+"""Thin ctypes binding of the C-ABI library ``libgad.so`` (see ``include/gad.h``).
+
+Argument marshalling only: every step of the epoch runs in the library's CUDA kernels.  PyTorch is
+used for what the boundary leaves to the caller: the device workspace and the stream.  There is no
+CPU fallback; importing works without a GPU (so the exported symbols can be checked), but every
+compute call needs the built library and a CUDA device and raises otherwise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgad.so")
+
+GAD_OK = 0
+ERRORS = {-1: "GAD_ERR_ARG", -2: "GAD_ERR_RANGE", -3: "GAD_ERR_UNSORTED", -4: "GAD_ERR_DUPLICATE", -5: "GAD_ERR_OOM",
+          -6: "GAD_ERR_NONFINITE", -7: "GAD_ERR_DEVICE_TIMEOUT", -8: "GAD_ERR_CUDA", -9: "GAD_ERR_UNSUPPORTED"}
+
+# Every symbol include/gad.h declares.
+SYMBOLS = (
+    "gad_workspace_bytes", "gad_create", "gad_train_epoch", "gad_get_loss", "gad_forward", "gad_subgraph_weights",
+    "gad_consensus", "gad_get_params", "gad_set_params", "gad_get_grads", "gad_param_count", "gad_store_sizes",
+    "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
+    "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_last_error", "gad_destroy",
+)
+
+
+class GadError(RuntimeError):
+    def __init__(self, code, msg=""):
+        self.code = code
+        super().__init__("%s (%d)%s" % (ERRORS.get(code, "GAD_ERR_?"), code, ": " + msg if msg else ""))
+
+
+class gad_csr(C.Structure):
+    _fields_ = [("n", C.c_int32), ("nnz", C.c_int64), ("rowptr", C.POINTER(C.c_int64)), ("col", C.POINTER(C.c_int32)),
+                ("w", C.POINTER(C.c_float))]
+
+
+class gad_partition(C.Structure):
+    _fields_ = [("K", C.c_int32), ("core_ptr", C.POINTER(C.c_int64)), ("core_nodes", C.POINTER(C.c_int32)),
+                ("halo_ptr", C.POINTER(C.c_int64)), ("halo_nodes", C.POINTER(C.c_int32))]
+
+
+class gad_config(C.Structure):
+    _fields_ = [("L", C.c_int32), ("dims", C.POINTER(C.c_int32)), ("lr", C.c_float), ("dropout", C.c_float),
+                ("seed", C.c_uint64), ("gemm_mode", C.c_int32), ("zeta_mode", C.c_int32), ("beta", C.c_float),
+                ("weighted", C.c_int32), ("flags", C.c_int32)]
+
+
+_lib = None
+
+
+def load():
+    """Loads libgad.so; raises if it has not been built (``python -m paper_2110_02987_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libgad.so is missing: build it with paper_2110_02987_b200/build.py "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.gad_last_error.restype = C.c_char_p
+        L.gad_last_error.argtypes = [C.c_void_p]
+        L.gad_destroy.restype = None
+        L.gad_destroy.argtypes = [C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _ptr(a, t):
+    return a.ctypes.data_as(C.POINTER(t)) if a is not None else None
+
+
+def _arr(a, dtype):
+    return None if a is None else np.ascontiguousarray(a, dtype=dtype)
+
+
+class _Inputs:
+    """Keeps the marshalled host arrays alive for the duration of a call."""
+
+    def __init__(self, n, rowptr, col, weights, core_ptr, core_nodes, halo_ptr, halo_nodes, dims, lr, dropout, seed,
+                 gemm_mode, zeta_mode, beta, weighted, flags):
+        self.rowptr = _arr(rowptr, np.int64)
+        self.col = _arr(col, np.int32)
+        self.w = _arr(weights, np.float32)
+        self.core_ptr = _arr(core_ptr, np.int64)
+        self.core_nodes = _arr(core_nodes, np.int32)
+        self.halo_ptr = _arr(halo_ptr, np.int64)
+        self.halo_nodes = _arr(halo_nodes, np.int32)
+        self.dims = np.asarray(dims, dtype=np.int32)
+        self.csr = gad_csr(int(n), int(self.rowptr[-1]) if self.rowptr is not None and self.rowptr.size else 0,
+                           _ptr(self.rowptr, C.c_int64), _ptr(self.col, C.c_int32), _ptr(self.w, C.c_float))
+        self.part = gad_partition(int(self.core_ptr.shape[0] - 1), _ptr(self.core_ptr, C.c_int64),
+                                  _ptr(self.core_nodes, C.c_int32), _ptr(self.halo_ptr, C.c_int64),
+                                  _ptr(self.halo_nodes, C.c_int32))
+        self.cfg = gad_config(int(self.dims.shape[0] - 1), _ptr(self.dims, C.c_int32), float(lr), float(dropout), int(seed),
+                              int(gemm_mode), int(zeta_mode), float(beta), 1 if weighted else 0, int(flags))
+
+
+def gad_workspace_bytes(n, rowptr, col, core_ptr, core_nodes, halo_ptr, halo_nodes, dims, *, weights=None, lr=0.01,
+                        dropout=0.0, seed=0, gemm_mode=0, zeta_mode=0, beta=1.0, weighted=True, flags=0) -> int:
+    L = load()
+    inp = _Inputs(n, rowptr, col, weights, core_ptr, core_nodes, halo_ptr, halo_nodes, dims, lr, dropout, seed, gemm_mode,
+                  zeta_mode, beta, weighted, flags)
+    out = C.c_size_t(0)
+    rc = L.gad_workspace_bytes(C.byref(inp.csr), C.byref(inp.part), C.byref(inp.cfg), C.byref(out))
+    if rc != GAD_OK:
+        raise GadError(rc, (L.gad_last_error(None) or b"").decode())
+    return int(out.value)
+
+
+class Gad:
+    """One library context: K GCN replicas over K augmented subgraphs on the current CUDA device.
+
+    Methods carry the names of the C entry points (without the ``gad_`` prefix where it reads better as a method:
+    ``train_epoch``, ``forward``, ``subgraph_weights``, ``consensus`` ...).
+    """
+
+    def __init__(self, n, rowptr, col, core_ptr, core_nodes, halo_ptr, halo_nodes, X, labels, split, dims, *,
+                 init_params=None, weights=None, lr=0.01, dropout=0.0, seed=0, gemm_mode=0, zeta_mode=0, beta=1.0,
+                 weighted=True, flags=0, stream=None, device=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the GAD library needs a CUDA device (there is no CPU fallback)")
+        L = load()
+        self._L = L
+        self._h = None
+        self.n = int(n)
+        self.dims = tuple(int(d) for d in dims)
+        inp = _Inputs(n, rowptr, col, weights, core_ptr, core_nodes, halo_ptr, halo_nodes, dims, lr, dropout, seed,
+                      gemm_mode, zeta_mode, beta, weighted, flags)
+        self.K = int(inp.part.K)
+        X = _arr(X, np.float32)
+        labels = _arr(labels, np.int32)
+        split = _arr(split, np.uint8)
+        if X.shape != (self.n, self.dims[0]) or labels.shape != (self.n,) or split.shape != (self.n,):
+            raise GadError(-1, "X / labels / split have the wrong shape")
+        init = _arr(init_params, np.float32)
+        nbytes = C.c_size_t(0)
+        rc = L.gad_workspace_bytes(C.byref(inp.csr), C.byref(inp.part), C.byref(inp.cfg), C.byref(nbytes))
+        if rc != GAD_OK:
+            raise GadError(rc, (L.gad_last_error(None) or b"").decode())
+        self.device = torch.device(device if device is not None else "cuda:%d" % torch.cuda.current_device())
+        self.workspace_bytes = int(nbytes.value)
+        with torch.cuda.device(self.device):
+            self._ws = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            base = self._ws.data_ptr()
+            aligned = (base + 255) // 256 * 256
+            self._stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            h = C.c_void_p(None)
+            rc = L.gad_create(C.byref(h), C.byref(inp.csr), C.byref(inp.part), _ptr(X, C.c_float), _ptr(labels, C.c_int32),
+                              _ptr(split, C.c_uint8), C.byref(inp.cfg), _ptr(init, C.c_float), C.c_void_p(aligned),
+                              C.c_size_t(self.workspace_bytes), C.c_void_p(self._stream.cuda_stream))
+        if rc != GAD_OK:
+            raise GadError(rc, (L.gad_last_error(None) or b"").decode())
+        self._h = h
+        P = C.c_int64(0)
+        self._ck(L.gad_param_count(self._h, C.byref(P)))
+        self.P = int(P.value)
+        a, b = C.c_int64(0), C.c_int64(0)
+        self._ck(L.gad_store_sizes(self._h, C.byref(a), C.byref(b)))
+        self.n_prime, self.nnz_prime = int(a.value), int(b.value)
+
+    # -- plumbing ------------------------------------------------------------------------------
+    def _ck(self, rc):
+        if rc != GAD_OK:
+            raise GadError(rc, (self._L.gad_last_error(self._h) or b"").decode())
+
+    def destroy(self):
+        if self._h is not None:
+            self._L.gad_destroy(self._h)
+            self._h = None
+            self._ws = None
+
+    close = destroy
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.destroy()
+
+    # -- the epoch -----------------------------------------------------------------------------
+    def train_epoch(self, loss_out=None, wait=True):
+        """gad_train_epoch.  With wait=True returns the float32 [K+1] losses (and waits for the stream); with
+        wait=False only enqueues the epoch and returns None.  ``loss_out`` may be a preallocated float32 [K+1]
+        array (e.g. a view of pinned memory)."""
+        if not wait:
+            self._ck(self._L.gad_train_epoch(self._h, None))
+            return None
+        out = loss_out if loss_out is not None else np.zeros(self.K + 1, dtype=np.float32)
+        self._ck(self._L.gad_train_epoch(self._h, _ptr(out, C.c_float)))
+        return out
+
+    def get_loss(self):
+        out = np.zeros(self.K + 1, dtype=np.float32)
+        self._ck(self._L.gad_get_loss(self._h, _ptr(out, C.c_float)))
+        return out
+
+    def forward(self):
+        out = np.zeros((self.n, self.dims[-1]), dtype=np.float32)
+        self._ck(self._L.gad_forward(self._h, _ptr(out, C.c_float)))
+        return out
+
+    def subgraph_weights(self):
+        z = np.zeros(self.K, dtype=np.float32)
+        w = np.zeros(self.K, dtype=np.float32)
+        self._ck(self._L.gad_subgraph_weights(self._h, _ptr(z, C.c_float), _ptr(w, C.c_float)))
+        return z, w
+
+    def consensus(self):
+        self._ck(self._L.gad_consensus(self._h))
+
+    # -- accessors -----------------------------------------------------------------------------
+    def get_params(self, k):
+        out = np.zeros(self.P, dtype=np.float32)
+        self._ck(self._L.gad_get_params(self._h, C.c_int32(k), _ptr(out, C.c_float)))
+        return out
+
+    def set_params(self, k, p):
+        p = _arr(p, np.float32)
+        if p.shape != (self.P,):
+            raise GadError(-1, "parameter vector has the wrong length")
+        self._ck(self._L.gad_set_params(self._h, C.c_int32(k), _ptr(p, C.c_float)))
+
+    def get_grads(self, k):
+        out = np.zeros(self.P, dtype=np.float32)
+        self._ck(self._L.gad_get_grads(self._h, C.c_int32(k), _ptr(out, C.c_float)))
+        return out
+
+    def get_store(self):
+        rowptr = np.zeros(self.n_prime + 1, dtype=np.int64)
+        col = np.zeros(self.nnz_prime, dtype=np.int32)
+        val = np.zeros(self.nnz_prime, dtype=np.float32)
+        sub_off = np.zeros(self.K + 1, dtype=np.int32)
+        gid = np.zeros(self.n_prime, dtype=np.int32)
+        deg = np.zeros(self.n_prime, dtype=np.int32)
+        self._ck(self._L.gad_get_store(self._h, _ptr(rowptr, C.c_int64), _ptr(col, C.c_int32), _ptr(val, C.c_float),
+                                       _ptr(sub_off, C.c_int32), _ptr(gid, C.c_int32), _ptr(deg, C.c_int32)))
+        return dict(rowptr=rowptr, col=col, val=val, sub_off=sub_off, gid=gid, deg=deg)
+
+    def get_activation(self, l):
+        out = np.zeros((self.n_prime, self.dims[l]), dtype=np.float32)
+        self._ck(self._L.gad_get_activation(self._h, C.c_int32(l), _ptr(out, C.c_float)))
+        return out
+
+    def set_inputs(self, X=None, labels=None):
+        """gad_set_inputs.  X / labels may be numpy arrays or (pinned) CPU torch tensors; they must stay alive
+        until the stream has consumed them."""
+        def host_ptr(a, ctype, np_dtype):
+            if a is None:
+                return None, None
+            if hasattr(a, "data_ptr"):
+                return a, C.cast(C.c_void_p(a.data_ptr()), C.POINTER(ctype))
+            a = _arr(a, np_dtype)
+            return a, _ptr(a, ctype)
+        kx, px = host_ptr(X, C.c_float, np.float32)
+        kl, pl = host_ptr(labels, C.c_int32, np.int32)
+        self._keep = (kx, kl)
+        self._ck(self._L.gad_set_inputs(self._h, px, pl))
+
+    @property
+    def epoch(self):
+        e = C.c_int64(0)
+        self._ck(self._L.gad_get_epoch(self._h, C.byref(e)))
+        return int(e.value)
+
+    @epoch.setter
+    def epoch(self, e):
+        self._ck(self._L.gad_set_epoch(self._h, C.c_int64(e)))
+
+    # -- profiling -----------------------------------------------------------------------------
+    def profile_enable(self, on=True):
+        self._ck(self._L.gad_profile_enable(self._h, C.c_int32(1 if on else 0)))
+
+    def profile_reset(self):
+        self._ck(self._L.gad_profile_reset(self._h))
+
+    def profile_read(self):
+        """List of dicts: name, launches, total_ms, bytes_per_launch, flops_per_launch."""
+        cnt = C.c_int32(0)
+        self._ck(self._L.gad_profile_count(self._h, C.byref(cnt)))
+        out = []
+        for i in range(cnt.value):
+            name = C.create_string_buffer(64)
+            n, ms, by, fl = C.c_int64(0), C.c_double(0), C.c_double(0), C.c_double(0)
+            self._ck(self._L.gad_profile_read(self._h, C.c_int32(i), name, C.byref(n), C.byref(ms), C.byref(by), C.byref(fl)))
+            out.append(dict(name=name.value.decode(), launches=int(n.value), total_ms=float(ms.value),
+                            bytes_per_launch=float(by.value), flops_per_launch=float(fl.value)))
+        return out
+
+
+def from_workload(w, init_params, **kw):
+    """A context for a ``gad_synth.Workload``."""
+    cp, cn, hp, hn = w.flat_partition()
+    kw.setdefault("lr", w.lr)
+    return Gad(w.n, w.rowptr, w.col, cp, cn, hp, hn, w.X, w.labels, w.split, w.dims, init_params=init_params, **kw)

@@ -1,0 +1,659 @@
+// The C boundary (include/gad.h): context, workspace plan, create, and the per-epoch launch sequence.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "gad_internal.h"
+
+using namespace gad;
+
+namespace {
+
+struct ProfEntry {
+    std::string name;
+    int64_t launches = 0;
+    double ms = 0.0, bytes = 0.0, flops = 0.0;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> pending;
+};
+
+// Everything whose size follows from (n, K, subgraph sizes, nnz', dims): used by gad_workspace_bytes and by
+// gad_create, so both agree byte for byte.
+struct Plan {
+    int32_t n = 0, K = 0, L = 0;
+    int64_t Np = 0, nnz = 0, P = 0, Pint = 0, pstride = 0;
+    std::vector<int32_t> dims;
+    std::vector<Layer> layers;
+    std::vector<int32_t> ld;          // [L+1]
+    int32_t maxld = 0;
+    std::vector<RowSpan> tiles, chunks, core_spans;
+    std::vector<int32_t> chunk_ptr;   // [K+1]
+    int64_t dw_partial = 0;           // floats per chunk
+    size_t bytes = 0;
+    // offsets into the workspace
+    size_t o_rowptr, o_ecv, o_perm, o_hub, o_trowptr, o_tecv, o_tperm, o_thub, o_sub_off, o_gid, o_deg, o_label, o_train,
+        o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
+        o_dw_partial, o_cs_partial, o_loss_partial, o_zeta_partial, o_zeta, o_loss, o_flags, o_zeta_f, o_w_f, o_stage,
+        o_stage_lab;
+    std::vector<size_t> o_H;
+};
+
+size_t take(size_t& cur, size_t bytes) {
+    size_t o = cur;
+    cur += (size_t)round_up((int64_t)std::max<size_t>(bytes, 4), 256);
+    return o;
+}
+
+int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off, const std::vector<int64_t>& core_count,
+              int64_t nnz, const gad_config* cfg, std::string& err) {
+    if (!cfg || cfg->L < 1 || !cfg->dims) { err = "config needs L >= 1 and dims"; return GAD_ERR_ARG; }
+    for (int l = 0; l <= cfg->L; ++l)
+        if (cfg->dims[l] < 1) { err = "layer size must be positive"; return GAD_ERR_ARG; }
+    if (!(cfg->dropout >= 0.f && cfg->dropout < 1.f)) { err = "dropout must be in [0,1)"; return GAD_ERR_ARG; }
+    if (cfg->gemm_mode != 0 && cfg->gemm_mode != 1) { err = "gemm_mode must be 0 or 1"; return GAD_ERR_ARG; }
+    if (cfg->zeta_mode == 1) { err = "zeta_mode 1 (pairwise form) is not implemented"; return GAD_ERR_UNSUPPORTED; }
+    if (cfg->zeta_mode != 0) { err = "zeta_mode must be 0 or 1"; return GAD_ERR_ARG; }
+    if (!(cfg->beta > 0.f)) { err = "beta must be positive"; return GAD_ERR_ARG; }
+    p.n = n; p.K = K; p.L = cfg->L; p.nnz = nnz; p.Np = sub_off[K];
+    p.dims.assign(cfg->dims, cfg->dims + cfg->L + 1);
+    p.ld.resize(p.L + 1);
+    p.maxld = 0;
+    for (int l = 0; l <= p.L; ++l) { p.ld[l] = (int32_t)round_up(p.dims[l], 4); p.maxld = std::max(p.maxld, p.ld[l]); }
+    p.layers.resize(p.L);
+    int64_t oi = 0, oe = 0;
+    p.dw_partial = 0;
+    for (int l = 0; l < p.L; ++l) {
+        Layer& y = p.layers[l];
+        y.fi = p.dims[l]; y.fo = p.dims[l + 1]; y.ldi = p.ld[l]; y.ldo = p.ld[l + 1]; y.ldw = p.ld[l + 1];
+        y.w_int = oi; oi += (int64_t)y.fi * y.ldw;
+        y.b_int = oi; oi += y.ldo;
+        y.w_ext = oe; oe += (int64_t)y.fi * y.fo;
+        y.b_ext = oe; oe += y.fo;
+        p.dw_partial = std::max(p.dw_partial, (int64_t)y.fi * y.ldw);
+    }
+    p.P = oe; p.Pint = oi; p.pstride = round_up(oi, 64);
+    // row tiles of the grouped transforms (128 rows, never across subgraphs) and reduction chunks
+    const int64_t target = 592;
+    int64_t R = round_up(std::max<int64_t>(1, (p.Np + target - 1) / target), 32);
+    R = std::min<int64_t>(std::max<int64_t>(R, 128), 16384);
+    p.chunk_ptr.assign(K + 1, 0);
+    for (int32_t k = 0; k < K; ++k) {
+        for (int32_t r = sub_off[k]; r < sub_off[k + 1]; r += 128)
+            p.tiles.push_back(RowSpan{r, std::min<int32_t>(128, sub_off[k + 1] - r), k, 0});
+        for (int64_t r = sub_off[k]; r < sub_off[k + 1]; r += R)
+            p.chunks.push_back(RowSpan{(int32_t)r, (int32_t)std::min<int64_t>(R, sub_off[k + 1] - r), k, 0});
+        p.chunk_ptr[k + 1] = (int32_t)p.chunks.size();
+        for (int64_t r = 0; r < core_count[k]; r += 256)
+            p.core_spans.push_back(RowSpan{(int32_t)(sub_off[k] + r), (int32_t)std::min<int64_t>(256, core_count[k] - r), k, 0});
+    }
+    const size_t Np = (size_t)p.Np, nc = p.chunks.size();
+    size_t cur = 0;
+    p.o_rowptr = take(cur, 8 * (Np + 1)); p.o_ecv = take(cur, 8 * (size_t)nnz);
+    p.o_perm = take(cur, 4 * Np); p.o_hub = take(cur, 4 * Np);
+    p.o_trowptr = take(cur, 8 * (Np + 1)); p.o_tecv = take(cur, 8 * (size_t)nnz);
+    p.o_tperm = take(cur, 4 * Np); p.o_thub = take(cur, 4 * Np);
+    p.o_sub_off = take(cur, 4 * (size_t)(K + 1)); p.o_gid = take(cur, 4 * Np); p.o_deg = take(cur, 4 * Np);
+    p.o_label = take(cur, 4 * Np); p.o_train = take(cur, Np);
+    p.o_deg_sum = take(cur, 8 * (size_t)K); p.o_deg_sq = take(cur, 8 * (size_t)K); p.o_inv_ntrain = take(cur, 4 * (size_t)K);
+    p.o_tiles = take(cur, sizeof(RowSpan) * p.tiles.size()); p.o_chunks = take(cur, sizeof(RowSpan) * nc);
+    p.o_chunk_ptr = take(cur, 4 * (size_t)(K + 1)); p.o_core_spans = take(cur, sizeof(RowSpan) * p.core_spans.size());
+    p.o_H.resize(p.L + 1);
+    for (int l = 0; l <= p.L; ++l) p.o_H[l] = take(cur, 4 * Np * (size_t)p.ld[l]);
+    p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
+    p.o_params = take(cur, 4 * (size_t)K * (size_t)p.pstride); p.o_grads = take(cur, 4 * (size_t)K * (size_t)p.pstride);
+    p.o_dw_partial = take(cur, 4 * nc * (size_t)p.dw_partial); p.o_cs_partial = take(cur, 4 * nc * (size_t)p.maxld);
+    p.o_loss_partial = take(cur, 4 * nc); p.o_zeta_partial = take(cur, 8 * nc * 2 * (size_t)p.ld[0]);
+    p.o_zeta = take(cur, 8 * (size_t)K); p.o_loss = take(cur, 4 * (size_t)(K + 1)); p.o_flags = take(cur, 16);
+    p.o_zeta_f = take(cur, 4 * (size_t)K); p.o_w_f = take(cur, 4 * (size_t)K);
+    p.o_stage = take(cur, 4 * (size_t)n * (size_t)std::max(p.dims[0], p.dims[p.L])); p.o_stage_lab = take(cur, 4 * (size_t)n);
+    p.bytes = cur;
+    return GAD_OK;
+}
+
+}  // namespace
+
+struct gad_ctx {
+    cudaStream_t stream = nullptr;
+    char* ws = nullptr;
+    Plan p;
+    gad_config cfg{};
+    std::string err;
+    bool symmetric = false;
+    SparseDev A, At;
+    int64_t epoch = 0;
+    std::vector<int32_t> sub_off, gid;
+    std::vector<int64_t> ntrain;
+    int64_t ntrain_total = 0;
+    bool profiling = false;
+    std::vector<ProfEntry> prof;
+    std::vector<float> host_block;  // staging for parameter pack / unpack
+
+    template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+    float* H(int l) const { return at<float>(p.o_H[l]); }
+};
+
+namespace {
+
+thread_local std::string g_last_error;  // also readable after a failed gad_create, when there is no context
+
+int fail(gad_ctx* c, int code, const std::string& msg) {
+    if (c) c->err = msg;
+    g_last_error = msg;
+    return code;
+}
+#define GAD_CK(call)                                                                                       \
+    do {                                                                                                   \
+        cudaError_t e_ = (call);                                                                           \
+        if (e_ != cudaSuccess)                                                                             \
+            return fail(ctx, GAD_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_));            \
+    } while (0)
+
+ProfEntry& prof_entry(gad_ctx* c, const char* name, int layer, double bytes, double flops) {
+    char buf[64];
+    if (layer >= 0) snprintf(buf, sizeof buf, "%s_l%d", name, layer); else snprintf(buf, sizeof buf, "%s", name);
+    for (auto& e : c->prof) if (e.name == buf) return e;
+    c->prof.push_back(ProfEntry{});
+    c->prof.back().name = buf;
+    c->prof.back().bytes = bytes;
+    c->prof.back().flops = flops;
+    return c->prof.back();
+}
+
+// Runs one launcher, optionally bracketed by events on the context's stream.
+template <class F>
+int run(gad_ctx* ctx, const char* name, int layer, double bytes, double flops, F&& launch) {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (ctx->profiling) {
+        GAD_CK(cudaEventCreate(&e0));
+        GAD_CK(cudaEventCreate(&e1));
+        GAD_CK(cudaEventRecord(e0, ctx->stream));
+    }
+    cudaError_t e = launch();
+    if (e != cudaSuccess) return fail(ctx, GAD_ERR_CUDA, std::string(name) + ": " + cudaGetErrorString(e));
+    if (ctx->profiling) {
+        GAD_CK(cudaEventRecord(e1, ctx->stream));
+        prof_entry(ctx, name, layer, bytes, flops).pending.emplace_back(e0, e1);
+    }
+    return GAD_OK;
+}
+#define GAD_RUN(...)                            \
+    do {                                        \
+        int rc_ = run(ctx, __VA_ARGS__);        \
+        if (rc_ != GAD_OK) return rc_;          \
+    } while (0)
+
+double spmm_bytes(const Plan& p, int F) { return 8.0 * p.nnz + 8.0 * p.Np + 8.0 * (double)p.Np * F; }
+
+int forward_pass(gad_ctx* ctx, bool train) {
+    const Plan& p = ctx->p;
+    float* Z = ctx->at<float>(p.o_G2);
+    const float* params = ctx->at<float>(p.o_params);
+    for (int l = 0; l < p.L; ++l) {
+        const Layer& y = p.layers[l];
+        GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+            return launch_gemm_rows_simt(0, ctx->H(l), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, Z, y.ldo,
+                                         ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, ctx->stream);
+        });
+        Epilogue ep{params, p.pstride, y.b_int, ctx->at<int32_t>(p.o_sub_off), p.K, l < p.L - 1 ? 1 : 0,
+                    train ? ctx->cfg.dropout : 0.f, ctx->cfg.seed, ctx->epoch, l};
+        GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
+                [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, ctx->stream); });
+    }
+    return GAD_OK;
+}
+
+int zeta_pass(gad_ctx* ctx) {
+    const Plan& p = ctx->p;
+    GAD_RUN("zeta_partial", -1, 4.0 * p.Np * (p.dims[0] + 1), 4.0 * p.Np * p.dims[0], [&] {
+        return launch_zeta_partial(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
+                                   (int)p.chunks.size(), ctx->at<int32_t>(p.o_sub_off), ctx->at<int64_t>(p.o_deg_sum),
+                                   ctx->at<double>(p.o_zeta_partial), ctx->stream);
+    });
+    GAD_RUN("zeta_final", -1, 16.0 * p.chunks.size() * p.ld[0], 0.0, [&] {
+        return launch_zeta_final(ctx->at<double>(p.o_zeta_partial), p.dims[0], p.ld[0], ctx->at<int32_t>(p.o_chunk_ptr), p.K,
+                                 ctx->at<int32_t>(p.o_sub_off), ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_deg_sq),
+                                 ctx->cfg.beta, ctx->at<double>(p.o_zeta), ctx->stream);
+    });
+    return GAD_OK;
+}
+
+int backward_pass(gad_ctx* ctx) {
+    const Plan& p = ctx->p;
+    float* G1 = ctx->at<float>(p.o_G1);
+    float* G2 = ctx->at<float>(p.o_G2);
+    float* grads = ctx->at<float>(p.o_grads);
+    const float* params = ctx->at<float>(p.o_params);
+    const RowSpan* chunks = ctx->at<RowSpan>(p.o_chunks);
+    const int nc = (int)p.chunks.size();
+    const int32_t* chunk_ptr = ctx->at<int32_t>(p.o_chunk_ptr);
+    const float scale = ctx->cfg.dropout > 0.f ? 1.f / (1.f - ctx->cfg.dropout) : 1.f;
+    for (int l = p.L - 1; l >= 0; --l) {
+        const Layer& y = p.layers[l];
+        GAD_RUN("bias_grad", l, 4.0 * p.Np * y.fo, 1.0 * p.Np * y.fo, [&] {
+            cudaError_t e = launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, ctx->stream);
+            if (e != cudaSuccess) return e;
+            return launch_reduce_chunks(ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr, p.K, grads, p.pstride, y.b_int, y.ldo,
+                                        ctx->stream);
+        });
+        GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
+                [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
+        GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+            cudaError_t e = launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, chunks, nc, ctx->at<float>(p.o_dw_partial),
+                                                y.ldw, ctx->stream);
+            if (e != cudaSuccess) return e;
+            return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, chunk_ptr, p.K, grads, p.pstride,
+                                        y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
+        });
+        if (l > 0)
+            GAD_RUN("gemm_dh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+                return launch_gemm_rows_simt(1, G2, y.ldo, y.fo, params, p.pstride, y.w_int, y.ldw, y.fi, G1, y.ldi,
+                                             ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), ctx->H(l), y.ldi, scale,
+                                             ctx->stream);
+            });
+    }
+    return GAD_OK;
+}
+
+void pack_params(const Plan& p, const float* ext, float* blk) {
+    std::fill(blk, blk + p.pstride, 0.f);
+    for (const Layer& y : p.layers) {
+        for (int i = 0; i < y.fi; ++i)
+            std::memcpy(blk + y.w_int + (int64_t)i * y.ldw, ext + y.w_ext + (int64_t)i * y.fo, sizeof(float) * y.fo);
+        std::memcpy(blk + y.b_int, ext + y.b_ext, sizeof(float) * y.fo);
+    }
+}
+void unpack_params(const Plan& p, const float* blk, float* ext) {
+    for (const Layer& y : p.layers) {
+        for (int i = 0; i < y.fi; ++i)
+            std::memcpy(ext + y.w_ext + (int64_t)i * y.fo, blk + y.w_int + (int64_t)i * y.ldw, sizeof(float) * y.fo);
+        std::memcpy(ext + y.b_ext, blk + y.b_int, sizeof(float) * y.fo);
+    }
+}
+
+uint64_t host_mix64(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ULL;
+    z = (z ^ (z >> 27)) * 0x94d049bb133111ebULL;
+    return z ^ (z >> 31);
+}
+
+int upload_sparse(gad_ctx* ctx, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col, const std::vector<float>& val,
+                  size_t o_rowptr, size_t o_ecv, size_t o_perm, size_t o_hub, SparseDev& out) {
+    const Plan& p = ctx->p;
+    std::vector<uint2> ecv(col.size());
+    for (size_t e = 0; e < col.size(); ++e) {
+        uint32_t bits;
+        std::memcpy(&bits, &val[e], 4);
+        ecv[e] = make_uint2((uint32_t)col[e], bits);
+    }
+    std::vector<int32_t> perm, hub;
+    bin_rows(rowptr, 2048, perm, hub);
+    GAD_CK(cudaMemcpyAsync(ctx->ws + o_rowptr, rowptr.data(), 8 * rowptr.size(), cudaMemcpyHostToDevice, ctx->stream));
+    if (!ecv.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_ecv, ecv.data(), 8 * ecv.size(), cudaMemcpyHostToDevice, ctx->stream));
+    if (!perm.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_perm, perm.data(), 4 * perm.size(), cudaMemcpyHostToDevice, ctx->stream));
+    if (!hub.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_hub, hub.data(), 4 * hub.size(), cudaMemcpyHostToDevice, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));  // the host vectors above go out of scope
+    out.rowptr = ctx->at<int64_t>(o_rowptr);
+    out.ecv = ctx->at<uint2>(o_ecv);
+    out.perm = ctx->at<int32_t>(o_perm);
+    out.hub = ctx->at<int32_t>(o_hub);
+    out.nperm = (int32_t)perm.size();
+    out.nhub = (int32_t)hub.size();
+    (void)p;
+    return GAD_OK;
+}
+
+template <class T>
+int upload(gad_ctx* ctx, size_t off, const std::vector<T>& v) {
+    if (!v.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + off, v.data(), sizeof(T) * v.size(), cudaMemcpyHostToDevice, ctx->stream));
+    return GAD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gad_workspace_bytes(const gad_csr* g, const gad_partition* part, const gad_config* cfg, size_t* bytes) {
+    if (!bytes) return GAD_ERR_ARG;
+    std::string err;
+    int64_t Np = 0, nnz = 0;
+    int rc = store_sizes(g, part, &Np, &nnz, err);
+    if (rc != GAD_OK) return fail(nullptr, rc, err);
+    std::vector<int32_t> sub_off(part->K + 1, 0);
+    std::vector<int64_t> core_count(part->K, 0);
+    for (int32_t k = 0; k < part->K; ++k) {
+        core_count[k] = part->core_ptr[k + 1] - part->core_ptr[k];
+        sub_off[k + 1] = sub_off[k] + (int32_t)(core_count[k] + part->halo_ptr[k + 1] - part->halo_ptr[k]);
+    }
+    Plan p;
+    rc = make_plan(p, g->n, part->K, sub_off, core_count, nnz, cfg, err);
+    if (rc != GAD_OK) return fail(nullptr, rc, err);
+    *bytes = p.bytes;
+    return GAD_OK;
+}
+
+int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const float* X, const int32_t* labels,
+               const uint8_t* split, const gad_config* cfg, const float* init_params, void* workspace, size_t workspace_bytes,
+               void* stream) {
+    if (!out) return GAD_ERR_ARG;
+    *out = nullptr;
+    if (!g || !part || !X || !labels || !split || !cfg || !workspace) return GAD_ERR_ARG;
+    if (((uintptr_t)workspace & 255) != 0) return GAD_ERR_ARG;
+    gad_ctx* ctx = new (std::nothrow) gad_ctx();
+    if (!ctx) return GAD_ERR_OOM;
+    struct Guard { gad_ctx*& c; bool ok = false; ~Guard() { if (!ok) { delete c; c = nullptr; } } } guard{ctx};
+    ctx->stream = (cudaStream_t)stream;
+    ctx->ws = (char*)workspace;
+    ctx->cfg = *cfg;
+    HostStore st;
+    int rc = build_store(g, part, true, st, ctx->err);
+    if (rc != GAD_OK) return fail(ctx, rc, ctx->err);
+    rc = make_plan(ctx->p, g->n, part->K, st.sub_off, st.core_count, st.nnz, cfg, ctx->err);
+    if (rc != GAD_OK) return fail(ctx, rc, ctx->err);
+    ctx->cfg.dims = ctx->p.dims.data();
+    const Plan& p = ctx->p;
+    if (workspace_bytes < p.bytes) return fail(ctx, GAD_ERR_OOM, "workspace smaller than gad_workspace_bytes");
+    const int C = p.dims[p.L];
+    for (int32_t u = 0; u < g->n; ++u) {
+        if (labels[u] < 0 || labels[u] >= C) return fail(ctx, GAD_ERR_RANGE, "label out of range");
+        if (split[u] > 2) return fail(ctx, GAD_ERR_RANGE, "split value out of range");
+    }
+    ctx->symmetric = st.symmetric;
+    ctx->sub_off = st.sub_off;
+    ctx->gid = st.gid;
+
+    rc = upload_sparse(ctx, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_perm, p.o_hub, ctx->A);
+    if (rc != GAD_OK) return rc;
+    if (!st.symmetric) {
+        rc = upload_sparse(ctx, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tperm, p.o_thub, ctx->At);
+        if (rc != GAD_OK) return rc;
+    }
+    // per-row labels and loss mask, per-subgraph degree sums and training counts
+    std::vector<int32_t> label((size_t)p.Np);
+    std::vector<uint8_t> train((size_t)p.Np);
+    std::vector<int64_t> deg_sum(p.K, 0), deg_sq(p.K, 0);
+    std::vector<float> inv_ntrain(p.K, 0.f);
+    ctx->ntrain.assign(p.K, 0);
+    ctx->ntrain_total = 0;
+    for (int32_t k = 0; k < p.K; ++k) {
+        for (int64_t r = st.sub_off[k]; r < st.sub_off[k + 1]; ++r) {
+            const int32_t u = st.gid[r];
+            label[r] = labels[u];
+            const bool core = (r - st.sub_off[k]) < st.core_count[k];
+            train[r] = (uint8_t)(core && split[u] == 0);
+            ctx->ntrain[k] += train[r];
+            deg_sum[k] += st.deg[r];
+            deg_sq[k] += (int64_t)st.deg[r] * st.deg[r];
+        }
+        inv_ntrain[k] = ctx->ntrain[k] > 0 ? 1.f / (float)ctx->ntrain[k] : 0.f;
+        ctx->ntrain_total += ctx->ntrain[k];
+    }
+    if ((rc = upload(ctx, p.o_sub_off, st.sub_off)) || (rc = upload(ctx, p.o_gid, st.gid)) || (rc = upload(ctx, p.o_deg, st.deg)) ||
+        (rc = upload(ctx, p.o_label, label)) || (rc = upload(ctx, p.o_train, train)) || (rc = upload(ctx, p.o_deg_sum, deg_sum)) ||
+        (rc = upload(ctx, p.o_deg_sq, deg_sq)) || (rc = upload(ctx, p.o_inv_ntrain, inv_ntrain)) ||
+        (rc = upload(ctx, p.o_tiles, p.tiles)) || (rc = upload(ctx, p.o_chunks, p.chunks)) ||
+        (rc = upload(ctx, p.o_chunk_ptr, p.chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)))
+        return rc;
+    // features: graph order -> staging -> store-row order with zero pad columns
+    GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage, X, 4 * (size_t)g->n * p.dims[0], cudaMemcpyHostToDevice, ctx->stream));
+    GAD_CK(launch_gather_rows(ctx->at<float>(p.o_stage), p.dims[0], ctx->at<int32_t>(p.o_gid), p.Np, ctx->H(0), p.ld[0], ctx->stream));
+    // parameters: K identical padded copies
+    std::vector<float> ext((size_t)p.P);
+    if (init_params) {
+        std::memcpy(ext.data(), init_params, sizeof(float) * (size_t)p.P);
+    } else {
+        uint64_t ctr = 0;
+        for (const Layer& y : p.layers) {
+            const double a = std::sqrt(6.0 / (y.fi + y.fo));
+            for (int64_t i = 0; i < (int64_t)y.fi * y.fo; ++i) {
+                uint64_t h = host_mix64(cfg->seed + 0x9e3779b97f4a7c15ULL * (++ctr));
+                ext[y.w_ext + i] = (float)((2.0 * ((h >> 11) * (1.0 / 9007199254740992.0)) - 1.0) * a);
+            }
+            for (int j = 0; j < y.fo; ++j) ext[y.b_ext + j] = 0.f;
+        }
+    }
+    ctx->host_block.assign((size_t)p.pstride, 0.f);
+    pack_params(p, ext.data(), ctx->host_block.data());
+    for (int32_t k = 0; k < p.K; ++k)
+        GAD_CK(cudaMemcpyAsync(ctx->at<float>(p.o_params) + (int64_t)k * p.pstride, ctx->host_block.data(), 4 * (size_t)p.pstride,
+                               cudaMemcpyHostToDevice, ctx->stream));
+    GAD_CK(cudaMemsetAsync(ctx->ws + p.o_grads, 0, 4 * (size_t)p.K * p.pstride, ctx->stream));
+    GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 16, ctx->stream));
+    GAD_CK(cudaMemsetAsync(ctx->ws + p.o_loss, 0, 4 * (size_t)(p.K + 1), ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    guard.ok = true;
+    *out = ctx;
+    return GAD_OK;
+}
+
+int gad_get_loss(gad_ctx* ctx, float* loss_out) {
+    if (!ctx || !loss_out) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    int32_t flag = 0;
+    GAD_CK(cudaMemcpyAsync(loss_out, ctx->ws + p.o_loss, 4 * (size_t)(p.K + 1), cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaMemcpyAsync(&flag, ctx->ws + p.o_flags, 4, cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    if (flag) {
+        GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 4, ctx->stream));
+        return fail(ctx, GAD_ERR_NONFINITE, "a subgraph loss is NaN or infinite");
+    }
+    return GAD_OK;
+}
+
+int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
+    if (!ctx) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    int rc = forward_pass(ctx, true);
+    if (rc != GAD_OK) return rc;
+    const int C = p.dims[p.L];
+    GAD_RUN("softmax_xent", -1, 8.0 * p.Np * C, 0.0, [&] {
+        cudaError_t e = launch_softmax_xent(ctx->H(p.L), p.ld[p.L], C, ctx->at<int32_t>(p.o_label), ctx->at<uint8_t>(p.o_train),
+                                            ctx->at<RowSpan>(p.o_chunks), (int)p.chunks.size(), ctx->at<float>(p.o_inv_ntrain),
+                                            ctx->at<float>(p.o_G1), ctx->at<float>(p.o_loss_partial), ctx->stream);
+        if (e != cudaSuccess) return e;
+        return launch_loss_final(ctx->at<float>(p.o_loss_partial), ctx->at<int32_t>(p.o_chunk_ptr), p.K, ctx->at<float>(p.o_inv_ntrain),
+                                 ctx->ntrain_total > 0 ? 1.f / (float)ctx->ntrain_total : 0.f, ctx->at<float>(p.o_loss),
+                                 ctx->at<int32_t>(p.o_flags), ctx->stream);
+    });
+    if ((rc = backward_pass(ctx)) != GAD_OK) return rc;
+    if ((rc = zeta_pass(ctx)) != GAD_OK) return rc;
+    GAD_RUN("sgd_consensus", -1, 12.0 * p.K * p.Pint, 4.0 * p.K * p.Pint, [&] {
+        return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
+                                    ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->stream);
+    });
+    ctx->epoch += 1;
+    if (loss_out) return gad_get_loss(ctx, loss_out);
+    return GAD_OK;
+}
+
+int gad_forward(gad_ctx* ctx, float* logits_out) {
+    if (!ctx || !logits_out) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    int rc = forward_pass(ctx, false);
+    if (rc != GAD_OK) return rc;
+    const int C = p.dims[p.L];
+    GAD_CK(cudaMemsetAsync(ctx->ws + p.o_stage, 0, 4 * (size_t)p.n * C, ctx->stream));
+    GAD_CK(launch_scatter_core(ctx->H(p.L), p.ld[p.L], C, ctx->at<int32_t>(p.o_gid), ctx->at<RowSpan>(p.o_core_spans),
+                               (int)p.core_spans.size(), ctx->at<float>(p.o_stage), ctx->stream));
+    GAD_CK(cudaMemcpyAsync(logits_out, ctx->ws + p.o_stage, 4 * (size_t)p.n * C, cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    return GAD_OK;
+}
+
+int gad_subgraph_weights(gad_ctx* ctx, float* zeta_out, float* w_out) {
+    if (!ctx) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    int rc = zeta_pass(ctx);
+    if (rc != GAD_OK) return rc;
+    GAD_CK(launch_weights(ctx->at<double>(p.o_zeta), p.K, ctx->cfg.weighted, ctx->at<float>(p.o_zeta_f), ctx->at<float>(p.o_w_f),
+                          ctx->stream));
+    if (zeta_out) GAD_CK(cudaMemcpyAsync(zeta_out, ctx->ws + p.o_zeta_f, 4 * (size_t)p.K, cudaMemcpyDeviceToHost, ctx->stream));
+    if (w_out) GAD_CK(cudaMemcpyAsync(w_out, ctx->ws + p.o_w_f, 4 * (size_t)p.K, cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    return GAD_OK;
+}
+
+int gad_consensus(gad_ctx* ctx) {
+    if (!ctx) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    int rc = zeta_pass(ctx);
+    if (rc != GAD_OK) return rc;
+    GAD_RUN("consensus", -1, 8.0 * p.K * p.Pint, 2.0 * p.K * p.Pint, [&] {
+        return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, 0.f,
+                                    ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 0, ctx->stream);
+    });
+    return GAD_OK;
+}
+
+int gad_param_count(const gad_ctx* ctx, int64_t* P) {
+    if (!ctx || !P) return GAD_ERR_ARG;
+    *P = ctx->p.P;
+    return GAD_OK;
+}
+
+static int get_block(gad_ctx* ctx, size_t base, int32_t k, float* out) {
+    if (!ctx || !out || k < 0 || k >= ctx->p.K) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    GAD_CK(cudaMemcpyAsync(ctx->host_block.data(), ctx->at<float>(base) + (int64_t)k * p.pstride, 4 * (size_t)p.pstride,
+                           cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    unpack_params(p, ctx->host_block.data(), out);
+    return GAD_OK;
+}
+int gad_get_params(gad_ctx* ctx, int32_t k, float* out) { return get_block(ctx, ctx ? ctx->p.o_params : 0, k, out); }
+int gad_get_grads(gad_ctx* ctx, int32_t k, float* out) { return get_block(ctx, ctx ? ctx->p.o_grads : 0, k, out); }
+
+int gad_set_params(gad_ctx* ctx, int32_t k, const float* in) {
+    if (!ctx || !in || k < 0 || k >= ctx->p.K) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    pack_params(p, in, ctx->host_block.data());
+    GAD_CK(cudaMemcpyAsync(ctx->at<float>(p.o_params) + (int64_t)k * p.pstride, ctx->host_block.data(), 4 * (size_t)p.pstride,
+                           cudaMemcpyHostToDevice, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    return GAD_OK;
+}
+
+int gad_store_sizes(const gad_ctx* ctx, int64_t* n_prime, int64_t* nnz_prime) {
+    if (!ctx) return GAD_ERR_ARG;
+    if (n_prime) *n_prime = ctx->p.Np;
+    if (nnz_prime) *nnz_prime = ctx->p.nnz;
+    return GAD_OK;
+}
+
+int gad_get_store(gad_ctx* ctx, int64_t* rowptr, int32_t* col, float* val, int32_t* sub_off, int32_t* gid, int32_t* deg) {
+    if (!ctx) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    if (rowptr) GAD_CK(cudaMemcpyAsync(rowptr, ctx->ws + p.o_rowptr, 8 * (size_t)(p.Np + 1), cudaMemcpyDeviceToHost, ctx->stream));
+    if (sub_off) GAD_CK(cudaMemcpyAsync(sub_off, ctx->ws + p.o_sub_off, 4 * (size_t)(p.K + 1), cudaMemcpyDeviceToHost, ctx->stream));
+    if (gid && p.Np) GAD_CK(cudaMemcpyAsync(gid, ctx->ws + p.o_gid, 4 * (size_t)p.Np, cudaMemcpyDeviceToHost, ctx->stream));
+    if (deg && p.Np) GAD_CK(cudaMemcpyAsync(deg, ctx->ws + p.o_deg, 4 * (size_t)p.Np, cudaMemcpyDeviceToHost, ctx->stream));
+    std::vector<uint2> ecv;
+    if ((col || val) && p.nnz) {
+        ecv.resize((size_t)p.nnz);
+        GAD_CK(cudaMemcpyAsync(ecv.data(), ctx->ws + p.o_ecv, 8 * (size_t)p.nnz, cudaMemcpyDeviceToHost, ctx->stream));
+    }
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    for (size_t e = 0; e < ecv.size(); ++e) {
+        if (col) col[e] = (int32_t)ecv[e].x;
+        if (val) std::memcpy(&val[e], &ecv[e].y, 4);
+    }
+    return GAD_OK;
+}
+
+int gad_get_activation(gad_ctx* ctx, int32_t l, float* out) {
+    if (!ctx || !out || l < 0 || l > ctx->p.L) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    if (p.Np == 0) return GAD_OK;
+    GAD_CK(cudaMemcpy2DAsync(out, 4 * (size_t)p.dims[l], ctx->H(l), 4 * (size_t)p.ld[l], 4 * (size_t)p.dims[l], (size_t)p.Np,
+                             cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    return GAD_OK;
+}
+
+int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels) {
+    if (!ctx) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    if (X) {
+        GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage, X, 4 * (size_t)p.n * p.dims[0], cudaMemcpyHostToDevice, ctx->stream));
+        GAD_RUN("gather_features", -1, 8.0 * p.Np * p.dims[0], 0.0, [&] {
+            return launch_gather_rows(ctx->at<float>(p.o_stage), p.dims[0], ctx->at<int32_t>(p.o_gid), p.Np, ctx->H(0), p.ld[0],
+                                      ctx->stream);
+        });
+    }
+    if (labels) {
+        GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage_lab, labels, 4 * (size_t)p.n, cudaMemcpyHostToDevice, ctx->stream));
+        GAD_RUN("gather_labels", -1, 8.0 * p.Np, 0.0, [&] {
+            return launch_gather_labels(ctx->at<int32_t>(p.o_stage_lab), ctx->at<int32_t>(p.o_gid), p.Np, ctx->at<int32_t>(p.o_label),
+                                        ctx->stream);
+        });
+    }
+    return GAD_OK;
+}
+
+int gad_get_epoch(const gad_ctx* ctx, int64_t* epoch) {
+    if (!ctx || !epoch) return GAD_ERR_ARG;
+    *epoch = ctx->epoch;
+    return GAD_OK;
+}
+int gad_set_epoch(gad_ctx* ctx, int64_t epoch) {
+    if (!ctx || epoch < 0) return GAD_ERR_ARG;
+    ctx->epoch = epoch;
+    return GAD_OK;
+}
+
+static int prof_drain(gad_ctx* ctx) {
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    for (auto& e : ctx->prof) {
+        for (auto& pr : e.pending) {
+            float ms = 0.f;
+            GAD_CK(cudaEventElapsedTime(&ms, pr.first, pr.second));
+            e.ms += ms;
+            e.launches += 1;
+            cudaEventDestroy(pr.first);
+            cudaEventDestroy(pr.second);
+        }
+        e.pending.clear();
+    }
+    return GAD_OK;
+}
+
+int gad_profile_enable(gad_ctx* ctx, int32_t on) {
+    if (!ctx) return GAD_ERR_ARG;
+    ctx->profiling = on != 0;
+    return GAD_OK;
+}
+int gad_profile_reset(gad_ctx* ctx) {
+    if (!ctx) return GAD_ERR_ARG;
+    int rc = prof_drain(ctx);
+    ctx->prof.clear();
+    return rc;
+}
+int gad_profile_count(const gad_ctx* ctx, int32_t* count) {
+    if (!ctx || !count) return GAD_ERR_ARG;
+    *count = (int32_t)ctx->prof.size();
+    return GAD_OK;
+}
+int gad_profile_read(gad_ctx* ctx, int32_t i, char* name64, int64_t* launches, double* total_ms, double* bytes_per_launch,
+                     double* flops_per_launch) {
+    if (!ctx || i < 0 || i >= (int32_t)ctx->prof.size()) return GAD_ERR_ARG;
+    int rc = prof_drain(ctx);
+    if (rc != GAD_OK) return rc;
+    const ProfEntry& e = ctx->prof[i];
+    if (name64) { std::strncpy(name64, e.name.c_str(), 63); name64[63] = 0; }
+    if (launches) *launches = e.launches;
+    if (total_ms) *total_ms = e.ms;
+    if (bytes_per_launch) *bytes_per_launch = e.bytes;
+    if (flops_per_launch) *flops_per_launch = e.flops;
+    return GAD_OK;
+}
+
+const char* gad_last_error(const gad_ctx* ctx) { return ctx ? ctx->err.c_str() : g_last_error.c_str(); }
+
+void gad_destroy(gad_ctx* ctx) {
+    if (!ctx) return;
+    for (auto& e : ctx->prof)
+        for (auto& pr : e.pending) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
+    delete ctx;
+}
+
+}  // extern "C"

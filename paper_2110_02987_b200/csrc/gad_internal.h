@@ -1,0 +1,126 @@
+// Internal declarations shared by the translation units of the library (not part of the boundary).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/gad.h"
+
+namespace gad {
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// ---------------------------------------------------------------------------------------------
+// Host-side result of building the block-diagonal store (create-time, not on the timed path).
+// ---------------------------------------------------------------------------------------------
+struct HostStore {
+    int32_t K = 0;
+    int64_t Np = 0, nnz = 0;
+    std::vector<int64_t> rowptr;   // [Np+1]
+    std::vector<int32_t> col;      // [nnz] store-row ids, ascending inside a row
+    std::vector<float> val;        // [nnz] A~ entries, computed in double and rounded once
+    std::vector<int32_t> sub_off;  // [K+1]
+    std::vector<int32_t> gid;      // [Np]
+    std::vector<int32_t> deg;      // [Np] local degree, self-loop excluded
+    std::vector<int64_t> core_count;  // [K]
+    bool symmetric = false;        // A~ equals its transpose entry by entry
+    std::vector<int64_t> t_rowptr; // transposed store (empty when symmetric)
+    std::vector<int32_t> t_col;
+    std::vector<float> t_val;
+};
+
+// Validates the inputs and fills the store; returns a GAD_* status and a message.
+int build_store(const gad_csr* g, const gad_partition* part, bool values, HostStore& out, std::string& err);
+// Sizes only (for gad_workspace_bytes).
+int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, std::string& err);
+
+// Rows ordered for the SpMM launch: rows with at least `hub_nnz` entries go to the hub list (one CTA each),
+// the others are binned by floor(log2(nnz)), heaviest bin first, ascending row id inside a bin.
+void bin_rows(const std::vector<int64_t>& rowptr, int64_t hub_nnz, std::vector<int32_t>& perm,
+              std::vector<int32_t>& hub);
+
+// ---------------------------------------------------------------------------------------------
+// Device views
+// ---------------------------------------------------------------------------------------------
+struct SparseDev {
+    const int64_t* rowptr = nullptr;  // [Np+1]
+    const uint2* ecv = nullptr;       // [nnz] packed (column, value bits)
+    const int32_t* perm = nullptr;    // binned non-hub rows
+    const int32_t* hub = nullptr;     // hub rows
+    int32_t nperm = 0, nhub = 0;
+};
+
+struct Layer {
+    int32_t fi, fo;        // F_l, F_{l+1}
+    int32_t ldi, ldo;      // leading dimensions of H^(l), H^(l+1) (multiples of 4 floats)
+    int32_t ldw;           // leading dimension of W_l rows inside the padded parameter block
+    int64_t w_int, b_int;  // offsets inside one replica's padded parameter block (multiples of 4 floats)
+    int64_t w_ext, b_ext;  // offsets inside the caller-visible [P] layout
+};
+
+// A run of rows that belongs to one subgraph: {first row, row count, subgraph, unused}.
+struct RowSpan { int32_t row0, nrows, k, pad; };
+
+struct Epilogue {            // of the forward SpMM: bias, ReLU, dropout
+    const float* params;     // padded parameter blocks
+    int64_t pstride;         // floats between replicas
+    int64_t b_int;           // bias offset inside a block
+    const int32_t* sub_off;  // [K+1]
+    int32_t K;
+    int32_t relu;            // 0 on the last layer
+    float dropout;
+    uint64_t seed;
+    int64_t epoch;
+    int32_t layer;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Kernel launchers (each enqueues on `s` and returns the cudaGetLastError of its launches)
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F,
+                        const Epilogue* epi, cudaStream_t s);
+
+// mode 0: C = A * W_k (W row-major [Kd x N], ld ldw); mode 1: C = (A * W_k^T) masked by Hmask > 0, scaled
+// (W row-major [N x Kd]).  Tiles never cross a subgraph.
+cudaError_t launch_gemm_rows_simt(int mode, const float* A, int lda, int Kd, const float* params, int64_t pstride,
+                                  int64_t w_int, int ldw, int N, float* C, int ldc, const RowSpan* tiles,
+                                  int ntiles, const float* Hmask, int ldh, float scale, cudaStream_t s);
+
+// partial[chunk] = H[chunk rows]^T * dZ[chunk rows]   ([M x ldw] each), one CTA column per chunk.
+cudaError_t launch_gemm_tn_simt(const float* H, int ldh, int M, const float* dZ, int ldz, int N,
+                                const RowSpan* chunks, int nchunks, float* partial, int ldw, cudaStream_t s);
+
+// out[k][off + i] = sum over the chunks of subgraph k, in chunk order, of partial[chunk][i], i < len.
+cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, const int32_t* chunk_ptr, int K,
+                                 float* out, int64_t ostride, int64_t off, int64_t len, cudaStream_t s);
+
+// partial[chunk][j] = sum over the chunk's rows of G[row][j], j < ld.
+cudaError_t launch_colsum_chunks(const float* G, int ld, const RowSpan* chunks, int nchunks, float* partial,
+                                 int64_t pstride_chunk, cudaStream_t s);
+
+cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_t* label, const uint8_t* train,
+                                const RowSpan* chunks, int nchunks, const float* inv_ntrain, float* dlogits,
+                                float* loss_partial, cudaStream_t s);
+cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_ptr, int K, const float* inv_ntrain,
+                              float inv_total, float* loss /*[K+1]*/, int32_t* nonfinite, cudaStream_t s);
+
+cudaError_t launch_zeta_partial(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks,
+                                int nchunks, const int32_t* sub_off, const int64_t* deg_sum, double* partial,
+                                cudaStream_t s);
+cudaError_t launch_zeta_final(const double* partial, int F, int ld, const int32_t* chunk_ptr, int K, const int32_t* sub_off,
+                              const int64_t* deg_sum, const int64_t* deg_sq, float beta, double* zeta, cudaStream_t s);
+
+cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
+                                 const double* zeta, int weighted, int with_sgd, cudaStream_t s);
+cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s);
+
+cudaError_t launch_gather_rows(const float* Xg, int F, const int32_t* gid, int64_t Np, float* H0, int ld,
+                               cudaStream_t s);
+cudaError_t launch_gather_labels(const int32_t* yg, const int32_t* gid, int64_t Np, int32_t* label, cudaStream_t s);
+cudaError_t launch_scatter_core(const float* logits, int ld, int C, const int32_t* gid, const RowSpan* core_spans,
+                                int nspans, float* out, cudaStream_t s);
+
+}  // namespace gad

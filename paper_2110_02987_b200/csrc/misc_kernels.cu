@@ -1,0 +1,376 @@
+// Memory-bound kernels of the epoch other than the SpMM: fused softmax cross-entropy with its gradient,
+// chunked column sums, the statistics of the variance-based importance weight, the fused SGD step +
+// weighted global consensus, and the create-time / accessor gathers.  Every reduction runs in a fixed order
+// (rows of a chunk in order, chunks of a subgraph in order, replicas in ascending k), so a run is bitwise
+// reproducible.
+#include <math.h>
+
+#include "gad_internal.h"
+
+namespace gad {
+
+// ---------------------------------------------------------------------------------------------
+// Softmax cross-entropy over the core training rows and d(loss)/d(logits)  (loss equation, Section 3.3, read
+// as multi-class cross-entropy averaged over the subgraph's training nodes).  One CTA per row chunk, one warp
+// per row; lanes stride over the classes.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restrict__ logits, int ld, int C,
+                                                           const int32_t* __restrict__ label,
+                                                           const uint8_t* __restrict__ train,
+                                                           const RowSpan* __restrict__ chunks,
+                                                           const float* __restrict__ inv_ntrain,
+                                                           float* __restrict__ dlogits, float* __restrict__ loss_partial) {
+    __shared__ float wsum[8];
+    const RowSpan c = chunks[blockIdx.x];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float inv = inv_ntrain[c.k];
+    float acc = 0.f;
+    for (int r = warp; r < c.nrows; r += 8) {
+        const long long row = c.row0 + r;
+        const float* z = logits + row * ld;
+        float* g = dlogits + row * ld;
+        if (!train[row]) {
+            for (int j = lane; j < ld; j += 32) g[j] = 0.f;
+            continue;
+        }
+        float mx = -INFINITY;
+        for (int j = lane; j < C; j += 32) mx = fmaxf(mx, z[j]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+        for (int j = lane; j < C; j += 32) se += expf(z[j] - mx);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        const float lse = mx + logf(se);
+        const int y = label[row];
+        acc += lse - z[y];
+        for (int j = lane; j < ld; j += 32) {
+            float v = 0.f;
+            if (j < C) v = (expf(z[j] - lse) - (j == y ? 1.f : 0.f)) * inv;
+            g[j] = v;
+        }
+    }
+    if (lane == 0) wsum[warp] = acc;  // every lane holds the same acc
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < 8; ++w) s += wsum[w];
+        loss_partial[blockIdx.x] = s;
+    }
+}
+
+// One thread per subgraph adds that subgraph's chunk sums in chunk order; thread 0 then adds the K subgraph
+// sums in ascending k for the global loss sum_k |T_k| L_k / sum_k |T_k|.
+__global__ void loss_final_kernel(const float* __restrict__ loss_partial, const int32_t* __restrict__ chunk_ptr, int K,
+                                  const float* __restrict__ inv_ntrain, float inv_total, float* __restrict__ loss,
+                                  int32_t* __restrict__ nonfinite) {
+    extern __shared__ float sums[];
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float s = 0.f;
+        for (int c = chunk_ptr[k]; c < chunk_ptr[k + 1]; ++c) s += loss_partial[c];
+        sums[k] = s;
+        loss[k] = s * inv_ntrain[k];
+        if (!isfinite(s)) atomicExch(nonfinite, 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int k = 0; k < K; ++k) s += sums[k];
+        loss[K] = s * inv_total;
+    }
+}
+
+cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_t* label, const uint8_t* train,
+                                const RowSpan* chunks, int nchunks, const float* inv_ntrain, float* dlogits,
+                                float* loss_partial, cudaStream_t s) {
+    if (nchunks > 0)
+        softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial);
+    return cudaGetLastError();
+}
+cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_ptr, int K, const float* inv_ntrain,
+                              float inv_total, float* loss, int32_t* nonfinite, cudaStream_t s) {
+    loss_final_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(loss_partial, chunk_ptr, K, inv_ntrain, inv_total, loss, nonfinite);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Column sums of a row chunk (bias gradient db = column sums of dPre over the subgraph's rows).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) colsum_chunks_kernel(const float* __restrict__ G, int ld,
+                                                            const RowSpan* __restrict__ chunks,
+                                                            float* __restrict__ partial, long long pstride_chunk) {
+    // threads = 8 row lanes x 32 column lanes of one float4 each; a block of 128 columns is summed over the
+    // rows ry, ry+8, ... by every row lane and the 8 row lanes are then added in order
+    __shared__ float4 sm[8][32];
+    const RowSpan c = chunks[blockIdx.x];
+    const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+    const int ld4 = ld >> 2;
+    for (int v0 = 0; v0 < ld4; v0 += 32) {
+        const int v = v0 + cx;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (v < ld4) {
+            const float4* g = reinterpret_cast<const float4*>(G + (long long)c.row0 * ld) + v;
+            int r = ry;
+            for (; r + 24 < c.nrows; r += 32) {
+                float4 a0 = g[(long long)r * ld4], a1 = g[(long long)(r + 8) * ld4];
+                float4 a2 = g[(long long)(r + 16) * ld4], a3 = g[(long long)(r + 24) * ld4];
+                s.x += a0.x; s.y += a0.y; s.z += a0.z; s.w += a0.w;
+                s.x += a1.x; s.y += a1.y; s.z += a1.z; s.w += a1.w;
+                s.x += a2.x; s.y += a2.y; s.z += a2.z; s.w += a2.w;
+                s.x += a3.x; s.y += a3.y; s.z += a3.z; s.w += a3.w;
+            }
+            for (; r < c.nrows; r += 8) {
+                float4 a0 = g[(long long)r * ld4];
+                s.x += a0.x; s.y += a0.y; s.z += a0.z; s.w += a0.w;
+            }
+        }
+        sm[ry][cx] = s;
+        __syncthreads();
+        if (ry == 0 && v < ld4) {
+            float4 t = sm[0][cx];
+            for (int w = 1; w < 8; ++w) { t.x += sm[w][cx].x; t.y += sm[w][cx].y; t.z += sm[w][cx].z; t.w += sm[w][cx].w; }
+            reinterpret_cast<float4*>(partial + (long long)blockIdx.x * pstride_chunk)[v] = t;
+        }
+        __syncthreads();
+    }
+}
+cudaError_t launch_colsum_chunks(const float* G, int ld, const RowSpan* chunks, int nchunks, float* partial,
+                                 int64_t pstride_chunk, cudaStream_t s) {
+    if (nchunks > 0) colsum_chunks_kernel<<<(unsigned)nchunks, 256, 0, s>>>(G, ld, chunks, partial, pstride_chunk);
+    return cudaGetLastError();
+}
+
+__global__ void reduce_chunks_kernel(const float* __restrict__ partial, long long pstride_chunk,
+                                     const int32_t* __restrict__ chunk_ptr, float* __restrict__ out, long long ostride,
+                                     long long off, long long len) {
+    const int k = blockIdx.y;
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= len) return;
+    float s = 0.f;
+    for (int c = chunk_ptr[k]; c < chunk_ptr[k + 1]; ++c) s += partial[(long long)c * pstride_chunk + i];
+    out[(long long)k * ostride + off + i] = s;
+}
+cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, const int32_t* chunk_ptr, int K, float* out,
+                                 int64_t ostride, int64_t off, int64_t len, cudaStream_t s) {
+    if (len > 0 && K > 0)
+        reduce_chunks_kernel<<<dim3((unsigned)((len + 255) / 256), (unsigned)K), 256, 0, s>>>(partial, pstride_chunk, chunk_ptr, out,
+                                                                                               ostride, off, len);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Variance-based importance (Section 3.4.1).  With p_i = deg_i / D (D = sum of local degrees; weight 1 and
+// D = n' when the subgraph has no edges) the distance statistic splits by feature dimension:
+//   sum_{i<j} p_i p_j |x_i - x_j|^2 = sum_f ( sum_i p_i (x_if - c_f)^2 - (sum_i p_i (x_if - c_f))^2 )
+// for any shift c_f; c_f = the subgraph's first row keeps the two sums small.  This kernel accumulates the
+// two weighted sums per chunk and per feature in double precision.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) zeta_partial_kernel(const float* __restrict__ X, int ld, int F,
+                                                           const int32_t* __restrict__ deg,
+                                                           const RowSpan* __restrict__ chunks,
+                                                           const int32_t* __restrict__ sub_off,
+                                                           const int64_t* __restrict__ deg_sum,
+                                                           double* __restrict__ partial) {
+    // threads = 8 row lanes x 32 column lanes of one float4 each (as in the column sums above)
+    __shared__ double sm[8][32][8];
+    const RowSpan c = chunks[blockIdx.x];
+    const bool uniform = deg_sum[c.k] == 0;
+    const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+    const int ld4 = ld >> 2;
+    const float4* x0 = reinterpret_cast<const float4*>(X + (long long)sub_off[c.k] * ld);
+    double* P = partial + (long long)blockIdx.x * 2 * ld;
+    for (int v0 = 0; v0 < ld4; v0 += 32) {
+        const int v = v0 + cx;
+        double a[4] = {0.0, 0.0, 0.0, 0.0}, b[4] = {0.0, 0.0, 0.0, 0.0};
+        if (v < ld4) {
+            const float4 sh = x0[v];
+            const float4* g = reinterpret_cast<const float4*>(X + (long long)c.row0 * ld) + v;
+            const int32_t* dg = deg + c.row0;
+            int r = ry;
+            for (; r + 8 < c.nrows; r += 16) {
+                const float4 u0 = g[(long long)r * ld4], u1 = g[(long long)(r + 8) * ld4];
+                const double w0 = uniform ? 1.0 : (double)dg[r], w1 = uniform ? 1.0 : (double)dg[r + 8];
+                const double d0[4] = {(double)(u0.x - sh.x), (double)(u0.y - sh.y), (double)(u0.z - sh.z), (double)(u0.w - sh.w)};
+                const double d1[4] = {(double)(u1.x - sh.x), (double)(u1.y - sh.y), (double)(u1.z - sh.z), (double)(u1.w - sh.w)};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    a[t] = fma(w0, d0[t], a[t]); b[t] = fma(w0 * d0[t], d0[t], b[t]);
+                    a[t] = fma(w1, d1[t], a[t]); b[t] = fma(w1 * d1[t], d1[t], b[t]);
+                }
+            }
+            for (; r < c.nrows; r += 8) {
+                const float4 u0 = g[(long long)r * ld4];
+                const double w0 = uniform ? 1.0 : (double)dg[r];
+                const double d0[4] = {(double)(u0.x - sh.x), (double)(u0.y - sh.y), (double)(u0.z - sh.z), (double)(u0.w - sh.w)};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) { a[t] = fma(w0, d0[t], a[t]); b[t] = fma(w0 * d0[t], d0[t], b[t]); }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { sm[ry][cx][t] = a[t]; sm[ry][cx][4 + t] = b[t]; }
+        __syncthreads();
+        if (ry == 0 && v < ld4) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                double sa = 0.0, sb = 0.0;
+                for (int w = 0; w < 8; ++w) { sa += sm[w][cx][t]; sb += sm[w][cx][4 + t]; }
+                P[4 * v + t] = sa;
+                P[ld + 4 * v + t] = sb;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(256) zeta_final_kernel(const double* __restrict__ partial, int F, int ld,
+                                                         const int32_t* __restrict__ chunk_ptr,
+                                                         const int32_t* __restrict__ sub_off,
+                                                         const int64_t* __restrict__ deg_sum,
+                                                         const int64_t* __restrict__ deg_sq, float beta,
+                                                         double* __restrict__ zeta) {
+    __shared__ double red[256];
+    const int k = blockIdx.x;
+    const long long n = sub_off[k + 1] - sub_off[k];
+    const bool uniform = deg_sum[k] == 0;
+    const double D = uniform ? (double)n : (double)deg_sum[k];
+    double q = 0.0;
+    if (n > 0)
+        for (int f = threadIdx.x; f < F; f += blockDim.x) {
+            double a = 0.0, b = 0.0;
+            for (int c = chunk_ptr[k]; c < chunk_ptr[k + 1]; ++c) {
+                a += partial[(long long)c * 2 * ld + f];
+                b += partial[(long long)c * 2 * ld + ld + f];
+            }
+            const double m1 = a / D;
+            q += b / D - m1 * m1;
+        }
+    red[threadIdx.x] = q;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        double z = 0.0;
+        if (n > 0) {
+            const double sq = uniform ? 1.0 / (double)n : (double)deg_sq[k] / (D * D);
+            const double S = 0.5 * (1.0 - sq);
+            const double Q = red[0] > 0.0 ? red[0] : 0.0;
+            if (S > 0.0) z = S / (sqrt(Q / S) + (double)beta);
+        }
+        zeta[k] = z;
+    }
+}
+
+cudaError_t launch_zeta_partial(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
+                                const int32_t* sub_off, const int64_t* deg_sum, double* partial, cudaStream_t s) {
+    if (nchunks > 0) zeta_partial_kernel<<<(unsigned)nchunks, 256, 0, s>>>(X, ld, F, deg, chunks, sub_off, deg_sum, partial);
+    return cudaGetLastError();
+}
+cudaError_t launch_zeta_final(const double* partial, int F, int ld, const int32_t* chunk_ptr, int K, const int32_t* sub_off,
+                              const int64_t* deg_sum, const int64_t* deg_sq, float beta, double* zeta, cudaStream_t s) {
+    zeta_final_kernel<<<(unsigned)K, 256, 0, s>>>(partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Consensus weights w_k = zeta_k / sum_j zeta_j (Section 3.4.2); 1/K for the plain average of Definition 3
+// or when every zeta is zero.  Computed by each CTA for itself (K is small).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void consensus_weights(const double* __restrict__ zeta, int K, int weighted, float* w_sm) {
+    __shared__ double total;
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int k = 0; k < K; ++k) t += zeta[k];
+        total = t;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < K; k += blockDim.x)
+        w_sm[k] = (weighted && total > 0.0) ? (float)(zeta[k] / total) : 1.f / (float)K;
+    __syncthreads();
+}
+
+// theta_k <- theta_k - lr * grad_k (each replica's own step, update equation of Section 3.3), then
+// theta_k <- sum_j w_j theta_j for every k (weighted global consensus, Section 3.4.2).  One float4 per thread.
+__global__ void __launch_bounds__(256) sgd_consensus_kernel(float* __restrict__ params, const float* __restrict__ grads,
+                                                            long long pstride, long long len4, int K, float lr,
+                                                            const double* __restrict__ zeta, int weighted, int with_sgd) {
+    extern __shared__ float w_sm[];
+    consensus_weights(zeta, K, weighted, w_sm);
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= len4) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < K; ++k) {
+        float4 p = reinterpret_cast<const float4*>(params + (long long)k * pstride)[i];
+        if (with_sgd) {
+            float4 g = reinterpret_cast<const float4*>(grads + (long long)k * pstride)[i];
+            p.x = fmaf(-lr, g.x, p.x); p.y = fmaf(-lr, g.y, p.y); p.z = fmaf(-lr, g.z, p.z); p.w = fmaf(-lr, g.w, p.w);
+        }
+        const float w = w_sm[k];
+        acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y); acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
+    }
+    for (int k = 0; k < K; ++k) reinterpret_cast<float4*>(params + (long long)k * pstride)[i] = acc;
+}
+cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
+                                 const double* zeta, int weighted, int with_sgd, cudaStream_t s) {
+    const long long len4 = len / 4;
+    if (len4 > 0)
+        sgd_consensus_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
+                                                                                                   zeta, weighted, with_sgd);
+    return cudaGetLastError();
+}
+
+__global__ void weights_kernel(const double* __restrict__ zeta, int K, int weighted, float* __restrict__ zeta_f,
+                               float* __restrict__ w_f) {
+    extern __shared__ float w_sm[];
+    consensus_weights(zeta, K, weighted, w_sm);
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        zeta_f[k] = (float)zeta[k];
+        w_f[k] = w_sm[k];
+    }
+}
+cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s) {
+    weights_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(zeta, K, weighted, zeta_f, w_f);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Gathers between graph-node order and store-row order.
+// ---------------------------------------------------------------------------------------------
+__global__ void gather_rows_kernel(const float* __restrict__ Xg, int F, const int32_t* __restrict__ gid, long long Np,
+                                   float* __restrict__ H0, int ld) {
+    const long long row = blockIdx.x;
+    const float* src = Xg + (long long)gid[row] * F;
+    float* dst = H0 + row * ld;
+    for (int j = threadIdx.x; j < ld; j += blockDim.x) dst[j] = j < F ? src[j] : 0.f;
+}
+cudaError_t launch_gather_rows(const float* Xg, int F, const int32_t* gid, int64_t Np, float* H0, int ld, cudaStream_t s) {
+    if (Np > 0) gather_rows_kernel<<<(unsigned)Np, 128, 0, s>>>(Xg, F, gid, Np, H0, ld);
+    return cudaGetLastError();
+}
+__global__ void gather_labels_kernel(const int32_t* __restrict__ yg, const int32_t* __restrict__ gid, long long Np,
+                                     int32_t* __restrict__ label) {
+    const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < Np) label[r] = yg[gid[r]];
+}
+cudaError_t launch_gather_labels(const int32_t* yg, const int32_t* gid, int64_t Np, int32_t* label, cudaStream_t s) {
+    if (Np > 0) gather_labels_kernel<<<(unsigned)((Np + 255) / 256), 256, 0, s>>>(yg, gid, Np, label);
+    return cudaGetLastError();
+}
+// Logits of the core rows back to graph-node order; one CTA per span of core rows.
+__global__ void scatter_core_kernel(const float* __restrict__ logits, int ld, int C, const int32_t* __restrict__ gid,
+                                    const RowSpan* __restrict__ spans, float* __restrict__ out) {
+    const RowSpan sp = spans[blockIdx.x];
+    for (long long i = threadIdx.x; i < (long long)sp.nrows * C; i += blockDim.x) {
+        const long long r = sp.row0 + i / C;
+        const int j = (int)(i % C);
+        out[(long long)gid[r] * C + j] = logits[r * ld + j];
+    }
+}
+cudaError_t launch_scatter_core(const float* logits, int ld, int C, const int32_t* gid, const RowSpan* core_spans, int nspans,
+                                float* out, cudaStream_t s) {
+    if (nspans > 0) scatter_core_kernel<<<(unsigned)nspans, 256, 0, s>>>(logits, ld, C, gid, core_spans, out);
+    return cudaGetLastError();
+}
+
+}  // namespace gad

@@ -1,0 +1,81 @@
+"""CPU checks of the boundary: the library loads, exports every declared symbol, and its host-side
+validation (reached through gad_workspace_bytes, which touches no GPU) rejects malformed inputs."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import __graft_entry__ as entry
+import paper_2110_02987_b200 as pkg
+from paper_2110_02987_b200 import GadError, gad_workspace_bytes
+from conftest import small_random_case, flat
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+
+
+def test_library_exports_every_symbol_the_header_declares():
+    text = open(os.path.join(ROOT, "include", "gad.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(gad_[a-z_]+)\s*\(", text))
+    assert declared == set(pkg.SYMBOLS)
+    lib = pkg.load()
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def _ws(case, dims=(6, 5, 3), **kw):
+    n, rowptr, col, w, core, halo = case
+    return gad_workspace_bytes(n, rowptr, col, *flat(core), *flat(halo), dims, **kw)
+
+
+def test_workspace_bytes_is_host_only_and_grows_with_the_problem():
+    a = _ws(small_random_case(0))
+    b = _ws(small_random_case(0), dims=(6, 50, 3))
+    c = _ws(small_random_case(0, n=80))
+    assert a > 0 and b > a and c > a and a % 256 == 0
+
+
+def test_malformed_inputs_are_rejected_on_the_host():
+    n, rowptr, col, w, core, halo = small_random_case(1)
+    bad = col.copy(); bad[3] = n
+    with pytest.raises(GadError) as e:
+        _ws((n, rowptr, bad, w, core, halo))
+    assert e.value.code == -2
+    rp = rowptr.copy(); rp[5], rp[6] = rp[6] + 1, rp[5]
+    with pytest.raises(GadError) as e:
+        _ws((n, rp, col, w, core, halo))
+    assert e.value.code in (-3, -1)
+    dup = [c.copy() for c in core]; dup[1] = np.concatenate([dup[1], core[0][:1]])
+    with pytest.raises(GadError) as e:
+        _ws((n, rowptr, col, w, dup, halo))
+    assert e.value.code == -4
+    h2 = [h.copy() for h in halo]; h2[0] = np.concatenate([h2[0], core[0][:1]])
+    with pytest.raises(GadError) as e:
+        _ws((n, rowptr, col, w, core, h2))
+    assert e.value.code == -4
+    h3 = [h.copy() for h in halo]; h3[2] = np.concatenate([h3[2], np.array([-1], dtype=np.int32)])
+    with pytest.raises(GadError) as e:
+        _ws((n, rowptr, col, w, core, h3))
+    assert e.value.code == -2
+    for kw, code in ((dict(dropout=1.0), -1), (dict(zeta_mode=1), -9), (dict(gemm_mode=7), -1), (dict(beta=0.0), -1)):
+        with pytest.raises(GadError) as e:
+            _ws((n, rowptr, col, w, core, halo), **kw)
+        assert e.value.code == code
+    with pytest.raises(GadError):
+        _ws((n, rowptr, col, w, core, halo), dims=(6, 0, 3))
+
+
+def test_compute_calls_fail_loudly_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    n, rowptr, col, w, core, halo = small_random_case(2)
+    with pytest.raises(RuntimeError):
+        pkg.Gad(n, rowptr, col, *flat(core), *flat(halo), np.zeros((n, 6), np.float32), np.zeros(n, np.int32),
+                np.zeros(n, np.uint8), (6, 5, 3))

@@ -1,0 +1,294 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element, on the same
+seeded inputs.  Tolerances: integer bookkeeping bit-exact; floating-point tensors (logits, gradients,
+parameters) max|a-b| / max|b| <= 1e-4 in fp32 mode; the 10-epoch loss curve within 1e-3."""
+import numpy as np
+import pytest
+
+import __graft_entry__ as entry
+from gad_synth import make_workload, glorot_params
+from conftest import small_random_case, flat, rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4
+LOSS_TOL = 1e-3
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+
+
+def pkg():
+    import paper_2110_02987_b200 as p
+    return p
+
+
+def orc():
+    from oracle import gad_oracle
+    return gad_oracle
+
+
+def make_pair(case, dims, seed=0, X=None, **kw):
+    n, rowptr, col, w, core, halo = case
+    rng = np.random.default_rng(1000 + seed)
+    if X is None:
+        X = rng.standard_normal((n, dims[0])).astype(np.float32)
+    y = rng.integers(0, dims[-1], size=n).astype(np.int32)
+    split = rng.integers(0, 3, size=n).astype(np.uint8)
+    theta = glorot_params(dims, rng, bias_scale=0.2)
+    cp, cn = flat(core)
+    hp, hn = flat(halo)
+    st = orc().Store(n, rowptr, col, cp, cn, hp, hn, weights=w)
+    okw = {k: v for k, v in kw.items() if k in ("lr", "dropout", "seed", "beta", "weighted")}
+    ref = orc().Model(st, X, y, split, dims, theta, **okw)
+    g = pkg().Gad(n, rowptr, col, cp, cn, hp, hn, X, y, split, dims, init_params=theta, weights=w, **kw)
+    return g, ref, st
+
+
+def check_store(g, st):
+    s = g.get_store()
+    assert np.array_equal(s["rowptr"], st.rowptr)
+    assert np.array_equal(s["col"], st.col)
+    assert np.array_equal(s["sub_off"], st.sub_off)
+    assert np.array_equal(s["gid"], st.gid)
+    assert np.array_equal(s["deg"], st.deg)
+    want = st.val.astype(np.float32)
+    ulp = np.abs(s["val"].view(np.int32).astype(np.int64) - want.view(np.int32).astype(np.int64))
+    assert ulp.max(initial=0) <= 1
+
+
+def check_epoch(g, ref, tol=TOL, loss_tol=1e-5):
+    lg = g.train_epoch()
+    lr = ref.train_epoch()
+    assert np.max(np.abs(lg - lr)) <= loss_tol + 1e-5 * np.max(np.abs(lr)), (lg, lr)
+    L = len(g.dims) - 1
+    for l in range(1, L + 1):
+        assert rel_err(g.get_activation(l), ref.activation(l)) <= tol, "activation %d" % l
+    for k in range(g.K):
+        assert rel_err(g.get_grads(k), ref.get_grads(k)) <= tol, "grads %d" % k
+        assert rel_err(g.get_params(k), ref.get_params(k)) <= tol, "params %d" % k
+
+
+@pytest.mark.parametrize("seed,directed,weighted,dims", [
+    (0, False, False, (6, 5, 3)),
+    (1, False, True, (13, 7, 5, 3)),
+    (2, True, False, (6, 5, 3)),
+    (3, True, True, (33, 130, 4)),
+    (4, False, False, (8, 4)),
+])
+def test_small_cases_store_and_one_epoch(seed, directed, weighted, dims):
+    case = small_random_case(seed, n=70, K=3, directed=directed, weighted=weighted)
+    g, ref, st = make_pair(case, dims, seed, lr=0.1)
+    with g:
+        check_store(g, st)
+        check_epoch(g, ref)
+        check_epoch(g, ref)
+
+
+def test_tiny_ten_epoch_loss_curve_and_parameters(tiny):
+    theta = glorot_params(tiny.dims, np.random.default_rng(0))
+    ref = orc().from_workload(tiny, theta)
+    with pkg().from_workload(tiny, theta) as g:
+        check_store(g, ref.store)
+        lg = np.array([g.train_epoch() for _ in range(10)])
+        lr = np.array([ref.train_epoch() for _ in range(10)])
+        assert np.max(np.abs(lg - lr)) <= LOSS_TOL
+        assert np.max(np.abs(lg - lr)) <= 2e-5          # far inside the bar in fp32 mode
+        for k in range(g.K):
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL
+        out = g.forward()
+        assert rel_err(out, ref.forward_global(tiny.n)) <= TOL
+
+
+def test_tiny_signal_learns_and_tracks_the_oracle(tiny_signal):
+    w = tiny_signal
+    theta = glorot_params(w.dims, np.random.default_rng(2))
+    ref = orc().from_workload(w, theta)
+    with pkg().from_workload(w, theta) as g:
+        lg = np.array([g.train_epoch() for _ in range(10)])
+        lr = np.array([ref.train_epoch() for _ in range(10)])
+        assert lr[-1, -1] < lr[0, -1] - 0.1
+        assert np.max(np.abs(lg - lr)) <= LOSS_TOL
+        for k in range(g.K):
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+
+
+def test_dropout_mask_matches_the_counter_based_definition(tiny_signal):
+    w = tiny_signal
+    theta = glorot_params(w.dims, np.random.default_rng(3))
+    ref = orc().from_workload(w, theta, dropout=0.25, seed=77)
+    with pkg().from_workload(w, theta, dropout=0.25, seed=77) as g:
+        for _ in range(3):
+            lg, lr = g.train_epoch(), ref.train_epoch()
+            assert np.max(np.abs(lg - lr)) <= 1e-4
+            h1g, h1r = g.get_activation(1), ref.activation(1)
+            assert np.array_equal(h1g == 0, h1r == 0)             # the same units dropped
+            assert rel_err(h1g, h1r) <= TOL
+        assert (h1r == 0).mean() > 0.3
+        for k in range(g.K):
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+        # inference applies no dropout
+        assert rel_err(g.forward(), ref.forward_global(w.n)) <= TOL
+
+
+def test_importance_weights_and_consensus(tiny):
+    theta = glorot_params(tiny.dims, np.random.default_rng(4))
+    ref = orc().from_workload(tiny, theta)
+    with pkg().from_workload(tiny, theta) as g:
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(zg - zr) / zr) <= 1e-6
+        assert np.max(np.abs(wg - wr)) <= 1e-6 and abs(float(wg.sum()) - 1.0) <= 1e-6
+        rng = np.random.default_rng(0)
+        for k in range(g.K):
+            t = theta + rng.standard_normal(theta.size).astype(np.float32)
+            g.set_params(k, t)
+            ref.set_params(k, t)
+        g.consensus()
+        ref.consensus()
+        first = g.get_params(0)
+        for k in range(g.K):
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= 1e-6
+            assert np.array_equal(g.get_params(k), first)          # every replica holds the same bits
+        g.consensus()
+        assert rel_err(g.get_params(0), first) <= 1e-6              # a second consensus changes nothing
+    with pkg().from_workload(tiny, theta, weighted=False) as g:
+        assert np.allclose(g.subgraph_weights()[1], 0.25)
+
+
+def test_large_feature_offsets_do_not_break_the_variance_statistics():
+    case = small_random_case(11, n=90, K=3)
+    X = (np.random.default_rng(5).standard_normal((90, 9)) + 300.0).astype(np.float32)
+    g, ref, _ = make_pair(case, (9, 4, 3), 11, X=X)
+    with g:
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(zg - zr) / zr) <= 1e-5
+
+
+def test_single_replica_and_degenerate_subgraphs():
+    # K = 1: the consensus is the identity; an empty subgraph and a subgraph without training nodes are legal
+    n, rowptr, col, w, core, halo = small_random_case(6, n=50, K=1, halo=False)
+    g, ref, st = make_pair((n, rowptr, col, w, core, halo), (6, 5, 3), 6, lr=0.2)
+    with g:
+        check_store(g, st)
+        check_epoch(g, ref)
+        before = g.get_params(0)
+        g.consensus()
+        assert np.array_equal(g.get_params(0), before)
+        assert g.subgraph_weights()[1][0] == 1.0
+    n, rowptr, col, w, core, halo = small_random_case(7, n=60, K=3)
+    core = [core[0], np.empty(0, np.int32), core[2]]
+    halo = [halo[0], np.empty(0, np.int32), halo[2]]
+    g, ref, st = make_pair((n, rowptr, col, w, core, halo), (6, 5, 3), 7, lr=0.2)
+    with g:
+        check_store(g, st)
+        check_epoch(g, ref)
+        zg, wg = g.subgraph_weights()
+        assert zg[1] == 0.0 and wg[1] == 0.0
+
+
+def test_isolated_nodes_and_no_edges():
+    n = 40
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    col = np.empty(0, dtype=np.int32)
+    core = [np.arange(0, 25, dtype=np.int32), np.arange(25, 40, dtype=np.int32)]
+    halo = [np.array([30], dtype=np.int32), np.empty(0, np.int32)]
+    g, ref, st = make_pair((n, rowptr, col, None, core, halo), (5, 4, 3), 8, lr=0.3)
+    with g:
+        check_store(g, st)
+        check_epoch(g, ref)
+        zg, _ = g.subgraph_weights()
+        zr, _ = ref.subgraph_weights()
+        assert np.allclose(zg, zr, rtol=1e-6)
+
+
+def test_hub_rows_and_wide_features():
+    # a star with 5000 leaves puts one row far above the hub threshold; 1030 features need two column slabs
+    n = 5001
+    leaves = np.arange(1, n)
+    src = np.concatenate([np.zeros(n - 1, dtype=np.int64), leaves])
+    dst = np.concatenate([leaves, np.zeros(n - 1, dtype=np.int64)])
+    order = np.lexsort((dst, src))
+    src, dst = src[order], dst[order]
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(np.bincount(src, minlength=n), out=rowptr[1:])
+    core = [np.arange(0, 3000, dtype=np.int32), np.arange(3000, n, dtype=np.int32)]
+    halo = [np.arange(3000, 3100, dtype=np.int32), np.array([0], dtype=np.int32)]
+    g, ref, st = make_pair((n, rowptr, dst.astype(np.int32), None, core, halo), (12, 1030, 3), 9, lr=0.05)
+    with g:
+        check_store(g, st)
+        check_epoch(g, ref)
+
+
+def test_runs_are_bitwise_reproducible_and_resume_is_exact(tiny_signal):
+    w = tiny_signal
+    theta = glorot_params(w.dims, np.random.default_rng(5))
+    with pkg().from_workload(w, theta, dropout=0.25, seed=3) as a:
+        la = np.array([a.train_epoch() for _ in range(10)])
+        pa = a.get_params(0)
+    with pkg().from_workload(w, theta, dropout=0.25, seed=3) as b:
+        lb = [b.train_epoch() for _ in range(5)]
+        saved = [b.get_params(k) for k in range(b.K)]
+        epoch = b.epoch
+    with pkg().from_workload(w, theta, dropout=0.25, seed=3) as c:
+        for k in range(c.K):
+            c.set_params(k, saved[k])
+        c.epoch = epoch
+        lb += [c.train_epoch() for _ in range(5)]
+        pc = c.get_params(0)
+    assert np.array_equal(la, np.array(lb))
+    assert np.array_equal(pa, pc)
+
+
+def test_set_inputs_replaces_features_and_labels(tiny):
+    w = tiny
+    theta = glorot_params(w.dims, np.random.default_rng(6))
+    rng = np.random.default_rng(9)
+    X2 = rng.standard_normal(w.X.shape).astype(np.float32)
+    y2 = rng.integers(0, 4, size=w.n).astype(np.int32)
+    cp, cn, hp, hn = w.flat_partition()
+    st = orc().Store(w.n, w.rowptr, w.col, cp, cn, hp, hn)
+    ref = orc().Model(st, X2, y2, w.split, w.dims, theta, lr=w.lr)
+    with pkg().from_workload(w, theta) as g:
+        g.set_inputs(X2, y2)
+        lg, lr = g.train_epoch(), ref.train_epoch()
+        assert np.max(np.abs(lg - lr)) <= 1e-5
+        assert rel_err(g.get_grads(1), ref.get_grads(1)) <= TOL
+
+
+def test_non_finite_loss_is_reported_not_trapped(tiny):
+    w = tiny
+    theta = glorot_params(w.dims, np.random.default_rng(7))
+    X = w.X.copy()
+    X[w.core[0][0], 0] = np.inf
+    cp, cn, hp, hn = w.flat_partition()
+    with pkg().Gad(w.n, w.rowptr, w.col, cp, cn, hp, hn, X, w.labels, w.split, w.dims, init_params=theta) as g:
+        with pytest.raises(pkg().GadError) as e:
+            g.train_epoch()
+        assert e.value.code == -6
+        g.set_inputs(w.X)                                   # the context stays usable
+        for k in range(g.K):
+            g.set_params(k, theta)
+        assert np.all(np.isfinite(g.train_epoch()))
+
+
+def test_c2_two_epochs_full_size():
+    w = make_workload("c2")
+    theta = glorot_params(w.dims, np.random.default_rng(0))
+    ref = orc().from_workload(w, theta)
+    with pkg().from_workload(w, theta) as g:
+        check_store(g, ref.store)
+        for _ in range(2):
+            lg, lr = g.train_epoch(), ref.train_epoch()
+            assert np.max(np.abs(lg - lr)) <= 1e-4
+        L = len(w.dims) - 1
+        assert rel_err(g.get_activation(L), ref.activation(L)) <= TOL
+        for k in range(g.K):
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(wg - wr)) <= 1e-6
