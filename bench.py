@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the GAD training epoch (all hot-path kernels) on seeded synthetic graphs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3k4|c3k8|c4|tiny|sweep] [--impl reference]
+
+A step is one call of gad_train_epoch: forward, loss, backward, importance weights and weighted consensus for
+all K replicas.  Prints ONE JSON line (rank 0).  ``value`` is epochs/s with every input resident in HBM;
+``e2e`` is the same metric through the C ABI with the step's features and labels copied from pinned host
+memory and the losses read back inside the timed region.  ``--impl reference`` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "GCN train epochs/s over K subgraphs"
+UNIT = "epochs/s"
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/; keyed by (workload, profile entry).  A kernel changed since its capture
+# has no entry (reported as null).
+NCU_TRAFFIC = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            p = json.load(open(path))
+            return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", p.get("bf16_tflops", 0.0))), "measured"
+        except Exception:
+            pass
+    return 6650.0, 1400.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, flag in zip(names, r[3:7]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def describe(w):
+    return "%s: n=%d, nnz=%d, K=%d, dims=%s; %s" % (w.name, w.n, w.nnz, w.K, "-".join(str(d) for d in w.dims), w.recipe)
+
+
+def run_reference(args, rank):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from gad_synth import make_workload, glorot_params
+    from oracle import gad_oracle as orc
+    orc.build()
+    w = make_workload(args.workload, **args.wl_kw)
+    theta = glorot_params(w.dims, np.random.default_rng(0))
+    cores = orc.threads()
+    # bound the run: whole epochs if K*... fits, else the first subgraph alone (1/K of an epoch's work)
+    m = orc.from_workload(w, theta)
+    t0 = time.perf_counter()
+    m.train_epoch()
+    one = time.perf_counter() - t0
+    total_steps = args.steps + args.warmup
+    if one * total_steps <= 150.0 or w.K == 1:
+        sample = "whole epochs of the workload (%d timed)" % args.steps
+        scale = 1.0
+        for _ in range(max(args.warmup - 1, 0)):
+            m.train_epoch()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            m.train_epoch()
+        dt = time.perf_counter() - t0
+    else:
+        m.close()
+        sub = type(w)(**{**w.__dict__})
+        sub.core, sub.halo = [w.core[0]], [w.halo[0]]
+        m = orc.from_workload(sub, theta)
+        m.train_epoch()
+        frac = (len(w.core[0]) + len(w.halo[0])) / float(sum(len(c) + len(h) for c, h in zip(w.core, w.halo)))
+        scale = frac
+        sample = "subgraph 0 of %d only (%.3f of the store rows) per step; epochs/s = steps * that fraction / time" % (w.K, frac)
+        steps = args.steps
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            m.train_epoch()
+            if time.perf_counter() - t0 > 150.0:
+                steps = _ + 1
+                break
+        dt = time.perf_counter() - t0
+        args.steps = steps
+    value = args.steps * scale / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(w)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def cpu_baseline(w, theta, budget_s=20.0):
+    from oracle import gad_oracle as orc
+    orc.build()
+    m = orc.from_workload(w, theta)
+    cores = orc.threads()
+    t0 = time.perf_counter()
+    m.train_epoch()
+    first = time.perf_counter() - t0
+    if first > budget_s and w.K > 1:
+        m.close()
+        sub = type(w)(**{**w.__dict__})
+        sub.core, sub.halo = [w.core[0]], [w.halo[0]]
+        m = orc.from_workload(sub, theta)
+        t0 = time.perf_counter()
+        m.train_epoch()
+        dt = time.perf_counter() - t0
+        frac = (len(w.core[0]) + len(w.halo[0])) / float(sum(len(c) + len(h) for c, h in zip(w.core, w.halo)))
+        return {"value": frac / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": "one epoch of subgraph 0 of %d (%.3f of the store rows), scaled to a whole epoch" % (w.K, frac)}
+    n, t0 = 0, time.perf_counter()
+    while True:
+        m.train_epoch()
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt + first > budget_s or n >= 20:
+            break
+    return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d whole epochs of the same workload after one warm-up epoch" % n}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="gad", choices=["gad", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--mean-deg", type=float, default=32)
+    ap.add_argument("--F", type=int, default=128)
+    ap.add_argument("--K", type=int, default=8)
+    ap.add_argument("--gemm-mode", type=int, default=0)
+    ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernels", action="store_true", help="also print the per-kernel table to stderr")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "gad" else args.warmup
+    args.wl_kw = {"scale": args.scale}
+    if args.workload == "sweep":
+        args.wl_kw.update(mean_deg=args.mean_deg, F=args.F, K=args.K)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+    from gad_synth import make_workload, glorot_params
+    import paper_2110_02987_b200 as pkg
+
+    if not os.path.exists(pkg.LIB_PATH):
+        if local_rank == 0:
+            entry.build()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    pkg.load()
+
+    # Replicas only: every rank runs the whole K-subgraph job on its own GPU (no collective on the data path).
+    w = make_workload(args.workload, **args.wl_kw)
+    theta = glorot_params(w.dims, np.random.default_rng(0))
+    g = pkg.from_workload(w, theta, gemm_mode=args.gemm_mode, flags=args.flags)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident throughput -------------------------------------------------------------------
+    for _ in range(args.warmup):
+        g.train_epoch(wait=False)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = pkg.launch_count()
+    with ClockSampler(local_rank) as clk:
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            g.train_epoch(wait=False)
+        e1.record()
+        barrier()
+    launches = pkg.launch_count() - l0
+    ms = e0.elapsed_time(e1)
+    loss = g.get_loss()
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * args.steps / (ms * 1e-3)
+
+    # ---- per-kernel timing (CUDA events on the library's stream, same steps) --------------------------
+    g.profile_enable(True)
+    g.profile_reset()
+    for _ in range(args.steps):
+        g.train_epoch(wait=False)
+    prof = g.profile_read()
+    g.profile_enable(False)
+    prof.sort(key=lambda e: -e["total_ms"])
+    total_prof = sum(e["total_ms"] for e in prof)
+    top = prof[0]
+    hbm_peak, tensor_peak, peak_kind = measured_peaks()
+    avg_ms = top["total_ms"] / max(top["launches"], 1)
+    roofline = {
+        "kernel": top["name"], "bound": "hbm", "achieved": top["bytes_per_launch"] / (avg_ms * 1e-3) / 1e9,
+        "peak": hbm_peak, "unit": "GB/s", "peak_source": peak_kind, "avg_launch_ms": avg_ms,
+        "share_of_step": top["total_ms"] / total_prof if total_prof > 0 else None,
+        "traffic": NCU_TRAFFIC.get((args.workload, top["name"])),
+    }
+    roofline["frac"] = roofline["achieved"] / hbm_peak
+    kernels = [{"name": e["name"], "ms_per_step": e["total_ms"] / args.steps, "share": e["total_ms"] / total_prof,
+                "GBps": e["bytes_per_launch"] * e["launches"] / (e["total_ms"] * 1e-3) / 1e9 if e["total_ms"] > 0 else None,
+                "TFLOPs": e["flops_per_launch"] * e["launches"] / (e["total_ms"] * 1e-3) / 1e12 if e["total_ms"] > 0 else None}
+               for e in prof]
+    if args.kernels and rank == 0:
+        for k in kernels:
+            sys.stderr.write("%-18s %9.4f ms/step  %5.1f%%  %9.1f GB/s  %8.2f TFLOP/s\n" %
+                             (k["name"], k["ms_per_step"], 100 * k["share"], k["GBps"] or 0, k["TFLOPs"] or 0))
+
+    # ---- end to end: inputs from pinned host memory, losses read back, every step ----------------------
+    Xp = torch.from_numpy(w.X).pin_memory()
+    yp = torch.from_numpy(w.labels).pin_memory()
+    loss_host = torch.zeros(g.K + 1, dtype=torch.float32).pin_memory()
+    loss_np = loss_host.numpy()
+    for _ in range(3):
+        g.set_inputs(Xp, yp)
+        g.train_epoch(loss_out=loss_np)
+    barrier()
+    e2e_steps = max(3, min(args.steps, 20))
+    e0.record()
+    for _ in range(e2e_steps):
+        g.set_inputs(Xp, yp)
+        g.train_epoch(loss_out=loss_np)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e = {"value": world * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
+           "h2d_bytes_per_step": int(Xp.numel() * 4 + yp.numel() * 4), "d2h_bytes_per_step": int((g.K + 1) * 4)}
+
+    ws_mb = g.workspace_bytes / 1e6
+    n_prime, nnz_prime = g.n_prime, g.nnz_prime
+    g.destroy()
+
+    line = None
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if args.gemm_mode == 0 else "bf16 operands, f32 accumulate", "data": "synthetic",
+            "config": {"workload": describe(w), "n_prime": n_prime, "nnz_prime": nnz_prime, "parallelism": "replicas only" if world > 1 else "1 GPU, K replicas batched",
+                       "l2": "per-epoch working set %.0f MB exceeds the 126 MB L2; no flush between steps" % ws_mb
+                             if ws_mb > 2 * 126 else "working set %.0f MB fits L2; consecutive epochs run warm" % ws_mb},
+            "edges_per_s": value * nnz_prime, "final_loss": float(loss[-1]),
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "kernels": kernels,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(w, theta)
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -122,12 +122,14 @@ def _c3(K, rng, scale):
     X = rng.standard_normal((n, 602), dtype=np.float32)
     y = (comm % 41).astype(np.int32)
     split = _split(n, rng)
-    core = bfs_partition(rowptr, col, K)
+    # contiguous blocks follow the planted communities, as a minimum-cut partition would; breadth-first
+    # blocks do not (two hops reach the whole graph), and cut about 70 % of the edges
+    core = contiguous_partition(n, K)
     halo = one_hop_halo(rowptr, col, core, frac_of_core=0.05)
     return Workload(
         name="c3k%d" % K, n=n, rowptr=rowptr, col=col, X=X, labels=y, split=split, core=core, halo=halo,
         dims=(602, 256, 41), lr=0.01, epochs=20,
-        recipe="50 planted communities, mean degree %g, 80%% intra; N(0,1)^602; K=%d BFS blocks; "
+        recipe="50 planted communities, mean degree %g, 80%% intra; N(0,1)^602; K=%d contiguous blocks; "
                "halo .05 of core" % (mean_deg, K))
 
 

@@ -170,6 +170,9 @@ int gad_profile_count(const gad_ctx* ctx, int32_t* count);
 int gad_profile_read(gad_ctx* ctx, int32_t i, char* name64, int64_t* launches, double* total_ms,
                      double* bytes_per_launch, double* flops_per_launch);
 
+/* Number of CUDA kernels this library has launched in this process so far (all contexts). */
+int gad_launch_count(int64_t* launches);
+
 /* Message of the context's last error; with ctx == NULL, of the calling thread's last error (e.g. after a failed
  * gad_create). */
 const char* gad_last_error(const gad_ctx* ctx);

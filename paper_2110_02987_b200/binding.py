@@ -24,7 +24,7 @@ SYMBOLS = (
     "gad_workspace_bytes", "gad_create", "gad_train_epoch", "gad_get_loss", "gad_forward", "gad_subgraph_weights",
     "gad_consensus", "gad_get_params", "gad_set_params", "gad_get_grads", "gad_param_count", "gad_store_sizes",
     "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
-    "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_last_error", "gad_destroy",
+    "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_launch_count", "gad_last_error", "gad_destroy",
 )
 
 
@@ -296,6 +296,15 @@ class Gad:
             out.append(dict(name=name.value.decode(), launches=int(n.value), total_ms=float(ms.value),
                             bytes_per_launch=float(by.value), flops_per_launch=float(fl.value)))
         return out
+
+
+def launch_count() -> int:
+    """gad_launch_count: CUDA kernels launched by the library in this process so far."""
+    n = C.c_int64(0)
+    rc = load().gad_launch_count(C.byref(n))
+    if rc != GAD_OK:
+        raise GadError(rc)
+    return int(n.value)
 
 
 def from_workload(w, init_params, **kw):

@@ -8,6 +8,11 @@
 
 using namespace gad;
 
+namespace gad { int64_t g_kernel_launches = 0; }
+
+// TMA descriptors kept per layer: forward A, B_hi, B_lo; input-gradient A, B_hi, B_lo; weight-gradient H, dZ.
+constexpr int kMapsPerLayer = 8;
+
 namespace {
 
 struct ProfEntry {
@@ -21,7 +26,7 @@ struct ProfEntry {
 // gad_create, so both agree byte for byte.
 struct Plan {
     int32_t n = 0, K = 0, L = 0;
-    int64_t Np = 0, nnz = 0, P = 0, Pint = 0, pstride = 0;
+    int64_t Np = 0, nnz = 0, P = 0, Pint = 0, pstride = 0, slots = 0;
     std::vector<int32_t> dims;
     std::vector<Layer> layers;
     std::vector<int32_t> ld;          // [L+1]
@@ -31,11 +36,11 @@ struct Plan {
     int64_t dw_partial = 0;           // floats per chunk
     size_t bytes = 0;
     // offsets into the workspace
-    size_t o_rowptr, o_ecv, o_perm, o_hub, o_trowptr, o_tecv, o_tperm, o_thub, o_sub_off, o_gid, o_deg, o_label, o_train,
+    size_t o_rowptr, o_ecv, o_perm, o_parts, o_fin, o_trowptr, o_tecv, o_tperm, o_tparts, o_tfin, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
         o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
         o_dw_partial, o_cs_partial, o_loss_partial, o_zeta_partial, o_zeta, o_loss, o_flags, o_zeta_f, o_w_f, o_stage,
         o_stage_lab;
-    std::vector<size_t> o_H;
+    std::vector<size_t> o_H, o_w_hi, o_w_lo, o_wt_hi, o_wt_lo;   // per layer
 };
 
 size_t take(size_t& cur, size_t bytes) {
@@ -45,7 +50,7 @@ size_t take(size_t& cur, size_t bytes) {
 }
 
 int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off, const std::vector<int64_t>& core_count,
-              int64_t nnz, const gad_config* cfg, std::string& err) {
+              int64_t nnz, int64_t slots, const gad_config* cfg, std::string& err) {
     if (!cfg || cfg->L < 1 || !cfg->dims) { err = "config needs L >= 1 and dims"; return GAD_ERR_ARG; }
     for (int l = 0; l <= cfg->L; ++l)
         if (cfg->dims[l] < 1) { err = "layer size must be positive"; return GAD_ERR_ARG; }
@@ -54,7 +59,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     if (cfg->zeta_mode == 1) { err = "zeta_mode 1 (pairwise form) is not implemented"; return GAD_ERR_UNSUPPORTED; }
     if (cfg->zeta_mode != 0) { err = "zeta_mode must be 0 or 1"; return GAD_ERR_ARG; }
     if (!(cfg->beta > 0.f)) { err = "beta must be positive"; return GAD_ERR_ARG; }
-    p.n = n; p.K = K; p.L = cfg->L; p.nnz = nnz; p.Np = sub_off[K];
+    p.n = n; p.K = K; p.L = cfg->L; p.nnz = nnz; p.Np = sub_off[K]; p.slots = slots;
     p.dims.assign(cfg->dims, cfg->dims + cfg->L + 1);
     p.ld.resize(p.L + 1);
     p.maxld = 0;
@@ -89,9 +94,11 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     const size_t Np = (size_t)p.Np, nc = p.chunks.size();
     size_t cur = 0;
     p.o_rowptr = take(cur, 8 * (Np + 1)); p.o_ecv = take(cur, 8 * (size_t)nnz);
-    p.o_perm = take(cur, 4 * Np); p.o_hub = take(cur, 4 * Np);
+    // work lists: at most one part per kShortRow entries plus one per row that is cut
+    const size_t max_parts = (size_t)(nnz / kShortRow + slots + 1), max_fin = (size_t)(nnz / kPartEntries + 1);
+    p.o_perm = take(cur, 4 * Np); p.o_parts = take(cur, 16 * max_parts); p.o_fin = take(cur, 16 * max_fin);
     p.o_trowptr = take(cur, 8 * (Np + 1)); p.o_tecv = take(cur, 8 * (size_t)nnz);
-    p.o_tperm = take(cur, 4 * Np); p.o_thub = take(cur, 4 * Np);
+    p.o_tperm = take(cur, 4 * Np); p.o_tparts = take(cur, 16 * max_parts); p.o_tfin = take(cur, 16 * max_fin);
     p.o_sub_off = take(cur, 4 * (size_t)(K + 1)); p.o_gid = take(cur, 4 * Np); p.o_deg = take(cur, 4 * Np);
     p.o_label = take(cur, 4 * Np); p.o_train = take(cur, Np);
     p.o_deg_sum = take(cur, 8 * (size_t)K); p.o_deg_sq = take(cur, 8 * (size_t)K); p.o_inv_ntrain = take(cur, 4 * (size_t)K);
@@ -99,6 +106,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_chunk_ptr = take(cur, 4 * (size_t)(K + 1)); p.o_core_spans = take(cur, sizeof(RowSpan) * p.core_spans.size());
     p.o_H.resize(p.L + 1);
     for (int l = 0; l <= p.L; ++l) p.o_H[l] = take(cur, 4 * Np * (size_t)p.ld[l]);
+    p.o_spmm_scratch = take(cur, 4 * (size_t)slots * (size_t)p.maxld);
     p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
     p.o_params = take(cur, 4 * (size_t)K * (size_t)p.pstride); p.o_grads = take(cur, 4 * (size_t)K * (size_t)p.pstride);
     p.o_dw_partial = take(cur, 4 * nc * (size_t)p.dw_partial); p.o_cs_partial = take(cur, 4 * nc * (size_t)p.maxld);
@@ -106,6 +114,12 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_zeta = take(cur, 8 * (size_t)K); p.o_loss = take(cur, 4 * (size_t)(K + 1)); p.o_flags = take(cur, 16);
     p.o_zeta_f = take(cur, 4 * (size_t)K); p.o_w_f = take(cur, 4 * (size_t)K);
     p.o_stage = take(cur, 4 * (size_t)n * (size_t)std::max(p.dims[0], p.dims[p.L])); p.o_stage_lab = take(cur, 4 * (size_t)n);
+    p.o_w_hi.resize(p.L); p.o_w_lo.resize(p.L); p.o_wt_hi.resize(p.L); p.o_wt_lo.resize(p.L);
+    for (int l = 0; l < p.L; ++l) {
+        const Layer& y = p.layers[l];
+        p.o_w_hi[l] = take(cur, 4 * (size_t)K * y.fi * y.ldw); p.o_w_lo[l] = take(cur, 4 * (size_t)K * y.fi * y.ldw);
+        p.o_wt_hi[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi); p.o_wt_lo[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi);
+    }
     p.bytes = cur;
     return GAD_OK;
 }
@@ -127,6 +141,10 @@ struct gad_ctx {
     bool profiling = false;
     std::vector<ProfEntry> prof;
     std::vector<float> host_block;  // staging for parameter pack / unpack
+    bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
+    int num_sms = 1;
+    struct alignas(64) TMap { unsigned char bytes[128]; };
+    std::vector<TMap> maps;         // per layer: forward A, B_hi, B_lo; input-gradient A, B_hi, B_lo
 
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
     float* H(int l) const { return at<float>(p.o_H[l]); }
@@ -188,9 +206,23 @@ int forward_pass(gad_ctx* ctx, bool train) {
     const Plan& p = ctx->p;
     float* Z = ctx->at<float>(p.o_G2);
     const float* params = ctx->at<float>(p.o_params);
+    const int passes = ctx->cfg.gemm_mode == 0 ? 3 : 1;
+    if (ctx->use_tc)
+        for (int l = 0; l < p.L; ++l) {
+            const Layer& y = p.layers[l];
+            GAD_RUN("split_weights", l, 20.0 * p.K * y.fi * y.fo, 0.0, [&] {
+                return launch_split_weights(params, p.pstride, y.w_int, y.fi, y.fo, y.ldw, y.ldi, p.K, ctx->at<float>(p.o_w_hi[l]),
+                                            ctx->at<float>(p.o_w_lo[l]), ctx->at<float>(p.o_wt_hi[l]), ctx->at<float>(p.o_wt_lo[l]),
+                                            ctx->stream);
+            });
+        }
     for (int l = 0; l < p.L; ++l) {
         const Layer& y = p.layers[l];
         GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+            if (ctx->use_tc)
+                return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 0, passes, y.fi, y.fo, Z,
+                                           y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f,
+                                           ctx->at<int32_t>(p.o_flags) + 1, ctx->num_sms, ctx->stream);
             return launch_gemm_rows_simt(0, ctx->H(l), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, Z, y.ldo,
                                          ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, ctx->stream);
         });
@@ -238,14 +270,23 @@ int backward_pass(gad_ctx* ctx) {
         GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                 [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
         GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
-            cudaError_t e = launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, chunks, nc, ctx->at<float>(p.o_dw_partial),
-                                                y.ldw, ctx->stream);
+            cudaError_t e = ctx->use_tc
+                                ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
+                                                    ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, chunks, nc,
+                                                    ctx->at<float>(p.o_dw_partial), ctx->at<int32_t>(p.o_flags) + 1, ctx->stream)
+                                : launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, chunks, nc,
+                                                      ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
             if (e != cudaSuccess) return e;
             return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, chunk_ptr, p.K, grads, p.pstride,
                                         y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
         });
         if (l > 0)
             GAD_RUN("gemm_dh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+                if (ctx->use_tc)
+                    return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 3], &ctx->maps[kMapsPerLayer * l + 4], &ctx->maps[kMapsPerLayer * l + 5], 1,
+                                               ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fo, y.fi, G1, y.ldi, ctx->at<RowSpan>(p.o_tiles),
+                                               (int)p.tiles.size(), ctx->H(l), y.ldi, scale, ctx->at<int32_t>(p.o_flags) + 1,
+                                               ctx->num_sms, ctx->stream);
                 return launch_gemm_rows_simt(1, G2, y.ldo, y.fo, params, p.pstride, y.w_int, y.ldw, y.fi, G1, y.ldi,
                                              ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), ctx->H(l), y.ldi, scale,
                                              ctx->stream);
@@ -277,7 +318,7 @@ uint64_t host_mix64(uint64_t z) {
 }
 
 int upload_sparse(gad_ctx* ctx, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col, const std::vector<float>& val,
-                  size_t o_rowptr, size_t o_ecv, size_t o_perm, size_t o_hub, SparseDev& out) {
+                  size_t o_rowptr, size_t o_ecv, size_t o_perm, size_t o_parts, size_t o_fin, SparseDev& out) {
     const Plan& p = ctx->p;
     std::vector<uint2> ecv(col.size());
     for (size_t e = 0; e < col.size(); ++e) {
@@ -285,20 +326,27 @@ int upload_sparse(gad_ctx* ctx, const std::vector<int64_t>& rowptr, const std::v
         std::memcpy(&bits, &val[e], 4);
         ecv[e] = make_uint2((uint32_t)col[e], bits);
     }
-    std::vector<int32_t> perm, hub;
-    bin_rows(rowptr, 2048, perm, hub);
+    RowWork work;
+    bin_rows(rowptr, work);
+    if (work.slots > p.slots) return fail(ctx, GAD_ERR_OOM, "SpMM scratch slots exceed the planned count");
+    const std::vector<int32_t>& perm = work.perm;
     GAD_CK(cudaMemcpyAsync(ctx->ws + o_rowptr, rowptr.data(), 8 * rowptr.size(), cudaMemcpyHostToDevice, ctx->stream));
     if (!ecv.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_ecv, ecv.data(), 8 * ecv.size(), cudaMemcpyHostToDevice, ctx->stream));
     if (!perm.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_perm, perm.data(), 4 * perm.size(), cudaMemcpyHostToDevice, ctx->stream));
-    if (!hub.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_hub, hub.data(), 4 * hub.size(), cudaMemcpyHostToDevice, ctx->stream));
+    if (!work.parts.empty())
+        GAD_CK(cudaMemcpyAsync(ctx->ws + o_parts, work.parts.data(), 16 * work.parts.size(), cudaMemcpyHostToDevice, ctx->stream));
+    if (!work.fin.empty())
+        GAD_CK(cudaMemcpyAsync(ctx->ws + o_fin, work.fin.data(), 16 * work.fin.size(), cudaMemcpyHostToDevice, ctx->stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));  // the host vectors above go out of scope
     out.rowptr = ctx->at<int64_t>(o_rowptr);
     out.ecv = ctx->at<uint2>(o_ecv);
     out.perm = ctx->at<int32_t>(o_perm);
-    out.hub = ctx->at<int32_t>(o_hub);
+    out.parts = ctx->at<int4>(o_parts);
+    out.fin = ctx->at<int4>(o_fin);
+    out.scratch = ctx->at<float>(p.o_spmm_scratch);
     out.nperm = (int32_t)perm.size();
-    out.nhub = (int32_t)hub.size();
-    (void)p;
+    out.nparts = (int32_t)work.parts.size();
+    out.nfin = (int32_t)work.fin.size();
     return GAD_OK;
 }
 
@@ -315,8 +363,8 @@ extern "C" {
 int gad_workspace_bytes(const gad_csr* g, const gad_partition* part, const gad_config* cfg, size_t* bytes) {
     if (!bytes) return GAD_ERR_ARG;
     std::string err;
-    int64_t Np = 0, nnz = 0;
-    int rc = store_sizes(g, part, &Np, &nnz, err);
+    int64_t Np = 0, nnz = 0, slots = 0;
+    int rc = store_sizes(g, part, &Np, &nnz, &slots, err);
     if (rc != GAD_OK) return fail(nullptr, rc, err);
     std::vector<int32_t> sub_off(part->K + 1, 0);
     std::vector<int64_t> core_count(part->K, 0);
@@ -325,7 +373,7 @@ int gad_workspace_bytes(const gad_csr* g, const gad_partition* part, const gad_c
         sub_off[k + 1] = sub_off[k] + (int32_t)(core_count[k] + part->halo_ptr[k + 1] - part->halo_ptr[k]);
     }
     Plan p;
-    rc = make_plan(p, g->n, part->K, sub_off, core_count, nnz, cfg, err);
+    rc = make_plan(p, g->n, part->K, sub_off, core_count, nnz, slots, cfg, err);
     if (rc != GAD_OK) return fail(nullptr, rc, err);
     *bytes = p.bytes;
     return GAD_OK;
@@ -347,7 +395,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     HostStore st;
     int rc = build_store(g, part, true, st, ctx->err);
     if (rc != GAD_OK) return fail(ctx, rc, ctx->err);
-    rc = make_plan(ctx->p, g->n, part->K, st.sub_off, st.core_count, st.nnz, cfg, ctx->err);
+    const int64_t slots = std::max(count_slots(st.rowptr), st.symmetric ? 0 : count_slots(st.t_rowptr));
+    rc = make_plan(ctx->p, g->n, part->K, st.sub_off, st.core_count, st.nnz, slots, cfg, ctx->err);
     if (rc != GAD_OK) return fail(ctx, rc, ctx->err);
     ctx->cfg.dims = ctx->p.dims.data();
     const Plan& p = ctx->p;
@@ -361,10 +410,10 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->sub_off = st.sub_off;
     ctx->gid = st.gid;
 
-    rc = upload_sparse(ctx, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_perm, p.o_hub, ctx->A);
+    rc = upload_sparse(ctx, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_perm, p.o_parts, p.o_fin, ctx->A);
     if (rc != GAD_OK) return rc;
     if (!st.symmetric) {
-        rc = upload_sparse(ctx, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tperm, p.o_thub, ctx->At);
+        rc = upload_sparse(ctx, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tperm, p.o_tparts, p.o_tfin, ctx->At);
         if (rc != GAD_OK) return rc;
     }
     // per-row labels and loss mask, per-subgraph degree sums and training counts
@@ -418,6 +467,39 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
                                cudaMemcpyHostToDevice, ctx->stream));
     GAD_CK(cudaMemsetAsync(ctx->ws + p.o_grads, 0, 4 * (size_t)p.K * p.pstride, ctx->stream));
     GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 16, ctx->stream));
+    // tensor-core path: operand copies start at zero (their pad columns are never written) and get TMA descriptors
+    {
+        int dev = 0;
+        GAD_CK(cudaGetDevice(&dev));
+        cudaDeviceProp prop;
+        GAD_CK(cudaGetDeviceProperties(&prop, dev));
+        ctx->num_sms = prop.multiProcessorCount;
+        ctx->use_tc = (cfg->flags & 1) == 0 && prop.major == 10 && p.Np > 0;
+    }
+    if (ctx->use_tc) {
+        ctx->maps.resize((size_t)kMapsPerLayer * p.L);
+        bool ok = true;
+        for (int l = 0; l < p.L && ok; ++l) {
+            const Layer& y = p.layers[l];
+            GAD_CK(cudaMemsetAsync(ctx->ws + p.o_w_hi[l], 0, 4 * (size_t)p.K * y.fi * y.ldw, ctx->stream));
+            GAD_CK(cudaMemsetAsync(ctx->ws + p.o_w_lo[l], 0, 4 * (size_t)p.K * y.fi * y.ldw, ctx->stream));
+            GAD_CK(cudaMemsetAsync(ctx->ws + p.o_wt_hi[l], 0, 4 * (size_t)p.K * y.fo * y.ldi, ctx->stream));
+            GAD_CK(cudaMemsetAsync(ctx->ws + p.o_wt_lo[l], 0, 4 * (size_t)p.K * y.fo * y.ldi, ctx->stream));
+            gad_ctx::TMap* m = &ctx->maps[(size_t)kMapsPerLayer * l];
+            // forward: A = H^(l) [Np x fi], B = W^T copies [K][fo][fi]
+            ok = ok && tc_make_map(&m[0], ctx->H(l), y.fi, p.Np, 0, 4ull * y.ldi, 0, 128);
+            ok = ok && tc_make_map(&m[1], ctx->at<float>(p.o_wt_hi[l]), y.fi, y.fo, p.K, 4ull * y.ldi, 4ull * y.fo * y.ldi, tc_bn_for(y.fo));
+            ok = ok && tc_make_map(&m[2], ctx->at<float>(p.o_wt_lo[l]), y.fi, y.fo, p.K, 4ull * y.ldi, 4ull * y.fo * y.ldi, tc_bn_for(y.fo));
+            // input gradient: A = dZ [Np x fo] (in G2), B = W copies [K][fi][fo]
+            ok = ok && tc_make_map(&m[3], ctx->at<float>(p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 128);
+            ok = ok && tc_make_map(&m[4], ctx->at<float>(p.o_w_hi[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
+            ok = ok && tc_make_map(&m[5], ctx->at<float>(p.o_w_lo[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
+            // weight gradient: 32-row tiles of H^(l) and of dZ (in G2)
+            ok = ok && tc_make_map(&m[6], ctx->H(l), y.fi, p.Np, 0, 4ull * y.ldi, 0, 32, true);
+            ok = ok && tc_make_map(&m[7], ctx->at<float>(p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 32, true);
+        }
+        if (!ok) return fail(ctx, GAD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    }
     GAD_CK(cudaMemsetAsync(ctx->ws + p.o_loss, 0, 4 * (size_t)(p.K + 1), ctx->stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));
     guard.ok = true;
@@ -428,10 +510,15 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
 int gad_get_loss(gad_ctx* ctx, float* loss_out) {
     if (!ctx || !loss_out) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
-    int32_t flag = 0;
+    int32_t flags[2] = {0, 0};
     GAD_CK(cudaMemcpyAsync(loss_out, ctx->ws + p.o_loss, 4 * (size_t)(p.K + 1), cudaMemcpyDeviceToHost, ctx->stream));
-    GAD_CK(cudaMemcpyAsync(&flag, ctx->ws + p.o_flags, 4, cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaMemcpyAsync(flags, ctx->ws + p.o_flags, 8, cudaMemcpyDeviceToHost, ctx->stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));
+    const int32_t flag = flags[0];
+    if (flags[1]) {
+        GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 8, ctx->stream));
+        return fail(ctx, GAD_ERR_DEVICE_TIMEOUT, "a bounded wait in the tensor-core transform ran out (role " + std::to_string(flags[1]) + ")");
+    }
     if (flag) {
         GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 4, ctx->stream));
         return fail(ctx, GAD_ERR_NONFINITE, "a subgraph loss is NaN or infinite");
@@ -644,6 +731,12 @@ int gad_profile_read(gad_ctx* ctx, int32_t i, char* name64, int64_t* launches, d
     if (total_ms) *total_ms = e.ms;
     if (bytes_per_launch) *bytes_per_launch = e.bytes;
     if (flops_per_launch) *flops_per_launch = e.flops;
+    return GAD_OK;
+}
+
+int gad_launch_count(int64_t* launches) {
+    if (!launches) return GAD_ERR_ARG;
+    *launches = gad::g_kernel_launches;
     return GAD_OK;
 }
 

@@ -13,6 +13,9 @@ namespace gad {
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 
+// Kernels launched by this library in this process (every <<<>>> adds one).
+extern int64_t g_kernel_launches;
+
 // ---------------------------------------------------------------------------------------------
 // Host-side result of building the block-diagonal store (create-time, not on the timed path).
 // ---------------------------------------------------------------------------------------------
@@ -27,20 +30,29 @@ struct HostStore {
     std::vector<int32_t> deg;      // [Np] local degree, self-loop excluded
     std::vector<int64_t> core_count;  // [K]
     bool symmetric = false;        // A~ equals its transpose entry by entry
-    std::vector<int64_t> t_rowptr; // transposed store (empty when symmetric)
+    std::vector<int64_t> t_rowptr; // transposed store (t_col, t_val empty when symmetric or when values were not asked for)
     std::vector<int32_t> t_col;
     std::vector<float> t_val;
 };
 
 // Validates the inputs and fills the store; returns a GAD_* status and a message.
 int build_store(const gad_csr* g, const gad_partition* part, bool values, HostStore& out, std::string& err);
-// Sizes only (for gad_workspace_bytes).
-int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, std::string& err);
+// Sizes only (for gad_workspace_bytes): rows, entries, and the SpMM scratch slots of the worse orientation.
+int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, int64_t* slots, std::string& err);
 
-// Rows ordered for the SpMM launch: rows with at least `hub_nnz` entries go to the hub list (one CTA each),
-// the others are binned by floor(log2(nnz)), heaviest bin first, ascending row id inside a bin.
-void bin_rows(const std::vector<int64_t>& rowptr, int64_t hub_nnz, std::vector<int32_t>& perm,
-              std::vector<int32_t>& hub);
+// Work lists of the SpMM launch.  Rows with fewer than kShortRow entries go to `perm`, binned by
+// floor(log2(entries)), heaviest bin first, ascending row id inside a bin.  Longer rows are cut into parts of at
+// most kPartEntries entries: parts = {row, first entry relative to the row, entries, scratch slot or -1 when the
+// row is a single part}; fin = {row, first scratch slot, slots, 0} for every row made of several parts.
+constexpr int64_t kShortRow = 64, kPartEntries = 512;
+struct RowWork {
+    std::vector<int32_t> perm;
+    std::vector<int4> parts, fin;
+    int64_t slots = 0;
+};
+void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out);
+// Scratch slots bin_rows would use, from the row lengths alone.
+int64_t count_slots(const std::vector<int64_t>& rowptr);
 
 // ---------------------------------------------------------------------------------------------
 // Device views
@@ -48,9 +60,11 @@ void bin_rows(const std::vector<int64_t>& rowptr, int64_t hub_nnz, std::vector<i
 struct SparseDev {
     const int64_t* rowptr = nullptr;  // [Np+1]
     const uint2* ecv = nullptr;       // [nnz] packed (column, value bits)
-    const int32_t* perm = nullptr;    // binned non-hub rows
-    const int32_t* hub = nullptr;     // hub rows
-    int32_t nperm = 0, nhub = 0;
+    const int32_t* perm = nullptr;    // binned short rows
+    const int4* parts = nullptr;      // parts of the long rows
+    const int4* fin = nullptr;        // rows made of several parts
+    float* scratch = nullptr;         // [slots x leading dimension of the output] partial rows
+    int32_t nperm = 0, nparts = 0, nfin = 0;
 };
 
 struct Layer {
@@ -88,6 +102,22 @@ cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out,
 cudaError_t launch_gemm_rows_simt(int mode, const float* A, int lda, int Kd, const float* params, int64_t pstride,
                                   int64_t w_int, int ldw, int N, float* C, int ldc, const RowSpan* tiles,
                                   int ntiles, const float* Hmask, int ldh, float scale, cudaStream_t s);
+
+// Tensor-core (tcgen05) version of launch_gemm_rows_simt.  The operands come through TMA descriptors made by
+// tc_make_map (A: [rows x Kd]; B, B_lo: [K][N][Kd] copies written by launch_split_weights); passes = 3 gives fp32
+// accuracy by operand splitting, passes = 1 plain TF32 operands.  err receives a role code if a bounded wait runs out.
+int tc_bn_for(int n_cols);
+bool tc_make_map(void* out_map, const void* base, uint64_t inner, uint64_t rows, uint64_t outer, uint64_t row_stride_bytes,
+                 uint64_t outer_stride_bytes, uint32_t box_rows, bool mn_major = false);
+cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w_int, int fi, int fo, int ldw, int ldkt, int K,
+                                 float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, cudaStream_t s);
+cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* mapBlo, int mode, int passes, int Kd, int n_cols,
+                                float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
+                                int32_t* err, int num_sms, cudaStream_t s);
+
+// Tensor-core version of launch_gemm_tn_simt; mapH / mapZ are 32-row-box descriptors of H^(l) and dZ.
+cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,
+                              int nchunks, float* partial, int32_t* err, cudaStream_t s);
 
 // partial[chunk] = H[chunk rows]^T * dZ[chunk rows]   ([M x ldw] each), one CTA column per chunk.
 cudaError_t launch_gemm_tn_simt(const float* H, int ldh, int M, const float* dZ, int ldz, int N,

@@ -105,6 +105,7 @@ static cudaError_t launch_rows_cfg(int mode, const float* A, int lda, int Kd, co
     else
         gemm_rows_kernel<BM, BN, BK, TM, TN, 1><<<grid, NT, 0, s>>>(A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles,
                                                                     Hmask, ldh, scale);
+    ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -189,12 +190,12 @@ cudaError_t launch_gemm_tn_simt(const float* H, int ldh, int M, const float* dZ,
         constexpr int BM = 128, BN = 64;
         int ntm = (M + BM - 1) / BM, ntn = (ldw + BN - 1) / BN;
         gemm_tn_kernel<BM, BN, 16, 8, 4><<<dim3((unsigned)(ntm * ntn), (unsigned)nchunks), 256, 0, s>>>(H, ldh, M, dZ, ldz, N, chunks, partial,
-                                                                                                     pstride_chunk, ldw, ntn);
+                                                                                                     pstride_chunk, ldw, ntn); ++g_kernel_launches;
     } else {
         constexpr int BM = 128, BN = 32;
         int ntm = (M + BM - 1) / BM, ntn = (ldw + BN - 1) / BN;
         gemm_tn_kernel<BM, BN, 16, 4, 4><<<dim3((unsigned)(ntm * ntn), (unsigned)nchunks), 256, 0, s>>>(H, ldh, M, dZ, ldz, N, chunks, partial,
-                                                                                                     pstride_chunk, ldw, ntn);
+                                                                                                     pstride_chunk, ldw, ntn); ++g_kernel_launches;
     }
     return cudaGetLastError();
 }

@@ -1,0 +1,584 @@
+// Grouped dense transforms on the 5th-generation tensor cores (tcgen05, accumulators in tensor memory):
+//   mode 0   Z_l  = H^(l) W_k^(l)                        (the H.W of the forward equation, Section 3.3)
+//   mode 1   dPre = (dZ_l W_k^(l)^T) masked by H^(l) > 0  (chain rule through the forward equation)
+// Both are C[rows x N] = A[rows x Kd] * B_k^T with A row-major (Kd contiguous) and B_k stored as N rows of Kd
+// contiguous values, i.e. both operands K-major.  Row tiles never cross a subgraph, so a tile uses one replica's B.
+//
+// fp32 accuracy from TF32 tensor cores: every operand value x is split into hi = x rounded to a 10-bit mantissa
+// (exactly representable in TF32) and lo = x - hi, rounded the same way, and the product is accumulated as
+// A_hi B_hi + A_hi B_lo + A_lo B_hi in fp32 (the dropped A_lo B_lo term and the rounding of lo are ~2^-22 relative).  B is split once per
+// epoch by a small kernel; A tiles are split in shared memory by two warps of the GEMM kernel.  With passes = 1
+// only A B is issued on the unsplit operands (TF32 operand precision).
+//
+// One persistent CTA per SM, 8 warps: warp 0 issues TMA loads (128B-swizzled tiles) through a 3-stage ring,
+// warps 2-3 split the A tile, warp 1 issues tcgen05.mma, warps 4-7 drain the accumulator (tcgen05.ld) while
+// the MMA warp already fills the second accumulator.  Every mbarrier wait is bounded: on a time-out the CTA
+// raises an error word, stops, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "gad_internal.h"
+
+namespace gad {
+
+namespace {
+
+constexpr int BM = 128, BK = 32, STAGES = 3, BN_MAX = 128;
+constexpr int A_BYTES = BM * BK * 4;                      // 16 KiB
+constexpr int B_BYTES = BN_MAX * BK * 4;                  // 16 KiB
+constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;    // A_hi | A_lo | B_hi | B_lo
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int TMEM_COLS = 2 * BN_MAX;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.b32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the wait ran out or another role of this CTA has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* err, int code) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    atomicExch(err, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+                 : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile written by TMA with the 128-byte swizzle: rows of 128 bytes,
+// groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2 (128B swizzle).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+// Instruction descriptor: fp32 accumulator, TF32 A and B, both K-major, N and M of the MMA.
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, "
+        "%25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Nearest value with a 10-bit mantissa (ties away from zero), i.e. exactly representable in TF32.
+// Infinities and NaNs pass through unchanged; a finite value that would round up to infinity is truncated.
+__device__ __forceinline__ float tf32_round(float x) {
+    const uint32_t b = __float_as_uint(x);
+    if ((b & 0x7F800000u) == 0x7F800000u) return x;
+    uint32_t r = (b + 0x1000u) & 0xFFFFE000u;
+    if ((r & 0x7F800000u) == 0x7F800000u) r = b & 0xFFFFE000u;
+    return __uint_as_float(r);
+}
+
+struct TcArgs {
+    const RowSpan* tiles;
+    int ntiles_rows, ntn, BN, Kd;
+    float* C;
+    int ldc;
+    const float* Hmask;
+    int ldh;
+    float scale;
+    int mode, passes;
+    int32_t* err;
+};
+
+__global__ void __launch_bounds__(256, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmBlo, const TcArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+    uint8_t* sm = smem_raw + pad;                 // 1024-byte aligned: the 128B swizzle pattern repeats every 1024 bytes
+    const uint32_t sm_addr = raw_addr + pad;
+    const uint32_t bars = sm_addr + STAGES * STAGE_BYTES;
+    auto full = [&](int s) { return bars + 8u * s; };
+    auto xfull = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto empty = [&](int s) { return bars + 8u * (2 * STAGES + s); };
+    auto tfull = [&](int i) { return bars + 8u * (3 * STAGES + i); };
+    auto tempty = [&](int i) { return bars + 8u * (3 * STAGES + 2 + i); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), 64); mbar_init(empty(s), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 128); }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int ntiles = a.ntiles_rows * a.ntn;
+    const int nkb = (a.Kd + BK - 1) / BK;
+    const uint32_t b_bytes = (uint32_t)a.BN * BK * 4;
+    const uint32_t tx_bytes = A_BYTES + (a.passes > 1 ? 2u : 1u) * b_bytes;
+
+    if (warp == 0 && lane == 0) {
+        // ---------------- TMA producer ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+            const RowSpan sp = a.tiles[t / a.ntn];
+            const int n0 = (t % a.ntn) * a.BN;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!(ok = mbar_wait(empty(stage), phase ^ 1u, abort_flag, a.err, 1))) break;
+                mbar_expect_tx(full(stage), tx_bytes);
+                const uint32_t base = sm_addr + stage * STAGE_BYTES;
+                tma_load_2d(base, &tmA, kb * BK, sp.row0, full(stage));
+                tma_load_3d(base + 2 * A_BYTES, &tmB, kb * BK, n0, sp.k, full(stage));
+                if (a.passes > 1) tma_load_3d(base + 2 * A_BYTES + B_BYTES, &tmBlo, kb * BK, n0, sp.k, full(stage));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---------------- MMA issuer ----------------
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        const uint32_t idesc = instr_desc(a.BN);
+        bool ok = true;
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+            if (!(ok = mbar_wait(tempty(acc), acc_phase ^ 1u, abort_flag, a.err, 2))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t d = tmem_base + (uint32_t)(acc * BN_MAX);
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 3))) break;
+                if (!(ok = mbar_wait(xfull(stage), phase, abort_flag, a.err, 4))) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t base = sm_addr + stage * STAGE_BYTES;
+                const uint64_t a_hi = smem_desc(base), a_lo = smem_desc(base + A_BYTES);
+                const uint64_t b_hi = smem_desc(base + 2 * A_BYTES), b_lo = smem_desc(base + 2 * A_BYTES + B_BYTES);
+                const int nks = min(BK / 8, (a.Kd - kb * BK + 7) / 8);
+                for (int ks = 0; ks < nks; ++ks) {
+                    const uint64_t adv = (uint64_t)(ks * 32 >> 4);   // 8 TF32 values = 32 bytes along K
+                    mma_tf32(d, a_hi + adv, b_hi + adv, idesc, (kb | ks) != 0 ? 1u : 0u);
+                    if (a.passes > 1) {
+                        mma_tf32(d, a_hi + adv, b_lo + adv, idesc, 1u);
+                        mma_tf32(d, a_lo + adv, b_hi + adv, idesc, 1u);
+                    }
+                }
+                mma_commit(empty(stage));     // the stage may be refilled once these MMAs have read it
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            mma_commit(tfull(acc));           // accumulator complete
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    } else if (warp == 2 || warp == 3) {
+        // ---------------- A split: hi = x rounded to TF32, lo = x - hi ----------------
+        const int tt = threadIdx.x - 64;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 5))) break;
+                if (a.passes > 1) {
+                    float4* hi = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES);
+                    float4* lo = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES + A_BYTES);
+#pragma unroll 4
+                    for (int j = 0; j < A_BYTES / 16 / 64; ++j) {
+                        const int i = tt + 64 * j;
+                        const float4 v = hi[i];
+                        float4 h, l;
+                        h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
+                        h.y = tf32_round(v.y); l.y = tf32_round(v.y - h.y);
+                        h.z = tf32_round(v.z); l.z = tf32_round(v.z - h.z);
+                        h.w = tf32_round(v.w); l.w = tf32_round(v.w - h.w);
+                        hi[i] = h;
+                        lo[i] = l;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+                }
+                mbar_arrive(xfull(stage));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp >= 4) {
+        // ---------------- epilogue: tensor memory -> registers -> global ----------------
+        const int q = warp & 3;                    // this warp may read tensor-memory lanes 32q .. 32q+31
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+            const RowSpan sp = a.tiles[t / a.ntn];
+            const int n0 = (t % a.ntn) * a.BN;
+            if (!(ok = mbar_wait(tfull(acc), acc_phase, abort_flag, a.err, 6))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int r = q * 32 + lane;
+            const bool row_ok = r < sp.nrows;
+            const long long row = (long long)sp.row0 + r;
+            for (int c0 = 0; c0 < a.BN && n0 + c0 < a.ldc; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN_MAX + c0), v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int n = n0 + c0 + 4 * j;
+                        if (n >= a.ldc) break;
+                        float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                               __uint_as_float(v[4 * j + 3]));
+                        if (a.mode == 1) {
+                            const float4 h = *reinterpret_cast<const float4*>(a.Hmask + row * a.ldh + n);
+                            o.x = h.x > 0.f ? o.x * a.scale : 0.f;
+                            o.y = h.y > 0.f ? o.y * a.scale : 0.f;
+                            o.z = h.z > 0.f ? o.z * a.scale : 0.f;
+                            o.w = h.w > 0.f ? o.w * a.scale : 0.f;
+                        }
+                        *reinterpret_cast<float4*>(a.C + row * a.ldc + n) = o;
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(tempty(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // Tear-down.  After a time-out, give loads that may still be in flight a bounded chance to land before the
+    // shared memory is released.
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0)
+        for (int s = 0; s < STAGES; ++s)
+            for (uint32_t i = 0; i < 4096u; ++i)
+                if (mbar_try_wait(full(s), 0) || mbar_try_wait(full(s), 1)) break;
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// W_k^(l) [fi x ldw] -> the four K-major operand copies the tensor-core kernels read:
+//   w_hi / w_lo   [K][fi][ldw]    (B of mode 1: rows n = input feature, Kd = output feature)
+//   wt_hi / wt_lo [K][fo][ldkt]   (B of mode 0: rows n = output feature, Kd = input feature)
+__global__ void split_weights_kernel(const float* __restrict__ params, long long pstride, long long w_int, int fi, int fo, int ldw,
+                                     int ldkt, float* __restrict__ w_hi, float* __restrict__ w_lo, float* __restrict__ wt_hi,
+                                     float* __restrict__ wt_lo) {
+    const int k = blockIdx.y;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)fi * ldw) return;
+    const int i = (int)(idx / ldw), j = (int)(idx % ldw);
+    const float w = params[(long long)k * pstride + w_int + idx];
+    const float h = tf32_round(w), l = tf32_round(w - h);
+    w_hi[(long long)k * fi * ldw + idx] = h;
+    w_lo[(long long)k * fi * ldw + idx] = l;
+    if (j < fo) {
+        wt_hi[((long long)k * fo + j) * ldkt + i] = h;
+        wt_lo[((long long)k * fo + j) * ldkt + i] = l;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Weight gradient dW_k = H_k^T dZ_k on the tensor cores: partial[chunk][m][n] = sum over the chunk's rows r of
+// H[r][m] dZ[r][n].  The reduction index is the row, so both operands are "MN-major": a tile of 32 rows x 32
+// values (128 bytes per row, swizzled in 32-byte units) is one block of the canonical layout, blocks of 32 values
+// are 4096 bytes apart (leading byte offset), groups of 4 rows 512 bytes apart (stride byte offset), and one MMA
+// (K = 8) consumes 8 rows.  Both operands are activations, so both are split into hi / lo in shared memory;
+// rows past the end of the chunk are zeroed there.  One CTA per (chunk, 128 x BN output tile).
+// ---------------------------------------------------------------------------------------------
+struct TnArgs {
+    const RowSpan* chunks;
+    int ntm, ntn, BN, M, ldw;   // output tiles per chunk, MMA N, valid output rows, leading dimension of the output
+    float* partial;
+    long long pstride_chunk;
+    int passes;
+    int32_t* err;
+};
+
+// MN-major TF32 tile: layout type 1 (128-byte swizzle of 32-byte units, repeating every 4 rows = 512 bytes), blocks of
+// 32 values 4096 bytes apart (leading byte offset), groups of 4 rows 512 bytes apart (stride byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(4096 >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)1 << 61);
+}
+
+__global__ void __launch_bounds__(256, 1)
+gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmZ, const TnArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+    uint8_t* sm = smem_raw + pad;
+    const uint32_t sm_addr = raw_addr + pad;
+    const uint32_t bars = sm_addr + STAGES * STAGE_BYTES;
+    auto full = [&](int s) { return bars + 8u * s; };
+    auto xfull = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto empty = [&](int s) { return bars + 8u * (2 * STAGES + s); };
+    const uint32_t tfull = bars + 8u * (3 * STAGES);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    constexpr int NSPLIT = 192;   // threads of warps 2..7
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), NSPLIT); mbar_init(empty(s), 1); }
+        mbar_init(tfull, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN_MAX) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tiles_per_chunk = a.ntm * a.ntn;
+    const RowSpan c = a.chunks[blockIdx.x / tiles_per_chunk];
+    const int tile = blockIdx.x % tiles_per_chunk;
+    const int m0 = (tile / a.ntn) * BM, n0 = (tile % a.ntn) * a.BN;
+    const int nkb = (c.nrows + BK - 1) / BK;
+    const int nb_blocks = (a.BN + 31) / 32;                    // 32-value blocks of the B tile
+    const uint32_t tx_bytes = (uint32_t)(4 + nb_blocks) * 4096u;
+    bool ok = true;
+
+    if (warp == 0 && lane == 0) {
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int kb = 0; kb < nkb; ++kb) {
+            if (!(ok = mbar_wait(empty(stage), phase ^ 1u, abort_flag, a.err, 11))) break;
+            mbar_expect_tx(full(stage), tx_bytes);
+            const uint32_t base = sm_addr + stage * STAGE_BYTES;
+            const int r = c.row0 + kb * BK;
+            for (int j = 0; j < 4; ++j) tma_load_2d(base + j * 4096, &tmH, m0 + 32 * j, r, full(stage));
+            for (int j = 0; j < nb_blocks; ++j) tma_load_2d(base + 2 * A_BYTES + j * 4096, &tmZ, n0 + 32 * j, r, full(stage));
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+    } else if (warp == 1 && lane == 0) {
+        int stage = 0;
+        uint32_t phase = 0;
+        const uint32_t idesc = instr_desc(a.BN) | (1u << 15) | (1u << 16);   // A and B MN-major
+        for (int kb = 0; kb < nkb; ++kb) {
+            if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 13))) break;
+            if (!(ok = mbar_wait(xfull(stage), phase, abort_flag, a.err, 14))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t base = sm_addr + stage * STAGE_BYTES;
+            const int nks = min(BK / 8, (c.nrows - kb * BK + 7) / 8);
+            for (int ks = 0; ks < nks; ++ks) {
+                const uint32_t off = (uint32_t)ks * 1024u;   // next group of 8 rows
+                const uint64_t a_hi = smem_desc_mn(base + off), a_lo = smem_desc_mn(base + A_BYTES + off);
+                const uint64_t b_hi = smem_desc_mn(base + 2 * A_BYTES + off), b_lo = smem_desc_mn(base + 2 * A_BYTES + B_BYTES + off);
+                mma_tf32(tmem_base, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
+                if (a.passes > 1) {
+                    mma_tf32(tmem_base, a_hi, b_lo, idesc, 1u);
+                    mma_tf32(tmem_base, a_lo, b_hi, idesc, 1u);
+                }
+            }
+            mma_commit(empty(stage));
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) mma_commit(tfull);
+    } else if (warp >= 2) {
+        // split both operand tiles into hi / lo and zero the rows past the end of the chunk
+        const int tt = threadIdx.x - 64;
+        int stage = 0;
+        uint32_t phase = 0;
+        const int nf4 = (4 + nb_blocks) * 256;                // float4 values of the stage's A and B tiles
+        for (int kb = 0; kb < nkb; ++kb) {
+            if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 15))) break;
+            const int rows_valid = min(BK, c.nrows - kb * BK);
+            if (a.passes > 1 || rows_valid < BK) {
+                uint8_t* sb = sm + stage * STAGE_BYTES;
+                for (int i = tt; i < nf4; i += NSPLIT) {
+                    const int blk = i >> 8, in = i & 255;                         // block of 32 values, float4 inside it
+                    const int row = in >> 3;                                      // 8 float4 per 128-byte row
+                    const int byte_off = (blk < 4 ? blk * 4096 : 2 * A_BYTES + (blk - 4) * 4096) + in * 16;
+                    float4* hi = reinterpret_cast<float4*>(sb + byte_off);
+                    float4* lo = reinterpret_cast<float4*>(sb + byte_off + (blk < 4 ? A_BYTES : B_BYTES));
+                    float4 v = *hi;
+                    if (row >= rows_valid) v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float4 h, l;
+                    h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
+                    h.y = tf32_round(v.y); l.y = tf32_round(v.y - h.y);
+                    h.z = tf32_round(v.z); l.z = tf32_round(v.z - h.z);
+                    h.w = tf32_round(v.w); l.w = tf32_round(v.w - h.w);
+                    *hi = a.passes > 1 ? h : v;
+                    if (a.passes > 1) *lo = l;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+            mbar_arrive(xfull(stage));
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    // epilogue by warps 4..7 once every MMA has completed
+    if (warp >= 4) {
+        const int q = warp & 3;
+        const bool done = mbar_wait(tfull, 0, abort_flag, a.err, 16);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int m = m0 + q * 32 + lane;
+        float* P = a.partial + (long long)(blockIdx.x / tiles_per_chunk) * a.pstride_chunk;
+        for (int c0 = 0; c0 < a.BN && n0 + c0 < a.ldw; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (done && m < a.M) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int n = n0 + c0 + 4 * j;
+                    if (n >= a.ldw) break;
+                    *reinterpret_cast<float4*>(P + (long long)m * a.ldw + n) =
+                        make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                    __uint_as_float(v[4 * j + 3]));
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN_MAX) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+}  // namespace
+
+int tc_bn_for(int n_cols) { return n_cols <= 16 ? 16 : n_cols <= 32 ? 32 : n_cols <= 64 ? 64 : 128; }
+
+// fp32 tensor [outer (z)] x [rows (y)] x [inner (x)], box = 32 floats x box_rows x 1, zero fill outside.  K-major
+// operand tiles use the 128-byte swizzle of 16-byte units; MN-major TF32 tiles need the 128-byte swizzle of
+// 32-byte units (the only MN-major layout the tensor cores accept for 32-bit operands).
+bool tc_make_map(void* out_map, const void* base, uint64_t inner, uint64_t rows, uint64_t outer, uint64_t row_stride_bytes,
+                 uint64_t outer_stride_bytes, uint32_t box_rows, bool mn_major) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const bool three = outer > 0;
+    cuuint64_t dims[3] = {inner, rows, three ? outer : 1};
+    cuuint64_t strides[2] = {row_stride_bytes, outer_stride_bytes};
+    cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(reinterpret_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, three ? 3 : 2, const_cast<void*>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w_int, int fi, int fo, int ldw, int ldkt, int K,
+                                 float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, cudaStream_t s) {
+    const long long n = (long long)fi * ldw;
+    split_weights_kernel<<<dim3((unsigned)((n + 255) / 256), (unsigned)K), 256, 0, s>>>(params, pstride, w_int, fi, fo, ldw, ldkt, w_hi, w_lo,
+                                                                                        wt_hi, wt_lo);
+    ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* mapBlo, int mode, int passes, int Kd, int n_cols,
+                                float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
+                                int32_t* err, int num_sms, cudaStream_t s) {
+    if (ntiles <= 0) return cudaSuccess;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    TcArgs a;
+    a.tiles = tiles; a.ntiles_rows = ntiles; a.BN = tc_bn_for(n_cols); a.ntn = (ldc + a.BN - 1) / a.BN; a.Kd = Kd;
+    a.C = C; a.ldc = ldc; a.Hmask = Hmask; a.ldh = ldh; a.scale = scale; a.mode = mode; a.passes = passes; a.err = err;
+    const long long total = (long long)ntiles * a.ntn;
+    const unsigned grid = (unsigned)(total < num_sms ? total : num_sms);
+    gemm_tc_kernel<<<grid, 256, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
+                                                 *reinterpret_cast<const CUtensorMap*>(mapBlo), a);
+    ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,
+                              int nchunks, float* partial, int32_t* err, cudaStream_t s) {
+    if (nchunks <= 0) return cudaSuccess;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    TnArgs a;
+    a.chunks = chunks; a.BN = tc_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;
+    a.partial = partial; a.pstride_chunk = (long long)M * ldw; a.passes = passes; a.err = err;
+    const unsigned grid = (unsigned)((long long)nchunks * a.ntm * a.ntn);
+    gemm_tn_tc_kernel<<<grid, 256, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapH), *reinterpret_cast<const CUtensorMap*>(mapZ), a);
+    ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace gad

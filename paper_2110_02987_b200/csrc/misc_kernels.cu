@@ -83,13 +83,13 @@ __global__ void loss_final_kernel(const float* __restrict__ loss_partial, const 
 cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_t* label, const uint8_t* train,
                                 const RowSpan* chunks, int nchunks, const float* inv_ntrain, float* dlogits,
                                 float* loss_partial, cudaStream_t s) {
-    if (nchunks > 0)
-        softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial);
+    if (nchunks > 0) {
+        softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_ptr, int K, const float* inv_ntrain,
                               float inv_total, float* loss, int32_t* nonfinite, cudaStream_t s) {
-    loss_final_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(loss_partial, chunk_ptr, K, inv_ntrain, inv_total, loss, nonfinite);
+    loss_final_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(loss_partial, chunk_ptr, K, inv_ntrain, inv_total, loss, nonfinite); ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(256) colsum_chunks_kernel(const float* __restr
 }
 cudaError_t launch_colsum_chunks(const float* G, int ld, const RowSpan* chunks, int nchunks, float* partial,
                                  int64_t pstride_chunk, cudaStream_t s) {
-    if (nchunks > 0) colsum_chunks_kernel<<<(unsigned)nchunks, 256, 0, s>>>(G, ld, chunks, partial, pstride_chunk);
+    if (nchunks > 0) { colsum_chunks_kernel<<<(unsigned)nchunks, 256, 0, s>>>(G, ld, chunks, partial, pstride_chunk); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 
@@ -152,9 +152,9 @@ __global__ void reduce_chunks_kernel(const float* __restrict__ partial, long lon
 }
 cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, const int32_t* chunk_ptr, int K, float* out,
                                  int64_t ostride, int64_t off, int64_t len, cudaStream_t s) {
-    if (len > 0 && K > 0)
+    if (len > 0 && K > 0) {
         reduce_chunks_kernel<<<dim3((unsigned)((len + 255) / 256), (unsigned)K), 256, 0, s>>>(partial, pstride_chunk, chunk_ptr, out,
-                                                                                               ostride, off, len);
+                                                                                               ostride, off, len); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 
@@ -264,12 +264,12 @@ __global__ void __launch_bounds__(256) zeta_final_kernel(const double* __restric
 
 cudaError_t launch_zeta_partial(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
                                 const int32_t* sub_off, const int64_t* deg_sum, double* partial, cudaStream_t s) {
-    if (nchunks > 0) zeta_partial_kernel<<<(unsigned)nchunks, 256, 0, s>>>(X, ld, F, deg, chunks, sub_off, deg_sum, partial);
+    if (nchunks > 0) { zeta_partial_kernel<<<(unsigned)nchunks, 256, 0, s>>>(X, ld, F, deg, chunks, sub_off, deg_sum, partial); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 cudaError_t launch_zeta_final(const double* partial, int F, int ld, const int32_t* chunk_ptr, int K, const int32_t* sub_off,
                               const int64_t* deg_sum, const int64_t* deg_sq, float beta, double* zeta, cudaStream_t s) {
-    zeta_final_kernel<<<(unsigned)K, 256, 0, s>>>(partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta);
+    zeta_final_kernel<<<(unsigned)K, 256, 0, s>>>(partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta); ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -314,9 +314,9 @@ __global__ void __launch_bounds__(256) sgd_consensus_kernel(float* __restrict__ 
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, cudaStream_t s) {
     const long long len4 = len / 4;
-    if (len4 > 0)
+    if (len4 > 0) {
         sgd_consensus_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
-                                                                                                   zeta, weighted, with_sgd);
+                                                                                                   zeta, weighted, with_sgd); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 
@@ -330,7 +330,7 @@ __global__ void weights_kernel(const double* __restrict__ zeta, int K, int weigh
     }
 }
 cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s) {
-    weights_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(zeta, K, weighted, zeta_f, w_f);
+    weights_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(zeta, K, weighted, zeta_f, w_f); ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -345,7 +345,7 @@ __global__ void gather_rows_kernel(const float* __restrict__ Xg, int F, const in
     for (int j = threadIdx.x; j < ld; j += blockDim.x) dst[j] = j < F ? src[j] : 0.f;
 }
 cudaError_t launch_gather_rows(const float* Xg, int F, const int32_t* gid, int64_t Np, float* H0, int ld, cudaStream_t s) {
-    if (Np > 0) gather_rows_kernel<<<(unsigned)Np, 128, 0, s>>>(Xg, F, gid, Np, H0, ld);
+    if (Np > 0) { gather_rows_kernel<<<(unsigned)Np, 128, 0, s>>>(Xg, F, gid, Np, H0, ld); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 __global__ void gather_labels_kernel(const int32_t* __restrict__ yg, const int32_t* __restrict__ gid, long long Np,
@@ -354,7 +354,7 @@ __global__ void gather_labels_kernel(const int32_t* __restrict__ yg, const int32
     if (r < Np) label[r] = yg[gid[r]];
 }
 cudaError_t launch_gather_labels(const int32_t* yg, const int32_t* gid, int64_t Np, int32_t* label, cudaStream_t s) {
-    if (Np > 0) gather_labels_kernel<<<(unsigned)((Np + 255) / 256), 256, 0, s>>>(yg, gid, Np, label);
+    if (Np > 0) { gather_labels_kernel<<<(unsigned)((Np + 255) / 256), 256, 0, s>>>(yg, gid, Np, label); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 // Logits of the core rows back to graph-node order; one CTA per span of core rows.
@@ -369,7 +369,7 @@ __global__ void scatter_core_kernel(const float* __restrict__ logits, int ld, in
 }
 cudaError_t launch_scatter_core(const float* logits, int ld, int C, const int32_t* gid, const RowSpan* core_spans, int nspans,
                                 float* out, cudaStream_t s) {
-    if (nspans > 0) scatter_core_kernel<<<(unsigned)nspans, 256, 0, s>>>(logits, ld, C, gid, core_spans, out);
+    if (nspans > 0) { scatter_core_kernel<<<(unsigned)nspans, 256, 0, s>>>(logits, ld, C, gid, core_spans, out); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 

@@ -2,11 +2,12 @@
 // aggregation half of the layer H^(l+1) = sigma(A~ (H^(l) W^(l)) + b) (Section 3.3, forward equation); run on
 // the transposed store it is the backward aggregation dZ = A~^T dPre.
 //
-// Work split: a group of GROUP lanes (4..32) owns one row and walks its entries; every lane keeps NV float4
-// accumulators, so a group covers 4*GROUP*NV feature columns with 16-byte loads of the dense operand.  Entries
-// are fetched GROUP at a time as packed (column, value) pairs and handed round with shuffles.  Rows come from a
-// list binned by length (heaviest first); rows above the hub threshold get a whole CTA each and a fixed-order
-// shared-memory reduction, so results never depend on scheduling.
+// Work split: a warp owns one row and walks its entries; GROUP lanes (4..32) span the feature columns with NV
+// float4 accumulators each (16-byte loads of the dense operand), and when GROUP < 32 the warp's 32/GROUP
+// sub-groups take different entries of the row at the same time.  Entries are fetched 32 at a time as packed
+// (column, value) pairs and handed round with shuffles.  Rows come from a list binned by length (heaviest
+// first); long rows are cut into parts with a whole CTA per part and fixed-order reductions (shared memory inside
+// a part, a scratch buffer between the parts of one row), so results never depend on scheduling.
 #include "gad_internal.h"
 
 namespace gad {
@@ -68,7 +69,7 @@ __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, i
             if (ep.relu) {
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    x[t] = fmaxf(x[t], 0.f);
+                    x[t] = x[t] > 0.f ? x[t] : (x[t] <= 0.f ? 0.f : x[t]);   // ReLU that lets NaN through
                     if (drop) x[t] = dropout_keep(key, ep.col0 + 4 * v + t, thr) ? x[t] * scale : 0.f;
                 }
             }
@@ -82,124 +83,180 @@ __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, i
     }
 }
 
-template <int NV>
-__device__ __forceinline__ void fma_row(float4 (&acc)[NV], const float* __restrict__ Z, int ldz, int col, float a, int gl,
-                                        int group, int F4) {
-    const float4* zr = reinterpret_cast<const float4*>(Z + (long long)col * ldz);
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-        int v = gl + group * j;
-        if (v < F4) {
-            float4 z = __ldg(zr + v);
-            acc[j].x = fmaf(a, z.x, acc[j].x);
-            acc[j].y = fmaf(a, z.y, acc[j].y);
-            acc[j].z = fmaf(a, z.z, acc[j].z);
-            acc[j].w = fmaf(a, z.w, acc[j].w);
-        }
-    }
-}
-
-// Entries [e0, e1) of one row accumulated by a group of lanes.
+// Entries [e0, e1) of one row accumulated by a whole warp.  The warp fetches 32 packed entries at a time (the
+// next batch is requested before the current one is consumed); with GROUP < 32 the 32/GROUP sub-groups take
+// different entries of the batch, each lane loading its own 16 bytes of the operand row, and the sub-group
+// sums are combined afterwards with a fixed butterfly.
 template <int NV, int GROUP>
 __device__ __forceinline__ void walk_entries(float4 (&acc)[NV], const uint2* __restrict__ ecv, long long e0, long long e1,
-                                             const float* __restrict__ Z, int ldz, int gl, unsigned gmask, int F4) {
-    for (long long e = e0; e < e1; e += GROUP) {
-        uint2 mine = make_uint2(0u, 0u);
-        if (e + gl < e1) mine = __ldg(ecv + e + gl);
-        int cnt = (int)min((long long)GROUP, e1 - e);
-        int t = 0;
-        for (; t + 4 <= cnt; t += 4) {
-            int c0 = __shfl_sync(gmask, (int)mine.x, t + 0, GROUP), c1 = __shfl_sync(gmask, (int)mine.x, t + 1, GROUP);
-            int c2 = __shfl_sync(gmask, (int)mine.x, t + 2, GROUP), c3 = __shfl_sync(gmask, (int)mine.x, t + 3, GROUP);
-            float a0 = __uint_as_float(__shfl_sync(gmask, mine.y, t + 0, GROUP));
-            float a1 = __uint_as_float(__shfl_sync(gmask, mine.y, t + 1, GROUP));
-            float a2 = __uint_as_float(__shfl_sync(gmask, mine.y, t + 2, GROUP));
-            float a3 = __uint_as_float(__shfl_sync(gmask, mine.y, t + 3, GROUP));
-            fma_row<NV>(acc, Z, ldz, c0, a0, gl, GROUP, F4);
-            fma_row<NV>(acc, Z, ldz, c1, a1, gl, GROUP, F4);
-            fma_row<NV>(acc, Z, ldz, c2, a2, gl, GROUP, F4);
-            fma_row<NV>(acc, Z, ldz, c3, a3, gl, GROUP, F4);
+                                             const float* __restrict__ Z, int ldz, int lane, int F4) {
+    constexpr int SG = 32 / GROUP;
+    const int gl = lane & (GROUP - 1), sg = lane / GROUP;
+    uint2 next = make_uint2(0u, 0u);
+    if (e0 + lane < e1) next = __ldg(ecv + e0 + lane);
+    for (long long e = e0; e < e1; e += 32) {
+        const uint2 mine = next;
+        if (e + 32 + lane < e1) next = __ldg(ecv + e + 32 + lane);
+        const int cnt = (int)min(32ll, e1 - e);
+        // U entries per sub-group are in flight together; a slot past the end of the batch re-reads the batch's
+        // first operand row with weight 0, so the loads stay unconditional and can all be issued at once
+        constexpr int U = NV <= 2 ? 4 : (NV <= 4 ? 2 : 1);
+        const int c_first = __shfl_sync(0xffffffffu, (int)mine.x, 0);
+        for (int t = 0; t < cnt; t += U * SG) {
+            int c[U];
+            float a[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int src = t + u * SG + sg;   // entry of the batch this sub-group takes
+                c[u] = __shfl_sync(0xffffffffu, (int)mine.x, src & 31);
+                a[u] = __uint_as_float(__shfl_sync(0xffffffffu, mine.y, src & 31));
+                if (src >= cnt) { a[u] = 0.f; c[u] = c_first; }
+            }
+            float4 z[U][NV];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float4* zr = reinterpret_cast<const float4*>(Z + (long long)c[u] * ldz);
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const int v = gl + GROUP * j;
+                    z[u][j] = v < F4 ? __ldg(zr + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    acc[j].x = fmaf(a[u], z[u][j].x, acc[j].x);
+                    acc[j].y = fmaf(a[u], z[u][j].y, acc[j].y);
+                    acc[j].z = fmaf(a[u], z[u][j].z, acc[j].z);
+                    acc[j].w = fmaf(a[u], z[u][j].w, acc[j].w);
+                }
         }
-        for (; t < cnt; ++t) {
-            int c = __shfl_sync(gmask, (int)mine.x, t, GROUP);
-            float a = __uint_as_float(__shfl_sync(gmask, mine.y, t, GROUP));
-            fma_row<NV>(acc, Z, ldz, c, a, gl, GROUP, F4);
-        }
+    }
+    if (SG > 1) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j)
+#pragma unroll
+            for (int o = GROUP; o < 32; o <<= 1) {
+                acc[j].x += __shfl_xor_sync(0xffffffffu, acc[j].x, o);
+                acc[j].y += __shfl_xor_sync(0xffffffffu, acc[j].y, o);
+                acc[j].z += __shfl_xor_sync(0xffffffffu, acc[j].z, o);
+                acc[j].w += __shfl_xor_sync(0xffffffffu, acc[j].w, o);
+            }
     }
 }
 
+// One warp per row of the binned list.
 template <int NV, int GROUP, bool EPI>
 __global__ void __launch_bounds__(256) spmm_rows_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
                                                         const int32_t* __restrict__ rows, int nrows,
                                                         const float* __restrict__ Z, int ldz, float* __restrict__ out,
                                                         int ldo, int F4, EpiDev ep) {
     const int lane = threadIdx.x & 31;
-    const int gl = lane & (GROUP - 1);
-    const unsigned gmask = GROUP == 32 ? 0xffffffffu : (((1u << GROUP) - 1u) << (lane & ~(GROUP - 1)));
-    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;
+    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (slot >= nrows) return;
     const int row = rows[slot];
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    walk_entries<NV, GROUP>(acc, ecv, rowptr[row], rowptr[row + 1], Z, ldz, gl, gmask, F4);
-    finish_row<NV, EPI>(acc, row, gl, GROUP, F4, out, ldo, ep);
+    walk_entries<NV, GROUP>(acc, ecv, rowptr[row], rowptr[row + 1], Z, ldz, lane, F4);
+    if (lane < GROUP) finish_row<NV, EPI>(acc, row, lane, GROUP, F4, out, ldo, ep);
 }
 
-// One CTA of 8 warps per hub row: warp w takes the w-th eighth of the entries; the eight partial rows are
-// added in warp order.
-template <int NV, bool EPI>
-__global__ void __launch_bounds__(256) spmm_hub_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
-                                                       const int32_t* __restrict__ rows, const float* __restrict__ Z,
-                                                       int ldz, float* __restrict__ out, int ldo, int F4, EpiDev ep) {
-    extern __shared__ float4 part[];  // [8][F4]
+// Long rows are cut into parts of at most kPartEntries entries; one CTA of 8 warps per part, warp w taking
+// the w-th eighth of the part, the eight partial rows added in warp order.  A row that is a single part is
+// finished here; a part of a longer row goes to scratch slot `part.w` and spmm_finish_kernel adds the row's
+// slots in order.
+template <int NV, int GROUP, bool EPI>
+__global__ void __launch_bounds__(256) spmm_parts_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
+                                                         const int4* __restrict__ parts, const float* __restrict__ Z,
+                                                         int ldz, float* __restrict__ out, int ldo, int F4,
+                                                         float* __restrict__ scratch, EpiDev ep) {
+    extern __shared__ float4 part_sm[];  // [8][F4]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int row = rows[blockIdx.x];
-    const long long e0 = rowptr[row], e1 = rowptr[row + 1];
-    const long long per = ((e1 - e0 + 7) / 8 + 31) / 32 * 32;
+    const int4 pt = parts[blockIdx.x];   // {row, first entry (relative to the row), entries, scratch slot or -1}
+    const int row = pt.x;
+    const long long e0 = rowptr[row] + pt.y, e1 = e0 + pt.z;
+    const long long per = ((pt.z + 7) / 8 + 31) / 32 * 32;
     const long long w0 = min(e1, e0 + per * warp), w1 = min(e1, w0 + per);
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    walk_entries<NV, 32>(acc, ecv, w0, w1, Z, ldz, lane, 0xffffffffu, F4);
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-        int v = lane + 32 * j;
-        if (v < F4) part[warp * F4 + v] = acc[j];
-    }
-    __syncthreads();
-    if (warp == 0) {
+    walk_entries<NV, GROUP>(acc, ecv, w0, w1, Z, ldz, lane, F4);
+    if (lane < GROUP) {
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
-            int v = lane + 32 * j;
+            int v = lane + GROUP * j;
+            if (v < F4) part_sm[warp * F4 + v] = acc[j];
+        }
+    }
+    __syncthreads();
+    if (warp == 0 && lane < GROUP) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            int v = lane + GROUP * j;
             float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
             if (v < F4)
                 for (int w = 0; w < 8; ++w) {
-                    float4 p = part[w * F4 + v];
+                    float4 p = part_sm[w * F4 + v];
                     s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
                 }
             acc[j] = s;
         }
-        finish_row<NV, EPI>(acc, row, lane, 32, F4, out, ldo, ep);
+        if (pt.w < 0) {
+            finish_row<NV, EPI>(acc, row, lane, GROUP, F4, out, ldo, ep);
+        } else {
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                int v = lane + GROUP * j;
+                if (v < F4) reinterpret_cast<float4*>(scratch + (long long)pt.w * ldo)[v] = acc[j];
+            }
+        }
     }
+}
+
+// Rows made of several parts: their scratch slots added in part order, then the epilogue.  One warp per row.
+template <int NV, int GROUP, bool EPI>
+__global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict__ fin, int nfin, const float* __restrict__ scratch,
+                                                          float* __restrict__ out, int ldo, int F4, EpiDev ep) {
+    const int lane = threadIdx.x & 31;
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (i >= nfin || lane >= GROUP) return;
+    const int4 f = fin[i];  // {row, first slot, slots, unused}
+    float4 acc[NV];
+#pragma unroll
+    for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = 0; p < f.z; ++p) {
+        const float4* src = reinterpret_cast<const float4*>(scratch + (long long)(f.y + p) * ldo);
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            int v = lane + GROUP * j;
+            if (v < F4) {
+                float4 t = src[v];
+                acc[j].x += t.x; acc[j].y += t.y; acc[j].z += t.z; acc[j].w += t.w;
+            }
+        }
+    }
+    finish_row<NV, EPI>(acc, f.x, lane, GROUP, F4, out, ldo, ep);
 }
 
 template <int NV, int GROUP, bool EPI>
 static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F4, const EpiDev& ep,
                                cudaStream_t s) {
-    if (A.nperm > 0) {
-        const int rows_per_cta = 256 / GROUP;
-        const unsigned grid = (unsigned)((A.nperm + rows_per_cta - 1) / rows_per_cta);
-        spmm_rows_kernel<NV, GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
+    if (A.nparts > 0) {  // long rows first: they are the longest items of work
+        spmm_parts_kernel<NV, GROUP, EPI><<<(unsigned)A.nparts, 256, (size_t)8 * F4 * sizeof(float4), s>>>(A.rowptr, A.ecv, A.parts, Z, ldz,
+                                                                                                          out, ldo, F4, A.scratch, ep);
+        ++g_kernel_launches;
     }
-    return cudaGetLastError();
-}
-template <int NV, bool EPI>
-static cudaError_t launch_hub(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F4, const EpiDev& ep,
-                              cudaStream_t s) {
-    if (A.nhub > 0)
-        spmm_hub_kernel<NV, EPI><<<(unsigned)A.nhub, 256, (size_t)8 * F4 * sizeof(float4), s>>>(A.rowptr, A.ecv, A.hub, Z, ldz,
-                                                                                               out, ldo, F4, ep);
+    if (A.nfin > 0) {
+        spmm_finish_kernel<NV, GROUP, EPI><<<(unsigned)((A.nfin + 7) / 8), 256, 0, s>>>(A.fin, A.nfin, A.scratch, out, ldo, F4, ep);
+        ++g_kernel_launches;
+    }
+    if (A.nperm > 0) {
+        const unsigned grid = (unsigned)((A.nperm + 7) / 8);
+        spmm_rows_kernel<NV, GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
+        ++g_kernel_launches;
+    }
     return cudaGetLastError();
 }
 
@@ -208,16 +265,11 @@ static cudaError_t dispatch(const SparseDev& A, const float* Z, int ldz, float* 
                             cudaStream_t s) {
     cudaError_t e;
 #define GAD_ROWS(NV, G) { e = launch_rows<NV, G, EPI>(A, Z, ldz, out, ldo, F4, ep, s); if (e != cudaSuccess) return e; }
-#define GAD_HUB(NV) { e = launch_hub<NV, EPI>(A, Z, ldz, out, ldo, F4, ep, s); if (e != cudaSuccess) return e; }
-    // hub rows first: they are the longest items of work
-    if (F4 <= 32) GAD_HUB(1) else if (F4 <= 64) GAD_HUB(2) else if (F4 <= 96) GAD_HUB(3) else if (F4 <= 128) GAD_HUB(4)
-    else if (F4 <= 160) GAD_HUB(5) else if (F4 <= 192) GAD_HUB(6) else GAD_HUB(8)
     if (F4 <= 4) GAD_ROWS(1, 4) else if (F4 <= 8) GAD_ROWS(1, 8) else if (F4 <= 16) GAD_ROWS(1, 16)
     else if (F4 <= 32) GAD_ROWS(1, 32) else if (F4 <= 64) GAD_ROWS(2, 32) else if (F4 <= 96) GAD_ROWS(3, 32)
     else if (F4 <= 128) GAD_ROWS(4, 32) else if (F4 <= 160) GAD_ROWS(5, 32) else if (F4 <= 192) GAD_ROWS(6, 32)
     else GAD_ROWS(8, 32)
 #undef GAD_ROWS
-#undef GAD_HUB
     return cudaSuccess;
 }
 

@@ -68,12 +68,13 @@ static inline int32_t node_of(const gad_partition* part, int32_t k, int64_t loca
     return local < nc ? part->core_nodes[part->core_ptr[k] + local] : part->halo_nodes[part->halo_ptr[k] + (local - nc)];
 }
 
-int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, std::string& err) {
+int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, int64_t* slots, std::string& err) {
     HostStore tmp;
     int rc = build_store(g, part, false, tmp, err);
     if (rc != GAD_OK) return rc;
     *Np = tmp.Np;
     *nnz = tmp.nnz;
+    *slots = std::max(count_slots(tmp.rowptr), count_slots(tmp.t_rowptr));
     return GAD_OK;
 }
 
@@ -169,7 +170,14 @@ int build_store(const gad_csr* g, const gad_partition* part, bool values, HostSt
     st.rowptr.assign((size_t)Np + 1, 0);
     for (int64_t r = 0; r < Np; ++r) st.rowptr[r + 1] = st.rowptr[r] + len[r + 1];
     st.nnz = st.rowptr[Np];
-    if (!values) return GAD_OK;
+    if (!values) {
+        // sizes only: the row lengths of the transposed store are the column counts
+        st.t_rowptr.assign((size_t)Np + 1, 0);
+        for (int64_t r = 0; r < Np; ++r)
+            for (int64_t i = 0; i < len[r + 1]; ++i) st.t_rowptr[tcol[ub[r] + i] + 1]++;
+        for (int64_t r = 0; r < Np; ++r) st.t_rowptr[r + 1] += st.t_rowptr[r];
+        return GAD_OK;
+    }
 
     // Compaction and normalisation: d~_i = row sum of (A'_k + I); A~_ij = a_ij / sqrt(d~_i d~_j).
     std::vector<double> dt((size_t)Np);
@@ -219,25 +227,40 @@ int build_store(const gad_csr* g, const gad_partition* part, bool values, HostSt
     return GAD_OK;
 }
 
-void bin_rows(const std::vector<int64_t>& rowptr, int64_t hub_nnz, std::vector<int32_t>& perm, std::vector<int32_t>& hub) {
+int64_t count_slots(const std::vector<int64_t>& rowptr) {
+    int64_t slots = 0;
+    for (size_t r = 0; r + 1 < rowptr.size(); ++r) {
+        int64_t len = rowptr[r + 1] - rowptr[r];
+        if (len > kPartEntries) slots += (len + kPartEntries - 1) / kPartEntries;
+    }
+    return slots;
+}
+
+void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out) {
     const int64_t Np = (int64_t)rowptr.size() - 1;
-    perm.clear();
-    hub.clear();
+    out.perm.clear(); out.parts.clear(); out.fin.clear(); out.slots = 0;
     std::vector<int64_t> count(64, 0);
     auto bin_of = [](int64_t len) { int b = 0; while (len > 1) { len >>= 1; ++b; } return b; };
     for (int64_t r = 0; r < Np; ++r) {
         int64_t len = rowptr[r + 1] - rowptr[r];
-        if (len >= hub_nnz) hub.push_back((int32_t)r);
-        else count[bin_of(len)]++;
+        if (len < kShortRow) count[bin_of(len)]++;
     }
     std::vector<int64_t> start(64, 0);
     int64_t acc = 0;
     for (int b = 63; b >= 0; --b) { start[b] = acc; acc += count[b]; }
-    perm.resize((size_t)acc);
+    out.perm.resize((size_t)acc);
+    // long rows: the rows made of several parts first, longest work first is not needed inside the parts list
+    // because every part is bounded
     for (int64_t r = 0; r < Np; ++r) {
         int64_t len = rowptr[r + 1] - rowptr[r];
-        if (len >= hub_nnz) continue;
-        perm[(size_t)start[bin_of(len)]++] = (int32_t)r;
+        if (len < kShortRow) { out.perm[(size_t)start[bin_of(len)]++] = (int32_t)r; continue; }
+        if (len <= kPartEntries) { out.parts.push_back(make_int4((int)r, 0, (int)len, -1)); continue; }
+        const int64_t np = (len + kPartEntries - 1) / kPartEntries;
+        out.fin.push_back(make_int4((int)r, (int)out.slots, (int)np, 0));
+        for (int64_t p = 0; p < np; ++p)
+            out.parts.push_back(make_int4((int)r, (int)(p * kPartEntries), (int)std::min(kPartEntries, len - p * kPartEntries),
+                                          (int)(out.slots + p)));
+        out.slots += np;
     }
 }
 
