@@ -170,6 +170,32 @@ int gad_profile_count(const gad_ctx* ctx, int32_t* count);
 int gad_profile_read(gad_ctx* ctx, int32_t i, char* name64, int64_t* launches, double* total_ms,
                      double* bytes_per_launch, double* flops_per_launch);
 
+/* The subgraph importance and consensus weights of gad_subgraph_weights, for callers that cannot allocate.
+ * (No counterpart in the paper: it computes the same zeta_k and w_k; only where the intermediate sums live differs.)
+ *
+ * Who needs it: code that runs where a cudaMalloc on its behalf is not possible - the device's memory already
+ * belongs to the host application's own pool, the call comes from inside a framework whose allocator owns the
+ * GPU, or an allocation (which may synchronise the device) has no place in a latency-critical loop.  This entry
+ * point needs no context and no workspace: it takes device inputs and device outputs only, and keeps its partial
+ * sums in a fixed 4 MiB array inside the library image.  Every GPU that loads the library holds that array until
+ * the process exits.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   X        device [rows x ld] floats, 16-byte aligned, row r = features of store row r (columns F..ld-1 ignored)
+ *   deg      device [rows]: degree of each row inside its subgraph, self-loop excluded
+ *   sub_off  device [K+1]: subgraph k owns rows sub_off[k] .. sub_off[k+1]-1, sub_off[K] = rows
+ *   zeta_out, w_out  device [K]
+ *   stream   a cudaStream_t; the four kernels are enqueued on it, the call does not wait
+ * Limits (the size of the fixed array): K <= 256, ld <= 4096, ld a multiple of 4, K * ld <= 16384; anything
+ * larger returns GAD_ERR_RANGE and launches nothing.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that device current);
+ * make that first call outside any stream capture.  All calls share the one array and it keeps the previous
+ * call's contents; every slot a call reads it has first rewritten itself, so nothing needs clearing, but two
+ * calls whose kernels overlap on the GPU (different streams or host threads) race on it - keep them on one
+ * stream or serialise them. */
+int gad_subgraph_weights_static(const float* X, int64_t rows, int32_t F, int32_t ld, const int32_t* deg,
+                                const int32_t* sub_off, int32_t K, float beta, int32_t weighted, float* zeta_out,
+                                float* w_out, void* stream);
+
 /* Number of CUDA kernels this library has launched in this process so far (all contexts). */
 int gad_launch_count(int64_t* launches);
 

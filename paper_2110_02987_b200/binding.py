@@ -24,7 +24,8 @@ SYMBOLS = (
     "gad_workspace_bytes", "gad_create", "gad_train_epoch", "gad_get_loss", "gad_forward", "gad_subgraph_weights",
     "gad_consensus", "gad_get_params", "gad_set_params", "gad_get_grads", "gad_param_count", "gad_store_sizes",
     "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
-    "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_launch_count", "gad_last_error", "gad_destroy",
+    "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_subgraph_weights_static", "gad_launch_count",
+    "gad_last_error", "gad_destroy",
 )
 
 
@@ -296,6 +297,32 @@ class Gad:
             out.append(dict(name=name.value.decode(), launches=int(n.value), total_ms=float(ms.value),
                             bytes_per_launch=float(by.value), flops_per_launch=float(fl.value)))
         return out
+
+
+def subgraph_weights_static(X, deg, sub_off, F, zeta_out, w_out, *, beta=1.0, weighted=True, stream=None):
+    """gad_subgraph_weights_static: zeta_k and w_k without a context, a workspace or any allocation.
+
+    For callers that may not allocate device memory (see include/gad.h).  Every argument is a CUDA torch tensor the
+    caller already owns: X float32 [rows, ld] (ld a multiple of 4), deg int32 [rows], sub_off int32 [K+1], and the
+    outputs zeta_out / w_out float32 [K].  The kernels are enqueued on ``stream`` (default: torch's current stream);
+    the call does not wait.  Limits: K <= 256, ld <= 4096, K * ld <= 16384."""
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream(X.device)
+    if not (X.is_cuda and X.dtype == torch.float32 and X.dim() == 2 and X.is_contiguous()):
+        raise GadError(-1, "X must be a contiguous float32 CUDA matrix")
+    for t, dt in ((deg, torch.int32), (sub_off, torch.int32), (zeta_out, torch.float32), (w_out, torch.float32)):
+        if not (t.is_cuda and t.dtype == dt and t.is_contiguous()):
+            raise GadError(-1, "deg / sub_off must be int32 and zeta_out / w_out float32 contiguous CUDA tensors")
+    K = int(sub_off.numel()) - 1
+    if zeta_out.numel() != K or w_out.numel() != K or deg.numel() != X.shape[0]:
+        raise GadError(-1, "tensor sizes do not match")
+    rc = load().gad_subgraph_weights_static(
+        C.c_void_p(X.data_ptr()), C.c_int64(X.shape[0]), C.c_int32(int(F)), C.c_int32(X.shape[1]), C.c_void_p(deg.data_ptr()),
+        C.c_void_p(sub_off.data_ptr()), C.c_int32(K), C.c_float(beta), C.c_int32(1 if weighted else 0),
+        C.c_void_p(zeta_out.data_ptr()), C.c_void_p(w_out.data_ptr()), C.c_void_p(stream.cuda_stream))
+    if rc != GAD_OK:
+        raise GadError(rc, "gad_subgraph_weights_static")
 
 
 def launch_count() -> int:
