@@ -7,11 +7,11 @@
 // fp32 accuracy from TF32 tensor cores: every operand value x is split into hi = x rounded to a 10-bit mantissa
 // (exactly representable in TF32) and lo = x - hi, rounded the same way, and the product is accumulated as
 // A_hi B_hi + A_hi B_lo + A_lo B_hi in fp32 (the dropped A_lo B_lo term and the rounding of lo are ~2^-22 relative).  B is split once per
-// epoch by a small kernel; A tiles are split in shared memory by two warps of the GEMM kernel.  With passes = 1
+// epoch by a small kernel; A tiles are split in shared memory by four warps of the GEMM kernel.  With passes = 1
 // only A B is issued on the unsplit operands (TF32 operand precision).
 //
-// One persistent CTA per SM, 8 warps: warp 0 issues TMA loads (128B-swizzled tiles) through a 3-stage ring,
-// warps 2-3 split the A tile, warp 1 issues tcgen05.mma, warps 4-7 drain the accumulator (tcgen05.ld) while
+// One persistent CTA per SM, 10 warps: warp 0 issues TMA loads (128B-swizzled tiles) through a 3-stage ring,
+// warps 2-5 split the A tile, warp 1 issues tcgen05.mma, warps 6-9 drain the accumulator (tcgen05.ld) while
 // the MMA warp already fills the second accumulator.  Every mbarrier wait is bounded: on a time-out the CTA
 // raises an error word, stops, frees its tensor memory and returns.
 #include <cuda.h>
@@ -113,13 +113,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 
 // Nearest value with a 10-bit mantissa (ties away from zero), i.e. exactly representable in TF32.
-// Infinities and NaNs pass through unchanged; a finite value that would round up to infinity is truncated.
+// Infinities, NaNs and the few finite values that would round up to infinity pass through unchanged.
 __device__ __forceinline__ float tf32_round(float x) {
     const uint32_t b = __float_as_uint(x);
-    if ((b & 0x7F800000u) == 0x7F800000u) return x;
-    uint32_t r = (b + 0x1000u) & 0xFFFFE000u;
-    if ((r & 0x7F800000u) == 0x7F800000u) r = b & 0xFFFFE000u;
-    return __uint_as_float(r);
+    const uint32_t r = (b + 0x1000u) & 0xFFFFE000u;
+    // keep NaNs (whose payload the addition could carry into the sign bit) and anything that would become infinite
+    return __uint_as_float((b & 0x7FFFFFFFu) < 0x7F7FF000u ? r : b);
 }
 
 struct TcArgs {
@@ -134,7 +133,7 @@ struct TcArgs {
     int32_t* err;
 };
 
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(320, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmBlo, const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -153,7 +152,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), 64); mbar_init(empty(s), 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), 128); mbar_init(empty(s), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 128); }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,7 +222,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mma_commit(tfull(acc));           // accumulator complete
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
-    } else if (warp == 2 || warp == 3) {
+    } else if (warp >= 2 && warp <= 5) {
         // ---------------- A split: hi = x rounded to TF32, lo = x - hi ----------------
         const int tt = threadIdx.x - 64;
         int stage = 0;
@@ -236,8 +235,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     float4* hi = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES);
                     float4* lo = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES + A_BYTES);
 #pragma unroll 4
-                    for (int j = 0; j < A_BYTES / 16 / 64; ++j) {
-                        const int i = tt + 64 * j;
+                    for (int j = 0; j < A_BYTES / 16 / 128; ++j) {
+                        const int i = tt + 128 * j;
                         const float4 v = hi[i];
                         float4 h, l;
                         h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
@@ -253,7 +252,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 6) {
         // ---------------- epilogue: tensor memory -> registers -> global ----------------
         const int q = warp & 3;                    // this warp may read tensor-memory lanes 32q .. 32q+31
         int acc = 0;
@@ -557,7 +556,7 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
     a.C = C; a.ldc = ldc; a.Hmask = Hmask; a.ldh = ldh; a.scale = scale; a.mode = mode; a.passes = passes; a.err = err;
     const long long total = (long long)ntiles * a.ntn;
     const unsigned grid = (unsigned)(total < num_sms ? total : num_sms);
-    gemm_tc_kernel<<<grid, 256, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
+    gemm_tc_kernel<<<grid, 320, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
                                                  *reinterpret_cast<const CUtensorMap*>(mapBlo), a);
     ++g_kernel_launches;
     return cudaGetLastError();

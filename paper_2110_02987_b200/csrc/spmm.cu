@@ -146,6 +146,43 @@ __device__ __forceinline__ void walk_entries(float4 (&acc)[NV], const uint2* __r
     }
 }
 
+// Narrow operands (at most 16 float4 per row): GROUP lanes per short row, 32/GROUP rows per warp.  A group fetches
+// GROUP entries at a time and has all of their operand rows in flight together; a slot past the end of the row
+// re-reads the row's own operand row (its self-loop is in the sum anyway) with weight 0.
+template <int GROUP, bool EPI>
+__global__ void __launch_bounds__(256) spmm_rows_narrow_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
+                                                               const int32_t* __restrict__ rows, int nrows,
+                                                               const float* __restrict__ Z, int ldz, float* __restrict__ out,
+                                                               int ldo, int F4, EpiDev ep) {
+    const int lane = threadIdx.x & 31, gl = lane & (GROUP - 1);
+    const unsigned gmask = ((1u << GROUP) - 1u) << (lane & ~(GROUP - 1));
+    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;
+    if (slot >= nrows) return;
+    const int row = rows[slot];
+    const long long e0 = rowptr[row], e1 = rowptr[row + 1];
+    float4 acc[1] = {make_float4(0.f, 0.f, 0.f, 0.f)};
+    for (long long e = e0; e < e1; e += GROUP) {
+        uint2 mine = make_uint2((uint32_t)row, 0u);
+        if (e + gl < e1) mine = __ldg(ecv + e + gl);
+        float4 z[GROUP];
+        float a[GROUP];
+#pragma unroll
+        for (int t = 0; t < GROUP; ++t) {
+            const int c = __shfl_sync(gmask, (int)mine.x, t, GROUP);
+            a[t] = __uint_as_float(__shfl_sync(gmask, mine.y, t, GROUP));
+            z[t] = gl < F4 ? __ldg(reinterpret_cast<const float4*>(Z + (long long)c * ldz) + gl) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int t = 0; t < GROUP; ++t) {
+            acc[0].x = fmaf(a[t], z[t].x, acc[0].x);
+            acc[0].y = fmaf(a[t], z[t].y, acc[0].y);
+            acc[0].z = fmaf(a[t], z[t].z, acc[0].z);
+            acc[0].w = fmaf(a[t], z[t].w, acc[0].w);
+        }
+    }
+    finish_row<1, EPI>(acc, row, gl, GROUP, F4, out, ldo, ep);
+}
+
 // One warp per row of the binned list.
 template <int NV, int GROUP, bool EPI>
 __global__ void __launch_bounds__(256) spmm_rows_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
@@ -253,8 +290,13 @@ static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, floa
         ++g_kernel_launches;
     }
     if (A.nperm > 0) {
-        const unsigned grid = (unsigned)((A.nperm + 7) / 8);
-        spmm_rows_kernel<NV, GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
+        if constexpr (GROUP < 32) {
+            const unsigned grid = (unsigned)(((long long)A.nperm * GROUP + 255) / 256);
+            spmm_rows_narrow_kernel<GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
+        } else {
+            const unsigned grid = (unsigned)((A.nperm + 7) / 8);
+            spmm_rows_kernel<NV, GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
+        }
         ++g_kernel_launches;
     }
     return cudaGetLastError();
