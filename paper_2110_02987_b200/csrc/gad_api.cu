@@ -31,13 +31,13 @@ struct Plan {
     std::vector<Layer> layers;
     std::vector<int32_t> ld;          // [L+1]
     int32_t maxld = 0;
-    std::vector<RowSpan> tiles, chunks, core_spans;
-    std::vector<int32_t> chunk_ptr;   // [K+1]
+    std::vector<RowSpan> tiles, chunks, dw_chunks, core_spans;
+    std::vector<int32_t> chunk_ptr, dw_chunk_ptr;   // [K+1]
     int64_t dw_partial = 0;           // floats per chunk
     size_t bytes = 0;
     // offsets into the workspace
     size_t o_rowptr, o_ecv, o_perm, o_parts, o_fin, o_trowptr, o_tecv, o_tperm, o_tparts, o_tfin, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
-        o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
+        o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_dw_chunks, o_dw_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
         o_dw_partial, o_cs_partial, o_loss_partial, o_zeta_partial, o_zeta, o_loss, o_flags, o_zeta_f, o_w_f, o_stage,
         o_stage_lab;
     std::vector<size_t> o_H, o_w_hi, o_w_lo, o_wt_hi, o_wt_lo;   // per layer
@@ -81,8 +81,19 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     const int64_t target = 592;
     int64_t R = round_up(std::max<int64_t>(1, (p.Np + target - 1) / target), 32);
     R = std::min<int64_t>(std::max<int64_t>(R, 128), 16384);
+    // The weight gradient has a long reduction per output tile, so it gets longer chunks: about two CTAs per SM over
+    // the layer with the most output tiles (128 x 128 each).
+    int64_t max_tiles = 1;
+    for (const Layer& y : p.layers) max_tiles = std::max<int64_t>(max_tiles, ((y.fi + 127) / 128) * (int64_t)((y.ldw + 127) / 128));
+    int64_t Rdw = round_up(std::max<int64_t>(1, p.Np * max_tiles / 296), 32);
+    // (not longer than 4096 rows: the CTAs that share a chunk then stay close enough to share it in L2)
+    Rdw = std::min<int64_t>(std::max<int64_t>(Rdw, 256), 4096);
     p.chunk_ptr.assign(K + 1, 0);
+    p.dw_chunk_ptr.assign(K + 1, 0);
     for (int32_t k = 0; k < K; ++k) {
+        for (int64_t r = sub_off[k]; r < sub_off[k + 1]; r += Rdw)
+            p.dw_chunks.push_back(RowSpan{(int32_t)r, (int32_t)std::min<int64_t>(Rdw, sub_off[k + 1] - r), k, 0});
+        p.dw_chunk_ptr[k + 1] = (int32_t)p.dw_chunks.size();
         for (int32_t r = sub_off[k]; r < sub_off[k + 1]; r += 128)
             p.tiles.push_back(RowSpan{r, std::min<int32_t>(128, sub_off[k + 1] - r), k, 0});
         for (int64_t r = sub_off[k]; r < sub_off[k + 1]; r += R)
@@ -94,8 +105,8 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     const size_t Np = (size_t)p.Np, nc = p.chunks.size();
     size_t cur = 0;
     p.o_rowptr = take(cur, 8 * (Np + 1)); p.o_ecv = take(cur, 8 * (size_t)nnz);
-    // work lists: at most one part per kShortRow entries plus one per row that is cut
-    const size_t max_parts = (size_t)(nnz / kShortRow + slots + 1), max_fin = (size_t)(nnz / kPartEntries + 1);
+    // work lists: one part per scratch slot, at most one cut row per kMinPart entries
+    const size_t max_parts = (size_t)(slots + 1), max_fin = (size_t)(nnz / kMinPart + 1);
     p.o_perm = take(cur, 4 * Np); p.o_parts = take(cur, 16 * max_parts); p.o_fin = take(cur, 16 * max_fin);
     p.o_trowptr = take(cur, 8 * (Np + 1)); p.o_tecv = take(cur, 8 * (size_t)nnz);
     p.o_tperm = take(cur, 4 * Np); p.o_tparts = take(cur, 16 * max_parts); p.o_tfin = take(cur, 16 * max_fin);
@@ -103,13 +114,17 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_label = take(cur, 4 * Np); p.o_train = take(cur, Np);
     p.o_deg_sum = take(cur, 8 * (size_t)K); p.o_deg_sq = take(cur, 8 * (size_t)K); p.o_inv_ntrain = take(cur, 4 * (size_t)K);
     p.o_tiles = take(cur, sizeof(RowSpan) * p.tiles.size()); p.o_chunks = take(cur, sizeof(RowSpan) * nc);
-    p.o_chunk_ptr = take(cur, 4 * (size_t)(K + 1)); p.o_core_spans = take(cur, sizeof(RowSpan) * p.core_spans.size());
+    p.o_chunk_ptr = take(cur, 4 * (size_t)(K + 1));
+    p.o_dw_chunks = take(cur, sizeof(RowSpan) * p.dw_chunks.size()); p.o_dw_chunk_ptr = take(cur, 4 * (size_t)(K + 1));
+    p.o_core_spans = take(cur, sizeof(RowSpan) * p.core_spans.size());
     p.o_H.resize(p.L + 1);
     for (int l = 0; l <= p.L; ++l) p.o_H[l] = take(cur, 4 * Np * (size_t)p.ld[l]);
-    p.o_spmm_scratch = take(cur, 4 * (size_t)slots * (size_t)p.maxld);
+    int32_t max_spmm_ld = 4;   // the SpMM runs at the widths F_1 .. F_L
+    for (int l = 1; l <= p.L; ++l) max_spmm_ld = std::max(max_spmm_ld, p.ld[l]);
+    p.o_spmm_scratch = take(cur, 4 * (size_t)slots * (size_t)max_spmm_ld);
     p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
     p.o_params = take(cur, 4 * (size_t)K * (size_t)p.pstride); p.o_grads = take(cur, 4 * (size_t)K * (size_t)p.pstride);
-    p.o_dw_partial = take(cur, 4 * nc * (size_t)p.dw_partial); p.o_cs_partial = take(cur, 4 * nc * (size_t)p.maxld);
+    p.o_dw_partial = take(cur, 4 * p.dw_chunks.size() * (size_t)p.dw_partial); p.o_cs_partial = take(cur, 4 * nc * (size_t)p.maxld);
     p.o_loss_partial = take(cur, 4 * nc); p.o_zeta_partial = take(cur, 8 * nc * 2 * (size_t)p.ld[0]);
     p.o_zeta = take(cur, 8 * (size_t)K); p.o_loss = take(cur, 4 * (size_t)(K + 1)); p.o_flags = take(cur, 16);
     p.o_zeta_f = take(cur, 4 * (size_t)K); p.o_w_f = take(cur, 4 * (size_t)K);
@@ -258,6 +273,9 @@ int backward_pass(gad_ctx* ctx) {
     const RowSpan* chunks = ctx->at<RowSpan>(p.o_chunks);
     const int nc = (int)p.chunks.size();
     const int32_t* chunk_ptr = ctx->at<int32_t>(p.o_chunk_ptr);
+    const RowSpan* dw_chunks = ctx->at<RowSpan>(p.o_dw_chunks);
+    const int ndw = (int)p.dw_chunks.size();
+    const int32_t* dw_chunk_ptr = ctx->at<int32_t>(p.o_dw_chunk_ptr);
     const float scale = ctx->cfg.dropout > 0.f ? 1.f / (1.f - ctx->cfg.dropout) : 1.f;
     for (int l = p.L - 1; l >= 0; --l) {
         const Layer& y = p.layers[l];
@@ -272,12 +290,12 @@ int backward_pass(gad_ctx* ctx) {
         GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
             cudaError_t e = ctx->use_tc
                                 ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
-                                                    ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, chunks, nc,
+                                                    ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, dw_chunks, ndw,
                                                     ctx->at<float>(p.o_dw_partial), ctx->at<int32_t>(p.o_flags) + 1, ctx->stream)
-                                : launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, chunks, nc,
+                                : launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, dw_chunks, ndw,
                                                       ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
             if (e != cudaSuccess) return e;
-            return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, chunk_ptr, p.K, grads, p.pstride,
+            return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, dw_chunk_ptr, p.K, grads, p.pstride,
                                         y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
         });
         if (l > 0)
@@ -440,7 +458,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         (rc = upload(ctx, p.o_label, label)) || (rc = upload(ctx, p.o_train, train)) || (rc = upload(ctx, p.o_deg_sum, deg_sum)) ||
         (rc = upload(ctx, p.o_deg_sq, deg_sq)) || (rc = upload(ctx, p.o_inv_ntrain, inv_ntrain)) ||
         (rc = upload(ctx, p.o_tiles, p.tiles)) || (rc = upload(ctx, p.o_chunks, p.chunks)) ||
-        (rc = upload(ctx, p.o_chunk_ptr, p.chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)))
+        (rc = upload(ctx, p.o_chunk_ptr, p.chunk_ptr)) || (rc = upload(ctx, p.o_dw_chunks, p.dw_chunks)) ||
+        (rc = upload(ctx, p.o_dw_chunk_ptr, p.dw_chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)))
         return rc;
     // features: graph order -> staging -> store-row order with zero pad columns
     GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage, X, 4 * (size_t)g->n * p.dims[0], cudaMemcpyHostToDevice, ctx->stream));

@@ -40,16 +40,18 @@ int build_store(const gad_csr* g, const gad_partition* part, bool values, HostSt
 // Sizes only (for gad_workspace_bytes): rows, entries, and the SpMM scratch slots of the worse orientation.
 int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, int64_t* slots, std::string& err);
 
-// Work lists of the SpMM launch.  Rows with fewer than kShortRow entries go to `perm`, binned by
-// floor(log2(entries)), heaviest bin first, ascending row id inside a bin.  Longer rows are cut into parts of at
-// most kPartEntries entries: parts = {row, first entry relative to the row, entries, scratch slot or -1 when the
-// row is a single part}; fin = {row, first scratch slot, slots, 0} for every row made of several parts.
-constexpr int64_t kShortRow = 64, kPartEntries = 512;
+// Work lists of the SpMM launch.  Rows of at most `part_entries` entries go to `perm` (one warp, or one lane
+// group, per row), binned by floor(log2(entries)), heaviest bin first, ascending row id inside a bin.  Longer rows
+// are cut into parts of `part_entries` entries, one warp per part: parts = {row, first entry relative to the row,
+// entries, scratch slot}; fin = {row, first scratch slot, slots, 0} for every row that was cut.  The part length
+// starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most two scratch slots per store row.
+constexpr int64_t kMinPart = 64, kMaxPart = 1024;
 struct RowWork {
     std::vector<int32_t> perm;
     std::vector<int4> parts, fin;
-    int64_t slots = 0;
+    int64_t slots = 0, part_entries = kMinPart;
 };
+int64_t part_entries_for(const std::vector<int64_t>& rowptr);
 void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out);
 // Scratch slots bin_rows would use, from the row lengths alone.
 int64_t count_slots(const std::vector<int64_t>& rowptr);

@@ -59,6 +59,73 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
     }
 }
 
+// Up to 128 classes: L lanes hold one row (a float4 each), 32/L rows per warp step, the row stays in registers.
+template <int L>
+__global__ void __launch_bounds__(256) softmax_xent_small_kernel(const float* __restrict__ logits, int ld, int C,
+                                                                 const int32_t* __restrict__ label,
+                                                                 const uint8_t* __restrict__ train,
+                                                                 const RowSpan* __restrict__ chunks,
+                                                                 const float* __restrict__ inv_ntrain,
+                                                                 float* __restrict__ dlogits, float* __restrict__ loss_partial) {
+    constexpr int RPW = 32 / L;
+    __shared__ float wsum[8];
+    const RowSpan c = chunks[blockIdx.x];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane / L, gl = lane & (L - 1);
+    const unsigned gmask = L == 32 ? 0xffffffffu : (((1u << L) - 1u) << (lane & ~(L - 1)));
+    const int ld4 = ld >> 2;
+    const float inv = inv_ntrain[c.k];
+    float acc = 0.f;
+    for (int r = warp * RPW + g; r < c.nrows; r += 8 * RPW) {
+        const long long row = c.row0 + r;
+        float4* gout = reinterpret_cast<float4*>(dlogits + row * ld);
+        if (!train[row]) {
+            if (gl < ld4) gout[gl] = make_float4(0.f, 0.f, 0.f, 0.f);
+            continue;
+        }
+        float z[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (gl < ld4) {
+            const float4 v = reinterpret_cast<const float4*>(logits + row * ld)[gl];
+            if (4 * gl + 0 < C) z[0] = v.x;
+            if (4 * gl + 1 < C) z[1] = v.y;
+            if (4 * gl + 2 < C) z[2] = v.z;
+            if (4 * gl + 3 < C) z[3] = v.w;
+        }
+        float mx = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+#pragma unroll
+        for (int o = L / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(gmask, mx, o, L));
+        float se = 0.f;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) se += 4 * gl + t < C ? expf(z[t] - mx) : 0.f;
+#pragma unroll
+        for (int o = L / 2; o > 0; o >>= 1) se += __shfl_xor_sync(gmask, se, o, L);
+        const float lse = mx + logf(se);
+        const int y = label[row];
+        const int yt = y & 3;
+        const float mine = yt == 0 ? z[0] : (yt == 1 ? z[1] : (yt == 2 ? z[2] : z[3]));
+        const float zy = __shfl_sync(gmask, mine, y >> 2, L);
+        if (gl == 0) acc += lse - zy;
+        if (gl < ld4) {
+            float o4[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int j = 4 * gl + t;
+                o4[t] = j < C ? (expf(z[t] - lse) - (j == y ? 1.f : 0.f)) * inv : 0.f;
+            }
+            gout[gl] = make_float4(o4[0], o4[1], o4[2], o4[3]);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) wsum[warp] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < 8; ++w) s += wsum[w];
+        loss_partial[blockIdx.x] = s;
+    }
+}
+
 // One thread per subgraph adds that subgraph's chunk sums in chunk order; thread 0 then adds the K subgraph
 // sums in ascending k for the global loss sum_k |T_k| L_k / sum_k |T_k|.
 __global__ void loss_final_kernel(const float* __restrict__ loss_partial, const int32_t* __restrict__ chunk_ptr, int K,
@@ -84,7 +151,18 @@ cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_
                                 const RowSpan* chunks, int nchunks, const float* inv_ntrain, float* dlogits,
                                 float* loss_partial, cudaStream_t s) {
     if (nchunks > 0) {
-        softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial); ++g_kernel_launches; }
+        const int ld4 = ld >> 2;
+#define GAD_SMALL(L) softmax_xent_small_kernel<L><<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial)
+        if (ld4 <= 1) GAD_SMALL(1);
+        else if (ld4 <= 2) GAD_SMALL(2);
+        else if (ld4 <= 4) GAD_SMALL(4);
+        else if (ld4 <= 8) GAD_SMALL(8);
+        else if (ld4 <= 16) GAD_SMALL(16);
+        else if (ld4 <= 32) GAD_SMALL(32);
+        else softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial);
+#undef GAD_SMALL
+        ++g_kernel_launches;
+    }
     return cudaGetLastError();
 }
 cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_ptr, int K, const float* inv_ntrain,
@@ -147,7 +225,16 @@ __global__ void reduce_chunks_kernel(const float* __restrict__ partial, long lon
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= len) return;
     float s = 0.f;
-    for (int c = chunk_ptr[k]; c < chunk_ptr[k + 1]; ++c) s += partial[(long long)c * pstride_chunk + i];
+    const int c1 = chunk_ptr[k + 1];
+    int c = chunk_ptr[k];
+    for (; c + 8 <= c1; c += 8) {   // eight chunks' values requested together, added in chunk order
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = partial[(long long)(c + u) * pstride_chunk + i];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
+    }
+    for (; c < c1; ++c) s += partial[(long long)c * pstride_chunk + i];
     out[(long long)k * ostride + off + i] = s;
 }
 cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, const int32_t* chunk_ptr, int K, float* out,
@@ -237,7 +324,19 @@ __global__ void __launch_bounds__(256) zeta_final_kernel(const double* __restric
     if (n > 0)
         for (int f = threadIdx.x; f < F; f += blockDim.x) {
             double a = 0.0, b = 0.0;
-            for (int c = chunk_ptr[k]; c < chunk_ptr[k + 1]; ++c) {
+            const int c1 = chunk_ptr[k + 1];
+            int c = chunk_ptr[k];
+            for (; c + 8 <= c1; c += 8) {   // eight chunks' values requested together, added in chunk order
+                double va[8], vb[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    va[u] = partial[(long long)(c + u) * 2 * ld + f];
+                    vb[u] = partial[(long long)(c + u) * 2 * ld + ld + f];
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { a += va[u]; b += vb[u]; }
+            }
+            for (; c < c1; ++c) {
                 a += partial[(long long)c * 2 * ld + f];
                 b += partial[(long long)c * 2 * ld + ld + f];
             }

@@ -6,8 +6,8 @@
 // float4 accumulators each (16-byte loads of the dense operand), and when GROUP < 32 the warp's 32/GROUP
 // sub-groups take different entries of the row at the same time.  Entries are fetched 32 at a time as packed
 // (column, value) pairs and handed round with shuffles.  Rows come from a list binned by length (heaviest
-// first); long rows are cut into parts with a whole CTA per part and fixed-order reductions (shared memory inside
-// a part, a scratch buffer between the parts of one row), so results never depend on scheduling.
+// first); long rows are cut into parts with a warp per part and a fixed-order sum of the parts through a scratch
+// buffer, so results never depend on scheduling.
 #include "gad_internal.h"
 
 namespace gad {
@@ -200,54 +200,28 @@ __global__ void __launch_bounds__(256) spmm_rows_kernel(const int64_t* __restric
     if (lane < GROUP) finish_row<NV, EPI>(acc, row, lane, GROUP, F4, out, ldo, ep);
 }
 
-// Long rows are cut into parts of at most kPartEntries entries; one CTA of 8 warps per part, warp w taking
-// the w-th eighth of the part, the eight partial rows added in warp order.  A row that is a single part is
-// finished here; a part of a longer row goes to scratch slot `part.w` and spmm_finish_kernel adds the row's
-// slots in order.
-template <int NV, int GROUP, bool EPI>
+// Long rows are cut into parts; one warp per part, its partial row goes to the part's scratch slot and
+// spmm_finish_kernel adds a row's slots in part order.  No barrier, no shared memory: a warp leaves as soon as
+// its own entries are done.
+template <int NV, int GROUP>
 __global__ void __launch_bounds__(256) spmm_parts_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
-                                                         const int4* __restrict__ parts, const float* __restrict__ Z,
-                                                         int ldz, float* __restrict__ out, int ldo, int F4,
-                                                         float* __restrict__ scratch, EpiDev ep) {
-    extern __shared__ float4 part_sm[];  // [8][F4]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int4 pt = parts[blockIdx.x];   // {row, first entry (relative to the row), entries, scratch slot or -1}
-    const int row = pt.x;
-    const long long e0 = rowptr[row] + pt.y, e1 = e0 + pt.z;
-    const long long per = ((pt.z + 7) / 8 + 31) / 32 * 32;
-    const long long w0 = min(e1, e0 + per * warp), w1 = min(e1, w0 + per);
+                                                         const int4* __restrict__ parts, int nparts,
+                                                         const float* __restrict__ Z, int ldz, int ldo, int F4,
+                                                         float* __restrict__ scratch) {
+    const int lane = threadIdx.x & 31;
+    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (slot >= nparts) return;
+    const int4 pt = parts[slot];   // {row, first entry (relative to the row), entries, scratch slot}
+    const long long e0 = rowptr[pt.x] + pt.y;
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    walk_entries<NV, GROUP>(acc, ecv, w0, w1, Z, ldz, lane, F4);
+    walk_entries<NV, GROUP>(acc, ecv, e0, e0 + pt.z, Z, ldz, lane, F4);
     if (lane < GROUP) {
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
             int v = lane + GROUP * j;
-            if (v < F4) part_sm[warp * F4 + v] = acc[j];
-        }
-    }
-    __syncthreads();
-    if (warp == 0 && lane < GROUP) {
-#pragma unroll
-        for (int j = 0; j < NV; ++j) {
-            int v = lane + GROUP * j;
-            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (v < F4)
-                for (int w = 0; w < 8; ++w) {
-                    float4 p = part_sm[w * F4 + v];
-                    s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
-                }
-            acc[j] = s;
-        }
-        if (pt.w < 0) {
-            finish_row<NV, EPI>(acc, row, lane, GROUP, F4, out, ldo, ep);
-        } else {
-#pragma unroll
-            for (int j = 0; j < NV; ++j) {
-                int v = lane + GROUP * j;
-                if (v < F4) reinterpret_cast<float4*>(scratch + (long long)pt.w * ldo)[v] = acc[j];
-            }
+            if (v < F4) reinterpret_cast<float4*>(scratch + (long long)pt.w * ldo)[v] = acc[j];
         }
     }
 }
@@ -281,8 +255,8 @@ template <int NV, int GROUP, bool EPI>
 static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F4, const EpiDev& ep,
                                cudaStream_t s) {
     if (A.nparts > 0) {  // long rows first: they are the longest items of work
-        spmm_parts_kernel<NV, GROUP, EPI><<<(unsigned)A.nparts, 256, (size_t)8 * F4 * sizeof(float4), s>>>(A.rowptr, A.ecv, A.parts, Z, ldz,
-                                                                                                          out, ldo, F4, A.scratch, ep);
+        spmm_parts_kernel<NV, GROUP><<<(unsigned)((A.nparts + 7) / 8), 256, 0, s>>>(A.rowptr, A.ecv, A.parts, A.nparts, Z, ldz, ldo, F4,
+                                                                                   A.scratch);
         ++g_kernel_launches;
     }
     if (A.nfin > 0) {

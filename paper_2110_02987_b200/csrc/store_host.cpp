@@ -227,39 +227,51 @@ int build_store(const gad_csr* g, const gad_partition* part, bool values, HostSt
     return GAD_OK;
 }
 
+int64_t part_entries_for(const std::vector<int64_t>& rowptr) {
+    const int64_t Np = (int64_t)rowptr.size() - 1;
+    int64_t part = kMinPart;
+    for (; part < kMaxPart; part *= 2) {
+        int64_t slots = 0;
+        for (int64_t r = 0; r < Np; ++r) {
+            const int64_t len = rowptr[r + 1] - rowptr[r];
+            if (len > part) slots += (len + part - 1) / part;
+        }
+        if (slots <= 2 * Np) break;
+    }
+    return part;
+}
+
 int64_t count_slots(const std::vector<int64_t>& rowptr) {
+    const int64_t part = part_entries_for(rowptr);
     int64_t slots = 0;
     for (size_t r = 0; r + 1 < rowptr.size(); ++r) {
-        int64_t len = rowptr[r + 1] - rowptr[r];
-        if (len > kPartEntries) slots += (len + kPartEntries - 1) / kPartEntries;
+        const int64_t len = rowptr[r + 1] - rowptr[r];
+        if (len > part) slots += (len + part - 1) / part;
     }
     return slots;
 }
 
 void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out) {
     const int64_t Np = (int64_t)rowptr.size() - 1;
-    out.perm.clear(); out.parts.clear(); out.fin.clear(); out.slots = 0;
+    const int64_t part = part_entries_for(rowptr);
+    out.perm.clear(); out.parts.clear(); out.fin.clear(); out.slots = 0; out.part_entries = part;
     std::vector<int64_t> count(64, 0);
     auto bin_of = [](int64_t len) { int b = 0; while (len > 1) { len >>= 1; ++b; } return b; };
     for (int64_t r = 0; r < Np; ++r) {
-        int64_t len = rowptr[r + 1] - rowptr[r];
-        if (len < kShortRow) count[bin_of(len)]++;
+        const int64_t len = rowptr[r + 1] - rowptr[r];
+        if (len <= part) count[bin_of(len)]++;
     }
     std::vector<int64_t> start(64, 0);
     int64_t acc = 0;
     for (int b = 63; b >= 0; --b) { start[b] = acc; acc += count[b]; }
     out.perm.resize((size_t)acc);
-    // long rows: the rows made of several parts first, longest work first is not needed inside the parts list
-    // because every part is bounded
     for (int64_t r = 0; r < Np; ++r) {
-        int64_t len = rowptr[r + 1] - rowptr[r];
-        if (len < kShortRow) { out.perm[(size_t)start[bin_of(len)]++] = (int32_t)r; continue; }
-        if (len <= kPartEntries) { out.parts.push_back(make_int4((int)r, 0, (int)len, -1)); continue; }
-        const int64_t np = (len + kPartEntries - 1) / kPartEntries;
+        const int64_t len = rowptr[r + 1] - rowptr[r];
+        if (len <= part) { out.perm[(size_t)start[bin_of(len)]++] = (int32_t)r; continue; }
+        const int64_t np = (len + part - 1) / part;
         out.fin.push_back(make_int4((int)r, (int)out.slots, (int)np, 0));
-        for (int64_t p = 0; p < np; ++p)
-            out.parts.push_back(make_int4((int)r, (int)(p * kPartEntries), (int)std::min(kPartEntries, len - p * kPartEntries),
-                                          (int)(out.slots + p)));
+        for (int64_t q = 0; q < np; ++q)
+            out.parts.push_back(make_int4((int)r, (int)(q * part), (int)std::min(part, len - q * part), (int)(out.slots + q)));
         out.slots += np;
     }
 }

@@ -95,6 +95,8 @@ def check_epoch(g, ref, tol=TOL, loss_tol=1e-5):
     (2, True, False, (6, 5, 3)),
     (3, True, True, (33, 130, 4)),
     (4, False, False, (8, 4)),
+    (5, False, False, (10, 150)),
+    (6, True, False, (7, 9, 40)),
 ])
 def test_small_cases_store_and_one_epoch(seed, directed, weighted, dims):
     case = small_random_case(seed, n=70, K=3, directed=directed, weighted=weighted)
