@@ -44,7 +44,7 @@ int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_
 // group, per row), binned by floor(log2(entries)), heaviest bin first, ascending row id inside a bin.  Longer rows
 // are cut into parts of `part_entries` entries, one warp per part: parts = {row, first entry relative to the row,
 // entries, scratch slot}; fin = {row, first scratch slot, slots, 0} for every row that was cut.  The part length
-// starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most two scratch slots per store row.
+// starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most one scratch slot per two store rows.
 constexpr int64_t kMinPart = 64, kMaxPart = 1024;
 struct RowWork {
     std::vector<int32_t> perm;

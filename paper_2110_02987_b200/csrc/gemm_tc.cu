@@ -27,6 +27,8 @@ constexpr int A_BYTES = BM * BK * 4;                      // 16 KiB
 constexpr int B_BYTES = BN_MAX * BK * 4;                  // 16 KiB
 constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;    // A_hi | A_lo | B_hi | B_lo
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int EPI_BYTES = 4 * 32 * 33 * 4;                // per-warp transpose tiles of the epilogue
+constexpr int SMEM_BYTES_ROWS = SMEM_BYTES + EPI_BYTES;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int TMEM_COLS = 2 * BN_MAX;
 
@@ -149,6 +151,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     auto tempty = [&](int i) { return bars + 8u * (3 * STAGES + 2 + i); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    float* epi_sm = reinterpret_cast<float*>(sm + STAGES * STAGE_BYTES + 256);   // 4 warps x 32 x 33 floats
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -263,30 +266,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int n0 = (t % a.ntn) * a.BN;
             if (!(ok = mbar_wait(tfull(acc), acc_phase, abort_flag, a.err, 6))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int r = q * 32 + lane;
-            const bool row_ok = r < sp.nrows;
-            const long long row = (long long)sp.row0 + r;
+            // A thread receives one accumulator row (32 columns at a time); the warp turns its 32 x 32 block through
+            // shared memory so that 8 lanes write 128 contiguous bytes of one output row.
+            float* tr = epi_sm + (warp - 6) * (32 * 33);
+            const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
             for (int c0 = 0; c0 < a.BN && n0 + c0 < a.ldc; c0 += 32) {
+                const int n = n0 + c0 + sub_c;
+                // the eight mask loads of this lane go out together, ahead of the accumulator read and of any store
+                float4 hm[8];
+                if (a.mode == 1) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = q * 32 + 4 * i + sub_r;
+                        hm[i] = (r < sp.nrows && n < a.ldc)
+                                    ? __ldg(reinterpret_cast<const float4*>(a.Hmask + ((long long)sp.row0 + r) * a.ldh + n))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN_MAX + c0), v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (row_ok) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int n = n0 + c0 + 4 * j;
-                        if (n >= a.ldc) break;
-                        float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
-                                               __uint_as_float(v[4 * j + 3]));
-                        if (a.mode == 1) {
-                            const float4 h = *reinterpret_cast<const float4*>(a.Hmask + row * a.ldh + n);
-                            o.x = h.x > 0.f ? o.x * a.scale : 0.f;
-                            o.y = h.y > 0.f ? o.y * a.scale : 0.f;
-                            o.z = h.z > 0.f ? o.z * a.scale : 0.f;
-                            o.w = h.w > 0.f ? o.w * a.scale : 0.f;
-                        }
-                        *reinterpret_cast<float4*>(a.C + row * a.ldc + n) = o;
+                for (int j = 0; j < 32; ++j) tr[lane * 33 + j] = __uint_as_float(v[j]);
+                __syncwarp();
+                float4 o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float* src = tr + (4 * i + sub_r) * 33 + sub_c;
+                    o[i] = make_float4(src[0], src[1], src[2], src[3]);
+                    if (a.mode == 1) {
+                        o[i].x = hm[i].x > 0.f ? o[i].x * a.scale : 0.f;
+                        o[i].y = hm[i].y > 0.f ? o[i].y * a.scale : 0.f;
+                        o[i].z = hm[i].z > 0.f ? o[i].z * a.scale : 0.f;
+                        o[i].w = hm[i].w > 0.f ? o[i].w * a.scale : 0.f;
                     }
                 }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = q * 32 + 4 * i + sub_r;
+                    if (r < sp.nrows && n < a.ldc) *reinterpret_cast<float4*>(a.C + ((long long)sp.row0 + r) * a.ldc + n) = o[i];
+                }
+                __syncwarp();
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(tempty(acc));
@@ -547,7 +567,7 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
     if (ntiles <= 0) return cudaSuccess;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_ROWS);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -556,7 +576,7 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
     a.C = C; a.ldc = ldc; a.Hmask = Hmask; a.ldh = ldh; a.scale = scale; a.mode = mode; a.passes = passes; a.err = err;
     const long long total = (long long)ntiles * a.ntn;
     const unsigned grid = (unsigned)(total < num_sms ? total : num_sms);
-    gemm_tc_kernel<<<grid, 320, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
+    gemm_tc_kernel<<<grid, 320, SMEM_BYTES_ROWS, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
                                                  *reinterpret_cast<const CUtensorMap*>(mapBlo), a);
     ++g_kernel_launches;
     return cudaGetLastError();

@@ -236,7 +236,7 @@ int64_t part_entries_for(const std::vector<int64_t>& rowptr) {
             const int64_t len = rowptr[r + 1] - rowptr[r];
             if (len > part) slots += (len + part - 1) / part;
         }
-        if (slots <= 2 * Np) break;
+        if (2 * slots <= Np) break;
     }
     return part;
 }
