@@ -34,6 +34,7 @@ struct Plan {
     std::vector<RowSpan> tiles, chunks, dw_chunks, core_spans;
     std::vector<int32_t> chunk_ptr, dw_chunk_ptr;   // [K+1]
     int64_t dw_partial = 0;           // floats per chunk
+    size_t o_counters = 0;            // arrival counters: [loss | K column sums | K zeta]
     size_t bytes = 0;
     // offsets into the workspace
     size_t o_rowptr, o_ecv, o_perm, o_parts, o_fin, o_trowptr, o_tecv, o_tperm, o_tparts, o_tfin, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
@@ -135,6 +136,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         p.o_w_hi[l] = take(cur, 4 * (size_t)K * y.fi * y.ldw); p.o_w_lo[l] = take(cur, 4 * (size_t)K * y.fi * y.ldw);
         p.o_wt_hi[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi); p.o_wt_lo[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi);
     }
+    p.o_counters = take(cur, 4 * (size_t)(1 + 2 * K));
     p.bytes = cur;
     return GAD_OK;
 }
@@ -251,15 +253,12 @@ int forward_pass(gad_ctx* ctx, bool train) {
 
 int zeta_pass(gad_ctx* ctx) {
     const Plan& p = ctx->p;
-    GAD_RUN("zeta_partial", -1, 4.0 * p.Np * (p.dims[0] + 1), 4.0 * p.Np * p.dims[0], [&] {
-        return launch_zeta_partial(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
-                                   (int)p.chunks.size(), ctx->at<int32_t>(p.o_sub_off), ctx->at<int64_t>(p.o_deg_sum),
-                                   ctx->at<double>(p.o_zeta_partial), ctx->stream);
-    });
-    GAD_RUN("zeta_final", -1, 16.0 * p.chunks.size() * p.ld[0], 0.0, [&] {
-        return launch_zeta_final(ctx->at<double>(p.o_zeta_partial), p.dims[0], p.ld[0], ctx->at<int32_t>(p.o_chunk_ptr), p.K,
-                                 ctx->at<int32_t>(p.o_sub_off), ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_deg_sq),
-                                 ctx->cfg.beta, ctx->at<double>(p.o_zeta), ctx->stream);
+    GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 1), 4.0 * p.Np * p.dims[0], [&] {
+        return launch_zeta(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
+                           (int)p.chunks.size(), ctx->at<int32_t>(p.o_chunk_ptr), ctx->at<int32_t>(p.o_sub_off),
+                           ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_deg_sq), ctx->cfg.beta,
+                           ctx->at<double>(p.o_zeta_partial), ctx->at<unsigned>(p.o_counters) + 1 + p.K, ctx->at<double>(p.o_zeta),
+                           ctx->stream);
     });
     return GAD_OK;
 }
@@ -280,20 +279,18 @@ int backward_pass(gad_ctx* ctx) {
     for (int l = p.L - 1; l >= 0; --l) {
         const Layer& y = p.layers[l];
         GAD_RUN("bias_grad", l, 4.0 * p.Np * y.fo, 1.0 * p.Np * y.fo, [&] {
-            cudaError_t e = launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, ctx->stream);
-            if (e != cudaSuccess) return e;
-            return launch_reduce_chunks(ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr, p.K, grads, p.pstride, y.b_int, y.ldo,
-                                        ctx->stream);
+            return launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr,
+                                        ctx->at<unsigned>(p.o_counters) + 1, grads, p.pstride, y.b_int, ctx->stream);
         });
         GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                 [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
         GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
-            cudaError_t e = ctx->use_tc
-                                ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
-                                                    ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, dw_chunks, ndw,
-                                                    ctx->at<float>(p.o_dw_partial), ctx->at<int32_t>(p.o_flags) + 1, ctx->stream)
-                                : launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, dw_chunks, ndw,
-                                                      ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
+            cudaError_t e =
+                ctx->use_tc ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
+                                                ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, dw_chunks, ndw,
+                                                ctx->at<float>(p.o_dw_partial), ctx->at<int32_t>(p.o_flags) + 1, ctx->stream)
+                            : launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, dw_chunks, ndw,
+                                                  ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
             if (e != cudaSuccess) return e;
             return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, dw_chunk_ptr, p.K, grads, p.pstride,
                                         y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
@@ -520,6 +517,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         if (!ok) return fail(ctx, GAD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     }
     GAD_CK(cudaMemsetAsync(ctx->ws + p.o_loss, 0, 4 * (size_t)(p.K + 1), ctx->stream));
+    GAD_CK(cudaMemsetAsync(ctx->ws + p.o_zeta, 0, 8 * (size_t)p.K, ctx->stream));   // empty subgraphs keep zeta = 0
+    GAD_CK(cudaMemsetAsync(ctx->ws + p.o_counters, 0, 4 * (size_t)(1 + 2 * p.K), ctx->stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));
     guard.ok = true;
     *out = ctx;
@@ -552,13 +551,11 @@ int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
     if (rc != GAD_OK) return rc;
     const int C = p.dims[p.L];
     GAD_RUN("softmax_xent", -1, 8.0 * p.Np * C, 0.0, [&] {
-        cudaError_t e = launch_softmax_xent(ctx->H(p.L), p.ld[p.L], C, ctx->at<int32_t>(p.o_label), ctx->at<uint8_t>(p.o_train),
-                                            ctx->at<RowSpan>(p.o_chunks), (int)p.chunks.size(), ctx->at<float>(p.o_inv_ntrain),
-                                            ctx->at<float>(p.o_G1), ctx->at<float>(p.o_loss_partial), ctx->stream);
-        if (e != cudaSuccess) return e;
-        return launch_loss_final(ctx->at<float>(p.o_loss_partial), ctx->at<int32_t>(p.o_chunk_ptr), p.K, ctx->at<float>(p.o_inv_ntrain),
-                                 ctx->ntrain_total > 0 ? 1.f / (float)ctx->ntrain_total : 0.f, ctx->at<float>(p.o_loss),
-                                 ctx->at<int32_t>(p.o_flags), ctx->stream);
+        return launch_softmax_xent(ctx->H(p.L), p.ld[p.L], C, ctx->at<int32_t>(p.o_label), ctx->at<uint8_t>(p.o_train),
+                                   ctx->at<RowSpan>(p.o_chunks), (int)p.chunks.size(), ctx->at<float>(p.o_inv_ntrain),
+                                   ctx->at<float>(p.o_G1), ctx->at<float>(p.o_loss_partial), ctx->at<int32_t>(p.o_chunk_ptr), p.K,
+                                   ctx->ntrain_total > 0 ? 1.f / (float)ctx->ntrain_total : 0.f, ctx->at<float>(p.o_loss),
+                                   ctx->at<int32_t>(p.o_flags), ctx->at<unsigned>(p.o_counters), ctx->stream);
     });
     if ((rc = backward_pass(ctx)) != GAD_OK) return rc;
     if ((rc = zeta_pass(ctx)) != GAD_OK) return rc;

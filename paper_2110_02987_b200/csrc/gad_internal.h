@@ -129,21 +129,24 @@ cudaError_t launch_gemm_tn_simt(const float* H, int ldh, int M, const float* dZ,
 cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, const int32_t* chunk_ptr, int K,
                                  float* out, int64_t ostride, int64_t off, int64_t len, cudaStream_t s);
 
-// partial[chunk][j] = sum over the chunk's rows of G[row][j], j < ld.
-cudaError_t launch_colsum_chunks(const float* G, int ld, const RowSpan* chunks, int nchunks, float* partial,
-                                 int64_t pstride_chunk, cudaStream_t s);
+// The three launchers below are single kernels whose last-arriving CTA (per subgraph, or overall for the loss)
+// finishes the reduction over the chunks in chunk order; `counters` are monotonic arrival counters, zero at creation.
 
+// out[k][off + j] = sum over the rows of subgraph k of G[row][j], j < ld  (counters: one per subgraph).
+cudaError_t launch_colsum_chunks(const float* G, int ld, const RowSpan* chunks, int nchunks, float* partial,
+                                 int64_t pstride_chunk, const int32_t* chunk_ptr, unsigned* counters, float* out,
+                                 int64_t ostride, int64_t off, cudaStream_t s);
+
+// dlogits, and loss[0..K-1] = mean loss of each subgraph, loss[K] = mean over all training rows  (counter: one).
 cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_t* label, const uint8_t* train,
                                 const RowSpan* chunks, int nchunks, const float* inv_ntrain, float* dlogits,
-                                float* loss_partial, cudaStream_t s);
-cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_ptr, int K, const float* inv_ntrain,
-                              float inv_total, float* loss /*[K+1]*/, int32_t* nonfinite, cudaStream_t s);
+                                float* loss_partial, const int32_t* chunk_ptr, int K, float inv_total, float* loss,
+                                int32_t* nonfinite, unsigned* counter, cudaStream_t s);
 
-cudaError_t launch_zeta_partial(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks,
-                                int nchunks, const int32_t* sub_off, const int64_t* deg_sum, double* partial,
-                                cudaStream_t s);
-cudaError_t launch_zeta_final(const double* partial, int F, int ld, const int32_t* chunk_ptr, int K, const int32_t* sub_off,
-                              const int64_t* deg_sum, const int64_t* deg_sq, float beta, double* zeta, cudaStream_t s);
+// zeta[k] of every subgraph that has rows  (counters: one per subgraph).
+cudaError_t launch_zeta(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
+                        const int32_t* chunk_ptr, const int32_t* sub_off, const int64_t* deg_sum, const int64_t* deg_sq,
+                        float beta, double* partial, unsigned* counters, double* zeta, cudaStream_t s);
 
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, cudaStream_t s);

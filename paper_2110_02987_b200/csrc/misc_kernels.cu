@@ -10,6 +10,56 @@
 namespace gad {
 
 // ---------------------------------------------------------------------------------------------
+// "The last CTA finishes the reduction": every CTA writes its partial result, then counts itself in; the CTA
+// whose arrival completes the group adds the partial results in their fixed order.  Which CTA that is varies
+// from run to run, the order of the additions does not, so the results stay bitwise reproducible.  Counters only
+// grow (a group is complete at every multiple of its size), so they never need resetting.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool cta_arrive_last(unsigned* counter, unsigned expected) {
+    __shared__ unsigned last_flag;
+    __threadfence();                  // this CTA's partial results are visible before its arrival is counted
+    __syncthreads();
+    if (threadIdx.x == 0) last_flag = (atomicAdd(counter, 1u) + 1u) % expected == 0u ? 1u : 0u;
+    __syncthreads();
+    const bool last = last_flag != 0u;
+    if (last) __threadfence();        // the other CTAs published their results before they arrived
+    return last;
+}
+
+struct LossTail {
+    const int32_t* chunk_ptr;   // [K+1]
+    int K;
+    float inv_total;
+    float* loss;                // [K+1]
+    int32_t* nonfinite;
+    unsigned* counter;
+};
+
+// One thread per subgraph adds that subgraph's chunk sums in chunk order; thread 0 then adds the K subgraph sums
+// in ascending k for the global loss sum_k |T_k| L_k / sum_k |T_k|.
+__device__ __forceinline__ void loss_finalize(const float* loss_partial, const float* __restrict__ inv_ntrain, const LossTail& t) {
+    __shared__ float sums[1024];
+    for (int k = threadIdx.x; k < t.K; k += blockDim.x) {
+        float s = 0.f;
+        for (int c = t.chunk_ptr[k]; c < t.chunk_ptr[k + 1]; ++c) s += __ldcg(loss_partial + c);
+        if (k < 1024) sums[k] = s;
+        t.loss[k] = s * inv_ntrain[k];
+        if (!isfinite(s)) atomicExch(t.nonfinite, 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int k = 0; k < t.K; ++k) {
+            if (k < 1024) { s += sums[k]; continue; }
+            float sk = 0.f;
+            for (int c = t.chunk_ptr[k]; c < t.chunk_ptr[k + 1]; ++c) sk += __ldcg(loss_partial + c);
+            s += sk;
+        }
+        t.loss[t.K] = s * t.inv_total;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Softmax cross-entropy over the core training rows and d(loss)/d(logits)  (loss equation, Section 3.3, read
 // as multi-class cross-entropy averaged over the subgraph's training nodes).  One CTA per row chunk, one warp
 // per row; lanes stride over the classes.
@@ -19,7 +69,7 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
                                                            const uint8_t* __restrict__ train,
                                                            const RowSpan* __restrict__ chunks,
                                                            const float* __restrict__ inv_ntrain,
-                                                           float* __restrict__ dlogits, float* __restrict__ loss_partial) {
+                                                           float* __restrict__ dlogits, float* loss_partial, LossTail fin) {
     __shared__ float wsum[8];
     const RowSpan c = chunks[blockIdx.x];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -57,6 +107,7 @@ __global__ void __launch_bounds__(256) softmax_xent_kernel(const float* __restri
         for (int w = 0; w < 8; ++w) s += wsum[w];
         loss_partial[blockIdx.x] = s;
     }
+    if (cta_arrive_last(fin.counter, gridDim.x)) loss_finalize(loss_partial, inv_ntrain, fin);
 }
 
 // Up to 128 classes: L lanes hold one row (a float4 each), 32/L rows per warp step, the row stays in registers.
@@ -66,7 +117,7 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(const float* __
                                                                  const uint8_t* __restrict__ train,
                                                                  const RowSpan* __restrict__ chunks,
                                                                  const float* __restrict__ inv_ntrain,
-                                                                 float* __restrict__ dlogits, float* __restrict__ loss_partial) {
+                                                                 float* __restrict__ dlogits, float* loss_partial, LossTail fin) {
     constexpr int RPW = 32 / L;
     __shared__ float wsum[8];
     const RowSpan c = chunks[blockIdx.x];
@@ -124,50 +175,27 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(const float* __
         for (int w = 0; w < 8; ++w) s += wsum[w];
         loss_partial[blockIdx.x] = s;
     }
-}
-
-// One thread per subgraph adds that subgraph's chunk sums in chunk order; thread 0 then adds the K subgraph
-// sums in ascending k for the global loss sum_k |T_k| L_k / sum_k |T_k|.
-__global__ void loss_final_kernel(const float* __restrict__ loss_partial, const int32_t* __restrict__ chunk_ptr, int K,
-                                  const float* __restrict__ inv_ntrain, float inv_total, float* __restrict__ loss,
-                                  int32_t* __restrict__ nonfinite) {
-    extern __shared__ float sums[];
-    for (int k = threadIdx.x; k < K; k += blockDim.x) {
-        float s = 0.f;
-        for (int c = chunk_ptr[k]; c < chunk_ptr[k + 1]; ++c) s += loss_partial[c];
-        sums[k] = s;
-        loss[k] = s * inv_ntrain[k];
-        if (!isfinite(s)) atomicExch(nonfinite, 1);
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float s = 0.f;
-        for (int k = 0; k < K; ++k) s += sums[k];
-        loss[K] = s * inv_total;
-    }
+    if (cta_arrive_last(fin.counter, gridDim.x)) loss_finalize(loss_partial, inv_ntrain, fin);
 }
 
 cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_t* label, const uint8_t* train,
                                 const RowSpan* chunks, int nchunks, const float* inv_ntrain, float* dlogits,
-                                float* loss_partial, cudaStream_t s) {
+                                float* loss_partial, const int32_t* chunk_ptr, int K, float inv_total, float* loss,
+                                int32_t* nonfinite, unsigned* counter, cudaStream_t s) {
     if (nchunks > 0) {
         const int ld4 = ld >> 2;
-#define GAD_SMALL(L) softmax_xent_small_kernel<L><<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial)
+        const LossTail fin{chunk_ptr, K, inv_total, loss, nonfinite, counter};
+#define GAD_SMALL(L) softmax_xent_small_kernel<L><<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial, fin)
         if (ld4 <= 1) GAD_SMALL(1);
         else if (ld4 <= 2) GAD_SMALL(2);
         else if (ld4 <= 4) GAD_SMALL(4);
         else if (ld4 <= 8) GAD_SMALL(8);
         else if (ld4 <= 16) GAD_SMALL(16);
         else if (ld4 <= 32) GAD_SMALL(32);
-        else softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial);
+        else softmax_xent_kernel<<<(unsigned)nchunks, 256, 0, s>>>(logits, ld, C, label, train, chunks, inv_ntrain, dlogits, loss_partial, fin);
 #undef GAD_SMALL
         ++g_kernel_launches;
     }
-    return cudaGetLastError();
-}
-cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_ptr, int K, const float* inv_ntrain,
-                              float inv_total, float* loss, int32_t* nonfinite, cudaStream_t s) {
-    loss_final_kernel<<<1, 256, (size_t)K * sizeof(float), s>>>(loss_partial, chunk_ptr, K, inv_ntrain, inv_total, loss, nonfinite); ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -175,8 +203,10 @@ cudaError_t launch_loss_final(const float* loss_partial, const int32_t* chunk_pt
 // Column sums of a row chunk (bias gradient db = column sums of dPre over the subgraph's rows).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) colsum_chunks_kernel(const float* __restrict__ G, int ld,
-                                                            const RowSpan* __restrict__ chunks,
-                                                            float* __restrict__ partial, long long pstride_chunk) {
+                                                            const RowSpan* __restrict__ chunks, float* partial,
+                                                            long long pstride_chunk, const int32_t* __restrict__ chunk_ptr,
+                                                            unsigned* counters, float* __restrict__ out, long long ostride,
+                                                            long long off) {
     // threads = 8 row lanes x 32 column lanes of one float4 each; a block of 128 columns is summed over the
     // rows ry, ry+8, ... by every row lane and the 8 row lanes are then added in order
     __shared__ float4 sm[8][32];
@@ -211,10 +241,31 @@ __global__ void __launch_bounds__(256) colsum_chunks_kernel(const float* __restr
         }
         __syncthreads();
     }
+    // the last CTA of this subgraph adds the subgraph's chunk sums in chunk order
+    const int c0 = chunk_ptr[c.k], c1 = chunk_ptr[c.k + 1];
+    if (!cta_arrive_last(counters + c.k, (unsigned)(c1 - c0))) return;
+    for (int j = threadIdx.x; j < ld; j += blockDim.x) {
+        float s = 0.f;
+        int cc = c0;
+        for (; cc + 8 <= c1; cc += 8) {   // eight chunks' values requested together, added in chunk order
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldcg(partial + (long long)(cc + u) * pstride_chunk + j);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += v[u];
+        }
+        for (; cc < c1; ++cc) s += __ldcg(partial + (long long)cc * pstride_chunk + j);
+        out[(long long)c.k * ostride + off + j] = s;
+    }
 }
+// Column sums of G over every subgraph's rows: out[k][off + j] = sum over the rows of subgraph k of G[row][j], j < ld.
 cudaError_t launch_colsum_chunks(const float* G, int ld, const RowSpan* chunks, int nchunks, float* partial,
-                                 int64_t pstride_chunk, cudaStream_t s) {
-    if (nchunks > 0) { colsum_chunks_kernel<<<(unsigned)nchunks, 256, 0, s>>>(G, ld, chunks, partial, pstride_chunk); ++g_kernel_launches; }
+                                 int64_t pstride_chunk, const int32_t* chunk_ptr, unsigned* counters, float* out,
+                                 int64_t ostride, int64_t off, cudaStream_t s) {
+    if (nchunks > 0) {
+        colsum_chunks_kernel<<<(unsigned)nchunks, 256, 0, s>>>(G, ld, chunks, partial, pstride_chunk, chunk_ptr, counters, out, ostride, off);
+        ++g_kernel_launches;
+    }
     return cudaGetLastError();
 }
 
@@ -252,12 +303,63 @@ cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, co
 // for any shift c_f; c_f = the subgraph's first row keeps the two sums small.  This kernel accumulates the
 // two weighted sums per chunk and per feature in double precision.
 // ---------------------------------------------------------------------------------------------
+// zeta_k = S_k / (D_k + beta) from the chunk sums of subgraph k, chunks added in order; run by one whole CTA.
+__device__ __forceinline__ void zeta_finalize(int k, const double* partial, int F, int ld, const int32_t* __restrict__ chunk_ptr,
+                                              const int32_t* __restrict__ sub_off, const int64_t* __restrict__ deg_sum,
+                                              const int64_t* __restrict__ deg_sq, float beta, double* __restrict__ zeta) {
+    __shared__ double red[256];
+    const long long n = sub_off[k + 1] - sub_off[k];
+    const bool uniform = deg_sum[k] == 0;
+    const double D = uniform ? (double)n : (double)deg_sum[k];
+    double q = 0.0;
+    if (n > 0)
+        for (int f = threadIdx.x; f < F; f += blockDim.x) {
+            double a = 0.0, b = 0.0;
+            const int c1 = chunk_ptr[k + 1];
+            int c = chunk_ptr[k];
+            for (; c + 8 <= c1; c += 8) {   // eight chunks' values requested together, added in chunk order
+                double va[8], vb[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    va[u] = __ldcg(partial + (long long)(c + u) * 2 * ld + f);
+                    vb[u] = __ldcg(partial + (long long)(c + u) * 2 * ld + ld + f);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { a += va[u]; b += vb[u]; }
+            }
+            for (; c < c1; ++c) {
+                a += __ldcg(partial + (long long)c * 2 * ld + f);
+                b += __ldcg(partial + (long long)c * 2 * ld + ld + f);
+            }
+            const double m1 = a / D;
+            q += b / D - m1 * m1;
+        }
+    red[threadIdx.x] = q;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        double z = 0.0;
+        if (n > 0) {
+            const double sq = uniform ? 1.0 / (double)n : (double)deg_sq[k] / (D * D);
+            const double S = 0.5 * (1.0 - sq);
+            const double Q = red[0] > 0.0 ? red[0] : 0.0;
+            if (S > 0.0) z = S / (sqrt(Q / S) + (double)beta);
+        }
+        zeta[k] = z;
+    }
+}
+
 __global__ void __launch_bounds__(256) zeta_partial_kernel(const float* __restrict__ X, int ld, int F,
                                                            const int32_t* __restrict__ deg,
                                                            const RowSpan* __restrict__ chunks,
                                                            const int32_t* __restrict__ sub_off,
-                                                           const int64_t* __restrict__ deg_sum,
-                                                           double* __restrict__ partial) {
+                                                           const int64_t* __restrict__ deg_sum, double* partial,
+                                                           const int32_t* __restrict__ chunk_ptr,
+                                                           const int64_t* __restrict__ deg_sq, float beta,
+                                                           unsigned* counters, double* __restrict__ zeta) {
     // threads = 8 row lanes x 32 column lanes of one float4 each (as in the column sums above)
     __shared__ double sm[8][32][8];
     const RowSpan c = chunks[blockIdx.x];
@@ -307,68 +409,20 @@ __global__ void __launch_bounds__(256) zeta_partial_kernel(const float* __restri
         }
         __syncthreads();
     }
+    // the last CTA of this subgraph turns the chunk sums into zeta_k
+    if (cta_arrive_last(counters + c.k, (unsigned)(chunk_ptr[c.k + 1] - chunk_ptr[c.k])))
+        zeta_finalize(c.k, partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta);
 }
 
-__global__ void __launch_bounds__(256) zeta_final_kernel(const double* __restrict__ partial, int F, int ld,
-                                                         const int32_t* __restrict__ chunk_ptr,
-                                                         const int32_t* __restrict__ sub_off,
-                                                         const int64_t* __restrict__ deg_sum,
-                                                         const int64_t* __restrict__ deg_sq, float beta,
-                                                         double* __restrict__ zeta) {
-    __shared__ double red[256];
-    const int k = blockIdx.x;
-    const long long n = sub_off[k + 1] - sub_off[k];
-    const bool uniform = deg_sum[k] == 0;
-    const double D = uniform ? (double)n : (double)deg_sum[k];
-    double q = 0.0;
-    if (n > 0)
-        for (int f = threadIdx.x; f < F; f += blockDim.x) {
-            double a = 0.0, b = 0.0;
-            const int c1 = chunk_ptr[k + 1];
-            int c = chunk_ptr[k];
-            for (; c + 8 <= c1; c += 8) {   // eight chunks' values requested together, added in chunk order
-                double va[8], vb[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    va[u] = partial[(long long)(c + u) * 2 * ld + f];
-                    vb[u] = partial[(long long)(c + u) * 2 * ld + ld + f];
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) { a += va[u]; b += vb[u]; }
-            }
-            for (; c < c1; ++c) {
-                a += partial[(long long)c * 2 * ld + f];
-                b += partial[(long long)c * 2 * ld + ld + f];
-            }
-            const double m1 = a / D;
-            q += b / D - m1 * m1;
-        }
-    red[threadIdx.x] = q;
-    __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) {
-        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
-        __syncthreads();
+// zeta[k] for every subgraph that has rows (the entry of an empty subgraph is left as it is: zero since creation).
+cudaError_t launch_zeta(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
+                        const int32_t* chunk_ptr, const int32_t* sub_off, const int64_t* deg_sum, const int64_t* deg_sq,
+                        float beta, double* partial, unsigned* counters, double* zeta, cudaStream_t s) {
+    if (nchunks > 0) {
+        zeta_partial_kernel<<<(unsigned)nchunks, 256, 0, s>>>(X, ld, F, deg, chunks, sub_off, deg_sum, partial, chunk_ptr, deg_sq, beta,
+                                                              counters, zeta);
+        ++g_kernel_launches;
     }
-    if (threadIdx.x == 0) {
-        double z = 0.0;
-        if (n > 0) {
-            const double sq = uniform ? 1.0 / (double)n : (double)deg_sq[k] / (D * D);
-            const double S = 0.5 * (1.0 - sq);
-            const double Q = red[0] > 0.0 ? red[0] : 0.0;
-            if (S > 0.0) z = S / (sqrt(Q / S) + (double)beta);
-        }
-        zeta[k] = z;
-    }
-}
-
-cudaError_t launch_zeta_partial(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
-                                const int32_t* sub_off, const int64_t* deg_sum, double* partial, cudaStream_t s) {
-    if (nchunks > 0) { zeta_partial_kernel<<<(unsigned)nchunks, 256, 0, s>>>(X, ld, F, deg, chunks, sub_off, deg_sum, partial); ++g_kernel_launches; }
-    return cudaGetLastError();
-}
-cudaError_t launch_zeta_final(const double* partial, int F, int ld, const int32_t* chunk_ptr, int K, const int32_t* sub_off,
-                              const int64_t* deg_sum, const int64_t* deg_sq, float beta, double* zeta, cudaStream_t s) {
-    zeta_final_kernel<<<(unsigned)K, 256, 0, s>>>(partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta); ++g_kernel_launches;
     return cudaGetLastError();
 }
 
