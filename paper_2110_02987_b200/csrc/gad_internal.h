@@ -45,10 +45,13 @@ int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_
 // are cut into parts of `part_entries` entries, one warp per part: parts = {row, first entry relative to the row,
 // entries, scratch slot}; fin = {row, first scratch slot, slots, 0} for every row that was cut.  The part length
 // starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most one scratch slot per two store rows.
+// items = every part and every uncut row as {row, low 32 bits of the first entry's position in the store,
+// (high bits << 16) | entries, scratch slot or -1 for an uncut row}, longest first (same binning): the work list of
+// the one-warp-per-item kernel that serves operands of more than 64 columns.
 constexpr int64_t kMinPart = 64, kMaxPart = 1024;
 struct RowWork {
     std::vector<int32_t> perm;
-    std::vector<int4> parts, fin;
+    std::vector<int4> parts, fin, items;
     int64_t slots = 0, part_entries = kMinPart;
 };
 int64_t part_entries_for(const std::vector<int64_t>& rowptr);
@@ -65,8 +68,9 @@ struct SparseDev {
     const int32_t* perm = nullptr;    // binned short rows
     const int4* parts = nullptr;      // parts of the long rows
     const int4* fin = nullptr;        // rows made of several parts
+    const int4* items = nullptr;      // parts and uncut rows together, longest first
     float* scratch = nullptr;         // [slots x leading dimension of the output] partial rows
-    int32_t nperm = 0, nparts = 0, nfin = 0;
+    int32_t nperm = 0, nparts = 0, nfin = 0, nitems = 0;
 };
 
 struct Layer {

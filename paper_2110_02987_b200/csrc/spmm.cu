@@ -45,7 +45,9 @@ struct EpiDev {
     long long pstride, b_int;
     const int32_t* sub_off;
     int K, relu, layer, col0;
-    float dropout;
+    int drop;             // dropout is applied (rate > 0 on a layer with ReLU)
+    uint32_t thr;         // keep an element when the top 24 bits of its hash reach this
+    float scale;          // 1 / (1 - rate)
     unsigned long long seed;
     long long epoch;
 };
@@ -56,9 +58,9 @@ __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, i
     if (EPI) {
         const int k = find_sub(ep.sub_off, ep.K, row);
         const float4* bias = reinterpret_cast<const float4*>(ep.params + (long long)k * ep.pstride + ep.b_int);
-        const bool drop = ep.dropout > 0.f && ep.relu;
-        const float scale = drop ? 1.f / (1.f - ep.dropout) : 1.f;
-        const uint32_t thr = drop ? (uint32_t)floor((double)ep.dropout * 16777216.0) : 0u;
+        const bool drop = ep.drop != 0;
+        const float scale = ep.scale;
+        const uint32_t thr = ep.thr;
         const uint64_t key = drop ? dropout_row_key(ep.seed, ep.epoch, ep.layer, row) : 0ull;
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
@@ -237,23 +239,143 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int p = 0; p < f.z; ++p) {
-        const float4* src = reinterpret_cast<const float4*>(scratch + (long long)(f.y + p) * ldo);
+    // four slots are loaded together and added in slot order (a slot past the last one counts as zero)
+    constexpr int Q = NV <= 2 ? 4 : (NV <= 4 ? 2 : 1);
+    for (int p = 0; p < f.z; p += Q) {
+        float4 t[Q][NV];
 #pragma unroll
-        for (int j = 0; j < NV; ++j) {
-            int v = lane + GROUP * j;
-            if (v < F4) {
-                float4 t = src[v];
-                acc[j].x += t.x; acc[j].y += t.y; acc[j].z += t.z; acc[j].w += t.w;
+        for (int q = 0; q < Q; ++q) {
+            const float4* src = reinterpret_cast<const float4*>(scratch + (long long)(f.y + p + q) * ldo);
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                const int v = lane + GROUP * j;
+                t[q][j] = (p + q < f.z && v < F4) ? src[v] : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
+#pragma unroll
+        for (int q = 0; q < Q; ++q)
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                acc[j].x += t[q][j].x; acc[j].y += t[q][j].y; acc[j].z += t[q][j].z; acc[j].w += t[q][j].w;
+            }
     }
     finish_row<NV, EPI>(acc, f.x, lane, GROUP, F4, out, ldo, ep);
+}
+
+// ---- operands wider than 64 columns: one warp per item of the unified list (a whole row or a part of a cut row) ----
+//
+// The warp stages 32 packed entries in shared memory (slots past the end of the item hold the item's own row with
+// weight 0, so every later read is unconditional), then every lane reads them back two at a time with one
+// 16-byte shared load, turns each column into an address with one multiply-add, and keeps UU operand rows
+// (16 bytes per lane each) in flight before the multiply-adds.  The last entries of a batch go through the
+// next smaller power of two, so a batch costs at most one round trip more than its full groups.
+template <int NV, int UU>
+__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const char* const (&zl)[NV], uint32_t ldzb) {
+    uint32_t c[UU];
+    float a[UU];
+    if constexpr (UU == 1) {
+        const uint2 v = st[0];
+        c[0] = v.x; a[0] = __uint_as_float(v.y);
+    } else {
+#pragma unroll
+        for (int p = 0; p < UU / 2; ++p) {
+            const uint4 v = reinterpret_cast<const uint4*>(st)[p];
+            c[2 * p] = v.x; a[2 * p] = __uint_as_float(v.y);
+            c[2 * p + 1] = v.z; a[2 * p + 1] = __uint_as_float(v.w);
+        }
+    }
+    float4 z[UU][NV];
+#pragma unroll
+    for (int u = 0; u < UU; ++u)
+#pragma unroll
+        for (int j = 0; j < NV; ++j)
+            z[u][j] = __ldg(reinterpret_cast<const float4*>(zl[j] + (unsigned long long)c[u] * ldzb));
+#pragma unroll
+    for (int u = 0; u < UU; ++u)
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            acc[j].x = fmaf(a[u], z[u][j].x, acc[j].x);
+            acc[j].y = fmaf(a[u], z[u][j].y, acc[j].y);
+            acc[j].z = fmaf(a[u], z[u][j].z, acc[j].z);
+            acc[j].w = fmaf(a[u], z[u][j].w, acc[j].w);
+        }
+}
+
+template <int NV, int V>
+__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const char* const (&zl)[NV], uint32_t ldzb) {
+    if constexpr (V >= 1) {
+        if (r > V / 2) gather_fma<NV, V>(acc, st, zl, ldzb);
+        else gather_tail<NV, V / 2>(acc, st, r, zl, ldzb);
+    }
+}
+
+constexpr int kItemWarps = 4;
+template <int NV> struct ItemCfg {
+    static constexpr int UU = NV == 1 ? 8 : (NV == 2 ? 4 : (NV <= 4 ? 2 : 1));   // operand rows in flight per lane
+    static constexpr int MINB = NV <= 2 ? 8 : (NV <= 4 ? 6 : 4);                // resident CTAs asked of the compiler
+};
+
+template <int NV, bool EPI>
+__global__ void __launch_bounds__(32 * kItemWarps, ItemCfg<NV>::MINB)
+spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z,
+                  int ldz, float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
+    constexpr int UU = ItemCfg<NV>::UU;
+    __shared__ __align__(16) uint2 stage_all[kItemWarps][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int idx = blockIdx.x * kItemWarps + warp;
+    if (idx >= nitems) return;
+    uint2* stage = stage_all[warp];
+    const int4 it = __ldg(items + idx);   // {row, entry position low, (position high << 16) | entries, scratch slot or -1}
+    const int row = it.x, len = (int)((uint32_t)it.z & 0xFFFFu);
+    const uint2* ent = ecv + (((long long)((uint32_t)it.z >> 16) << 32) | (long long)(uint32_t)it.y);
+    const uint2 pad = make_uint2((uint32_t)row, 0u);
+    // per-lane operand pointers; lanes past the last column read the last one (their sums are never stored)
+    const char* zl[NV];
+#pragma unroll
+    for (int j = 0; j < NV; ++j) zl[j] = reinterpret_cast<const char*>(Z) + 16ll * min(lane + 32 * j, F4 - 1);
+    const uint32_t ldzb = 4u * (uint32_t)ldz;
+    float4 acc[NV];
+#pragma unroll
+    for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    uint2 next = lane < len ? __ldg(ent + lane) : pad;
+    for (int b = 0; b < len; b += 32) {
+        const uint2 mine = next;
+        const int cnt = min(32, len - b);
+        next = b + 32 + lane < len ? __ldg(ent + b + 32 + lane) : pad;
+        __syncwarp();   // the previous batch has been read by every lane
+        stage[lane] = mine;
+        __syncwarp();
+        int t = 0;
+        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU>(acc, stage + t, zl, ldzb);
+        gather_tail<NV, UU / 2>(acc, stage + t, cnt - t, zl, ldzb);
+    }
+    if (it.w >= 0) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            const int v = lane + 32 * j;
+            if (v < F4) reinterpret_cast<float4*>(scratch + (long long)it.w * ldo)[v] = acc[j];
+        }
+    } else {
+        finish_row<NV, EPI>(acc, row, lane, 32, F4, out, ldo, ep);
+    }
 }
 
 template <int NV, int GROUP, bool EPI>
 static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F4, const EpiDev& ep,
                                cudaStream_t s) {
+    if constexpr (GROUP == 32) {
+        if (A.nitems > 0) {
+            spmm_items_kernel<NV, EPI><<<(unsigned)((A.nitems + kItemWarps - 1) / kItemWarps), 32 * kItemWarps, 0, s>>>(
+                A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+            ++g_kernel_launches;
+        }
+        if (A.nfin > 0) {
+            spmm_finish_kernel<NV, GROUP, EPI><<<(unsigned)((A.nfin + 7) / 8), 256, 0, s>>>(A.fin, A.nfin, A.scratch, out, ldo, F4, ep);
+            ++g_kernel_launches;
+        }
+        return cudaGetLastError();
+    }
     if (A.nparts > 0) {  // long rows first: they are the longest items of work
         spmm_parts_kernel<NV, GROUP><<<(unsigned)((A.nparts + 7) / 8), 256, 0, s>>>(A.rowptr, A.ecv, A.parts, A.nparts, Z, ldz, ldo, F4,
                                                                                    A.scratch);
@@ -299,7 +421,10 @@ cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out,
         if (epi) {
             ep.params = epi->params; ep.pstride = epi->pstride; ep.b_int = epi->b_int + 4ll * c0;
             ep.sub_off = epi->sub_off; ep.K = epi->K; ep.relu = epi->relu; ep.layer = epi->layer;
-            ep.dropout = epi->dropout; ep.seed = epi->seed; ep.epoch = epi->epoch; ep.col0 = 4 * c0;
+            ep.drop = epi->dropout > 0.f && epi->relu;
+            ep.thr = ep.drop ? (uint32_t)floor((double)epi->dropout * 16777216.0) : 0u;
+            ep.scale = ep.drop ? 1.f / (1.f - epi->dropout) : 1.f;
+            ep.seed = epi->seed; ep.epoch = epi->epoch; ep.col0 = 4 * c0;
         }
         cudaError_t e = epi ? dispatch<true>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s)
                             : dispatch<false>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s);

@@ -254,7 +254,7 @@ int64_t count_slots(const std::vector<int64_t>& rowptr) {
 void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out) {
     const int64_t Np = (int64_t)rowptr.size() - 1;
     const int64_t part = part_entries_for(rowptr);
-    out.perm.clear(); out.parts.clear(); out.fin.clear(); out.slots = 0; out.part_entries = part;
+    out.perm.clear(); out.parts.clear(); out.fin.clear(); out.items.clear(); out.slots = 0; out.part_entries = part;
     std::vector<int64_t> count(64, 0);
     auto bin_of = [](int64_t len) { int b = 0; while (len > 1) { len >>= 1; ++b; } return b; };
     for (int64_t r = 0; r < Np; ++r) {
@@ -273,6 +273,21 @@ void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out) {
         for (int64_t q = 0; q < np; ++q)
             out.parts.push_back(make_int4((int)r, (int)(q * part), (int)std::min(part, len - q * part), (int)(out.slots + q)));
         out.slots += np;
+    }
+    // the unified list: parts and uncut rows, longest first
+    auto pack = [&](int64_t row, int64_t e0, int64_t len, int64_t slot) {
+        return make_int4((int)row, (int)(uint32_t)(e0 & 0xFFFFFFFFll), (int)(uint32_t)(((e0 >> 32) << 16) | len), (int)slot);
+    };
+    std::vector<int64_t> icount(64, 0), istart(64, 0);
+    for (const int4& pt : out.parts) icount[bin_of(pt.z)]++;
+    for (int32_t r : out.perm) icount[bin_of(rowptr[r + 1] - rowptr[r])]++;
+    acc = 0;
+    for (int b = 63; b >= 0; --b) { istart[b] = acc; acc += icount[b]; }
+    out.items.resize((size_t)acc);
+    for (const int4& pt : out.parts) out.items[(size_t)istart[bin_of(pt.z)]++] = pack(pt.x, rowptr[pt.x] + pt.y, pt.z, pt.w);
+    for (int32_t r : out.perm) {
+        const int64_t len = rowptr[r + 1] - rowptr[r];
+        out.items[(size_t)istart[bin_of(len)]++] = pack(r, rowptr[r], len, -1);
     }
 }
 
