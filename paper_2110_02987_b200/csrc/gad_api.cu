@@ -334,7 +334,8 @@ uint64_t host_mix64(uint64_t z) {
     return z ^ (z >> 31);
 }
 
-int upload_sparse(gad_ctx* ctx, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col, const std::vector<float>& val,
+int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col,
+                  const std::vector<float>& val,
                   size_t o_rowptr, size_t o_ecv, size_t o_perm, size_t o_parts, size_t o_fin, size_t o_items, SparseDev& out) {
     const Plan& p = ctx->p;
     std::vector<uint2> ecv(col.size());
@@ -344,7 +345,7 @@ int upload_sparse(gad_ctx* ctx, const std::vector<int64_t>& rowptr, const std::v
         ecv[e] = make_uint2((uint32_t)col[e], bits);
     }
     RowWork work;
-    bin_rows(rowptr, work);
+    bin_rows(rowptr, sub_off, work);
     if (work.slots > p.slots) return fail(ctx, GAD_ERR_OOM, "SpMM scratch slots exceed the planned count");
     const std::vector<int32_t>& perm = work.perm;
     GAD_CK(cudaMemcpyAsync(ctx->ws + o_rowptr, rowptr.data(), 8 * rowptr.size(), cudaMemcpyHostToDevice, ctx->stream));
@@ -364,6 +365,7 @@ int upload_sparse(gad_ctx* ctx, const std::vector<int64_t>& rowptr, const std::v
     out.fin = ctx->at<int4>(o_fin);
     out.items = ctx->at<int4>(o_items);
     out.nitems = (int32_t)work.items.size();
+    out.nrows = (int64_t)rowptr.size() - 1;
     out.scratch = ctx->at<float>(p.o_spmm_scratch);
     out.nperm = (int32_t)perm.size();
     out.nparts = (int32_t)work.parts.size();
@@ -431,10 +433,10 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->sub_off = st.sub_off;
     ctx->gid = st.gid;
 
-    rc = upload_sparse(ctx, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_perm, p.o_parts, p.o_fin, p.o_items, ctx->A);
+    rc = upload_sparse(ctx, st.sub_off, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_perm, p.o_parts, p.o_fin, p.o_items, ctx->A);
     if (rc != GAD_OK) return rc;
     if (!st.symmetric) {
-        rc = upload_sparse(ctx, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tperm, p.o_tparts, p.o_tfin, p.o_titems, ctx->At);
+        rc = upload_sparse(ctx, st.sub_off, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tperm, p.o_tparts, p.o_tfin, p.o_titems, ctx->At);
         if (rc != GAD_OK) return rc;
     }
     // per-row labels and loss mask, per-subgraph degree sums and training counts

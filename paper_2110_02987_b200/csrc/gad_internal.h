@@ -46,7 +46,8 @@ int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_
 // entries, scratch slot}; fin = {row, first scratch slot, slots, 0} for every row that was cut.  The part length
 // starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most one scratch slot per two store rows.
 // items = every part and every uncut row as {row, low 32 bits of the first entry's position in the store,
-// (high bits << 16) | entries, scratch slot or -1 for an uncut row}, longest first (same binning): the work list of
+// (high bits << 16) | entries, scratch slot or -1 for an uncut row}, subgraph by subgraph and longest first inside a
+// subgraph (same binning): the work list of
 // the one-warp-per-item kernel that serves operands of more than 64 columns.
 constexpr int64_t kMinPart = 64, kMaxPart = 1024;
 struct RowWork {
@@ -55,7 +56,7 @@ struct RowWork {
     int64_t slots = 0, part_entries = kMinPart;
 };
 int64_t part_entries_for(const std::vector<int64_t>& rowptr);
-void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out);
+void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& sub_off, RowWork& out);
 // Scratch slots bin_rows would use, from the row lengths alone.
 int64_t count_slots(const std::vector<int64_t>& rowptr);
 
@@ -71,6 +72,7 @@ struct SparseDev {
     const int4* items = nullptr;      // parts and uncut rows together, longest first
     float* scratch = nullptr;         // [slots x leading dimension of the output] partial rows
     int32_t nperm = 0, nparts = 0, nfin = 0, nitems = 0;
+    int64_t nrows = 0;                // rows (and columns) of the store
 };
 
 struct Layer {

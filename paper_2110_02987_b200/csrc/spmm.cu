@@ -269,8 +269,22 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
 // 16-byte shared load, turns each column into an address with one multiply-add, and keeps UU operand rows
 // (16 bytes per lane each) in flight before the multiply-adds.  The last entries of a batch go through the
 // next smaller power of two, so a batch costs at most one round trip more than its full groups.
-template <int NV, int UU>
-__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const char* const (&zl)[NV], uint32_t ldzb) {
+// Where a lane finds its 16 bytes of operand row c: operand start + c * (row stride in bytes) + the lane's column
+// offset.  With OFF32 the whole operand is smaller than 4 GiB and the offset is formed in 32 bits by one multiply-add.
+template <int NV, bool OFF32>
+struct ZLane {
+    const char* base;      // OFF32: start of the operand (the same for the whole warp)
+    const char* ptr[NV];   // otherwise: start of the operand plus the lane's column offset
+    uint32_t off[NV];
+    uint32_t ldzb;
+    __device__ __forceinline__ float4 load(uint32_t c, int j) const {
+        if constexpr (OFF32) return __ldg(reinterpret_cast<const float4*>(base + (c * ldzb + off[j])));
+        else return __ldg(reinterpret_cast<const float4*>(ptr[j] + (unsigned long long)c * ldzb));
+    }
+};
+
+template <int NV, int UU, bool OFF32>
+__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const ZLane<NV, OFF32>& zl) {
     uint32_t c[UU];
     float a[UU];
     if constexpr (UU == 1) {
@@ -288,8 +302,7 @@ __device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, c
 #pragma unroll
     for (int u = 0; u < UU; ++u)
 #pragma unroll
-        for (int j = 0; j < NV; ++j)
-            z[u][j] = __ldg(reinterpret_cast<const float4*>(zl[j] + (unsigned long long)c[u] * ldzb));
+        for (int j = 0; j < NV; ++j) z[u][j] = zl.load(c[u], j);
 #pragma unroll
     for (int u = 0; u < UU; ++u)
 #pragma unroll
@@ -301,21 +314,35 @@ __device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, c
         }
 }
 
-template <int NV, int V>
-__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const char* const (&zl)[NV], uint32_t ldzb) {
+template <int NV, int V, bool OFF32>
+__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const ZLane<NV, OFF32>& zl) {
     if constexpr (V >= 1) {
-        if (r > V / 2) gather_fma<NV, V>(acc, st, zl, ldzb);
-        else gather_tail<NV, V / 2>(acc, st, r, zl, ldzb);
+        if (r > V / 2) gather_fma<NV, V, OFF32>(acc, st, zl);
+        else gather_tail<NV, V / 2, OFF32>(acc, st, r, zl);
     }
 }
 
+// Operand rows in flight per lane and resident warps asked of the compiler: short items make the chain
+// item -> entries -> operand rows the cost, and more resident warps hide it better than more loads per warp.
+#ifndef GAD_SPMM_UU1
+#define GAD_SPMM_UU1 2
+#endif
+#ifndef GAD_SPMM_MINB1
+#define GAD_SPMM_MINB1 16
+#endif
+#ifndef GAD_SPMM_UU2
+#define GAD_SPMM_UU2 2
+#endif
+#ifndef GAD_SPMM_MINB2
+#define GAD_SPMM_MINB2 10
+#endif
 constexpr int kItemWarps = 4;
 template <int NV> struct ItemCfg {
-    static constexpr int UU = NV == 1 ? 8 : (NV == 2 ? 4 : (NV <= 4 ? 2 : 1));   // operand rows in flight per lane
-    static constexpr int MINB = NV <= 2 ? 8 : (NV <= 4 ? 6 : 4);                // resident CTAs asked of the compiler
+    static constexpr int UU = NV == 1 ? GAD_SPMM_UU1 : (NV == 2 ? GAD_SPMM_UU2 : (NV <= 4 ? 2 : 1));
+    static constexpr int MINB = NV == 1 ? GAD_SPMM_MINB1 : (NV == 2 ? GAD_SPMM_MINB2 : (NV <= 4 ? 6 : 4));   // CTAs of 4 warps per SM
 };
 
-template <int NV, bool EPI>
+template <int NV, bool EPI, bool OFF32>
 __global__ void __launch_bounds__(32 * kItemWarps, ItemCfg<NV>::MINB)
 spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z,
                   int ldz, float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
@@ -329,11 +356,15 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
     const int row = it.x, len = (int)((uint32_t)it.z & 0xFFFFu);
     const uint2* ent = ecv + (((long long)((uint32_t)it.z >> 16) << 32) | (long long)(uint32_t)it.y);
     const uint2 pad = make_uint2((uint32_t)row, 0u);
-    // per-lane operand pointers; lanes past the last column read the last one (their sums are never stored)
-    const char* zl[NV];
+    // lanes past the last column read the last one (their sums are never stored)
+    ZLane<NV, OFF32> zl;
+    zl.base = reinterpret_cast<const char*>(Z);
+    zl.ldzb = 4u * (uint32_t)ldz;
 #pragma unroll
-    for (int j = 0; j < NV; ++j) zl[j] = reinterpret_cast<const char*>(Z) + 16ll * min(lane + 32 * j, F4 - 1);
-    const uint32_t ldzb = 4u * (uint32_t)ldz;
+    for (int j = 0; j < NV; ++j) {
+        zl.off[j] = 16u * (uint32_t)min(lane + 32 * j, F4 - 1);
+        zl.ptr[j] = zl.base + zl.off[j];
+    }
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -347,8 +378,8 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
         stage[lane] = mine;
         __syncwarp();
         int t = 0;
-        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU>(acc, stage + t, zl, ldzb);
-        gather_tail<NV, UU / 2>(acc, stage + t, cnt - t, zl, ldzb);
+        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU, OFF32>(acc, stage + t, zl);
+        gather_tail<NV, UU / 2, OFF32>(acc, stage + t, cnt - t, zl);
     }
     if (it.w >= 0) {
 #pragma unroll
@@ -366,8 +397,12 @@ static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, floa
                                cudaStream_t s) {
     if constexpr (GROUP == 32) {
         if (A.nitems > 0) {
-            spmm_items_kernel<NV, EPI><<<(unsigned)((A.nitems + kItemWarps - 1) / kItemWarps), 32 * kItemWarps, 0, s>>>(
-                A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+            const unsigned grid = (unsigned)((A.nitems + kItemWarps - 1) / kItemWarps);
+            // every byte of the operand within 4 GiB of its start: 32-bit offsets
+            if ((unsigned long long)A.nrows * 4ull * (unsigned long long)ldz < (1ull << 32))
+                spmm_items_kernel<NV, EPI, true><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+            else
+                spmm_items_kernel<NV, EPI, false><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
             ++g_kernel_launches;
         }
         if (A.nfin > 0) {

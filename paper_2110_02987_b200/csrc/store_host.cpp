@@ -251,7 +251,7 @@ int64_t count_slots(const std::vector<int64_t>& rowptr) {
     return slots;
 }
 
-void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out) {
+void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& sub_off, RowWork& out) {
     const int64_t Np = (int64_t)rowptr.size() - 1;
     const int64_t part = part_entries_for(rowptr);
     out.perm.clear(); out.parts.clear(); out.fin.clear(); out.items.clear(); out.slots = 0; out.part_entries = part;
@@ -274,20 +274,25 @@ void bin_rows(const std::vector<int64_t>& rowptr, RowWork& out) {
             out.parts.push_back(make_int4((int)r, (int)(q * part), (int)std::min(part, len - q * part), (int)(out.slots + q)));
         out.slots += np;
     }
-    // the unified list: parts and uncut rows, longest first
+    // the unified list: subgraph by subgraph (the operand rows one subgraph gathers stay together in L2), parts
+    // and uncut rows of a subgraph longest first
     auto pack = [&](int64_t row, int64_t e0, int64_t len, int64_t slot) {
         return make_int4((int)row, (int)(uint32_t)(e0 & 0xFFFFFFFFll), (int)(uint32_t)(((e0 >> 32) << 16) | len), (int)slot);
     };
-    std::vector<int64_t> icount(64, 0), istart(64, 0);
-    for (const int4& pt : out.parts) icount[bin_of(pt.z)]++;
-    for (int32_t r : out.perm) icount[bin_of(rowptr[r + 1] - rowptr[r])]++;
-    acc = 0;
-    for (int b = 63; b >= 0; --b) { istart[b] = acc; acc += icount[b]; }
-    out.items.resize((size_t)acc);
-    for (const int4& pt : out.parts) out.items[(size_t)istart[bin_of(pt.z)]++] = pack(pt.x, rowptr[pt.x] + pt.y, pt.z, pt.w);
+    const int64_t K = (int64_t)sub_off.size() - 1;
+    std::vector<int32_t> sub_of((size_t)Np);
+    for (int64_t k = 0; k < K; ++k)
+        for (int64_t r = sub_off[k]; r < sub_off[k + 1]; ++r) sub_of[(size_t)r] = (int32_t)k;
+    auto key = [&](int64_t row, int64_t len) { return (size_t)(sub_of[(size_t)row] * 64 + (63 - bin_of(len))); };
+    std::vector<int64_t> istart((size_t)K * 64 + 1, 0);
+    for (const int4& pt : out.parts) istart[key(pt.x, pt.z) + 1]++;
+    for (int32_t r : out.perm) istart[key(r, rowptr[r + 1] - rowptr[r]) + 1]++;
+    for (size_t i = 1; i < istart.size(); ++i) istart[i] += istart[i - 1];
+    out.items.resize((size_t)istart.back());
+    for (const int4& pt : out.parts) out.items[(size_t)istart[key(pt.x, pt.z)]++] = pack(pt.x, rowptr[pt.x] + pt.y, pt.z, pt.w);
     for (int32_t r : out.perm) {
         const int64_t len = rowptr[r + 1] - rowptr[r];
-        out.items[(size_t)istart[bin_of(len)]++] = pack(r, rowptr[r], len, -1);
+        out.items[(size_t)istart[key(r, len)]++] = pack(r, rowptr[r], len, -1);
     }
 }
 
