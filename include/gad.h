@@ -79,7 +79,9 @@ typedef struct {
     int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form (GAD_ERR_UNSUPPORTED)       */
     float beta;           /* beta of the importance weight (Section 3.4.1); the paper uses 1                  */
     int32_t weighted;     /* 1: weighted global consensus (Section 3.4.2); 0: plain average (Definition 3)    */
-    int32_t flags;        /* bit 0: force the SIMT transform even where a tensor-core kernel exists           */
+    int32_t flags;        /* bit 0: force the SIMT transform even where a tensor-core kernel exists;
+                             bit 1: layer 0 aggregates first and keeps A~ H^(0) from one epoch to the next (it
+                             changes only with the features, i.e. with gad_set_inputs)                        */
 } gad_config;
 
 /* Bytes of device workspace gad_create needs for these inputs.  Host-only; touches no GPU. */

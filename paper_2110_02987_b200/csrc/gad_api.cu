@@ -34,6 +34,8 @@ struct Plan {
     std::vector<RowSpan> tiles, chunks, dw_chunks, core_spans;
     std::vector<int32_t> chunk_ptr, dw_chunk_ptr;   // [K+1]
     int64_t dw_partial = 0;           // floats per chunk
+    bool agg_first0 = false;          // layer 0 aggregates before it transforms
+    size_t o_P = 0;                   // A~ H^(0)  [Np x ld0], only with agg_first0
     size_t o_counters = 0;            // arrival counters: [loss | K column sums | K zeta]
     size_t bytes = 0;
     // offsets into the workspace
@@ -65,6 +67,9 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.ld.resize(p.L + 1);
     p.maxld = 0;
     for (int l = 0; l <= p.L; ++l) { p.ld[l] = (int32_t)round_up(p.dims[l], 4); p.maxld = std::max(p.maxld, p.ld[l]); }
+    // Layer 0 needs no gradient with respect to its input, so aggregating first costs one SpMM at the width F_0 where
+    // transforming first costs two at F_1; keeping A~ H^(0) across epochs (flag bit 1) removes that one as well.
+    p.agg_first0 = (cfg->flags & 2) != 0 || p.dims[0] <= 2 * p.dims[1];
     p.layers.resize(p.L);
     int64_t oi = 0, oe = 0;
     p.dw_partial = 0;
@@ -122,8 +127,8 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_core_spans = take(cur, sizeof(RowSpan) * p.core_spans.size());
     p.o_H.resize(p.L + 1);
     for (int l = 0; l <= p.L; ++l) p.o_H[l] = take(cur, 4 * Np * (size_t)p.ld[l]);
-    int32_t max_spmm_ld = 4;   // the SpMM runs at the widths F_1 .. F_L
-    for (int l = 1; l <= p.L; ++l) max_spmm_ld = std::max(max_spmm_ld, p.ld[l]);
+    int32_t max_spmm_ld = 4;   // the SpMM runs at the widths F_1 .. F_L, and at F_0 when layer 0 aggregates first
+    for (int l = p.agg_first0 ? 0 : 1; l <= p.L; ++l) max_spmm_ld = std::max(max_spmm_ld, p.ld[l]);
     p.o_spmm_scratch = take(cur, 4 * (size_t)slots * (size_t)max_spmm_ld);
     p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
     p.o_params = take(cur, 4 * (size_t)K * (size_t)p.pstride); p.o_grads = take(cur, 4 * (size_t)K * (size_t)p.pstride);
@@ -139,6 +144,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         p.o_wt_hi[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi); p.o_wt_lo[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi);
     }
     p.o_counters = take(cur, 4 * (size_t)(1 + 2 * K));
+    if (p.agg_first0) p.o_P = take(cur, 4 * Np * (size_t)p.ld[0]);
     p.bytes = cur;
     return GAD_OK;
 }
@@ -160,6 +166,8 @@ struct gad_ctx {
     bool profiling = false;
     std::vector<ProfEntry> prof;
     std::vector<float> host_block;  // staging for parameter pack / unpack
+    bool hoist = false;             // keep A~ H^(0) across epochs (config flag bit 1)
+    bool P_valid = false;           // A~ H^(0) matches the current features
     bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
     int num_sms = 1;
     struct alignas(64) TMap { unsigned char bytes[128]; };
@@ -237,16 +245,35 @@ int forward_pass(gad_ctx* ctx, bool train) {
         }
     for (int l = 0; l < p.L; ++l) {
         const Layer& y = p.layers[l];
+        Epilogue ep{params, p.pstride, y.b_int, ctx->at<int32_t>(p.o_sub_off), p.K, l < p.L - 1 ? 1 : 0,
+                    train ? ctx->cfg.dropout : 0.f, ctx->cfg.seed, ctx->epoch, l};
+        const bool agg_first = l == 0 && p.agg_first0;
+        if (agg_first) {
+            // A~ (X W) = (A~ X) W: aggregate at the input width, finish the layer in the transform's epilogue
+            if (!(ctx->hoist && ctx->P_valid)) {
+                GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
+                        [&] { return launch_spmm(ctx->A, ctx->H(0), y.ldi, ctx->at<float>(p.o_P), y.ldi, y.fi, nullptr, ctx->stream); });
+                ctx->P_valid = true;
+            }
+            const ActEpi act = make_act(ep, 0);
+            GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+                if (ctx->use_tc)
+                    return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 2, passes, y.fi, y.fo,
+                                               ctx->H(l + 1), y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, &act,
+                                               ctx->at<int32_t>(p.o_flags) + 1, ctx->num_sms, ctx->stream);
+                return launch_gemm_rows_simt(2, ctx->at<float>(p.o_P), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, ctx->H(l + 1), y.ldo,
+                                             ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, &act, ctx->stream);
+            });
+            continue;
+        }
         GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
             if (ctx->use_tc)
                 return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 0, passes, y.fi, y.fo, Z,
-                                           y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f,
+                                           y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr,
                                            ctx->at<int32_t>(p.o_flags) + 1, ctx->num_sms, ctx->stream);
             return launch_gemm_rows_simt(0, ctx->H(l), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, Z, y.ldo,
-                                         ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, ctx->stream);
+                                         ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr, ctx->stream);
         });
-        Epilogue ep{params, p.pstride, y.b_int, ctx->at<int32_t>(p.o_sub_off), p.K, l < p.L - 1 ? 1 : 0,
-                    train ? ctx->cfg.dropout : 0.f, ctx->cfg.seed, ctx->epoch, l};
         GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                 [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, ctx->stream); });
     }
@@ -284,15 +311,17 @@ int backward_pass(gad_ctx* ctx) {
             return launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr,
                                         ctx->at<unsigned>(p.o_counters) + 1, grads, p.pstride, y.b_int, ctx->stream);
         });
-        GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
-                [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
+        const bool agg_first = l == 0 && p.agg_first0;   // then dW = (A~ X)^T dPre and nothing flows further back
+        if (!agg_first)
+            GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
+                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
         GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
             cudaError_t e =
                 ctx->use_tc ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
                                                 ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, dw_chunks, ndw,
                                                 ctx->at<float>(p.o_dw_partial), ctx->at<int32_t>(p.o_flags) + 1, ctx->stream)
-                            : launch_gemm_tn_simt(ctx->H(l), y.ldi, y.fi, G2, y.ldo, y.fo, dw_chunks, ndw,
-                                                  ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
+                            : launch_gemm_tn_simt(agg_first ? ctx->at<float>(p.o_P) : ctx->H(l), y.ldi, y.fi, agg_first ? G1 : G2, y.ldo,
+                                                  y.fo, dw_chunks, ndw, ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
             if (e != cudaSuccess) return e;
             return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, dw_chunk_ptr, p.K, grads, p.pstride,
                                         y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
@@ -302,10 +331,10 @@ int backward_pass(gad_ctx* ctx) {
                 if (ctx->use_tc)
                     return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 3], &ctx->maps[kMapsPerLayer * l + 4], &ctx->maps[kMapsPerLayer * l + 5], 1,
                                                ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fo, y.fi, G1, y.ldi, ctx->at<RowSpan>(p.o_tiles),
-                                               (int)p.tiles.size(), ctx->H(l), y.ldi, scale, ctx->at<int32_t>(p.o_flags) + 1,
+                                               (int)p.tiles.size(), ctx->H(l), y.ldi, scale, nullptr, ctx->at<int32_t>(p.o_flags) + 1,
                                                ctx->num_sms, ctx->stream);
                 return launch_gemm_rows_simt(1, G2, y.ldo, y.fo, params, p.pstride, y.w_int, y.ldw, y.fi, G1, y.ldi,
-                                             ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), ctx->H(l), y.ldi, scale,
+                                             ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), ctx->H(l), y.ldi, scale, nullptr,
                                              ctx->stream);
             });
     }
@@ -415,6 +444,7 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->stream = (cudaStream_t)stream;
     ctx->ws = (char*)workspace;
     ctx->cfg = *cfg;
+    ctx->hoist = (cfg->flags & 2) != 0;
     HostStore st;
     int rc = build_store(g, part, true, st, ctx->err);
     if (rc != GAD_OK) return fail(ctx, rc, ctx->err);
@@ -511,7 +541,9 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
             GAD_CK(cudaMemsetAsync(ctx->ws + p.o_wt_lo[l], 0, 4 * (size_t)p.K * y.fo * y.ldi, ctx->stream));
             gad_ctx::TMap* m = &ctx->maps[(size_t)kMapsPerLayer * l];
             // forward: A = H^(l) [Np x fi], B = W^T copies [K][fo][fi]
-            ok = ok && tc_make_map(&m[0], ctx->H(l), y.fi, p.Np, 0, 4ull * y.ldi, 0, 128);
+            const bool agg_first = l == 0 && p.agg_first0;   // then the transform and the weight gradient read A~ H^(0), and dW reads dPre (G1)
+            float* Hin = agg_first ? ctx->at<float>(p.o_P) : ctx->H(l);
+            ok = ok && tc_make_map(&m[0], Hin, y.fi, p.Np, 0, 4ull * y.ldi, 0, 128);
             ok = ok && tc_make_map(&m[1], ctx->at<float>(p.o_wt_hi[l]), y.fi, y.fo, p.K, 4ull * y.ldi, 4ull * y.fo * y.ldi, tc_bn_for(y.fo));
             ok = ok && tc_make_map(&m[2], ctx->at<float>(p.o_wt_lo[l]), y.fi, y.fo, p.K, 4ull * y.ldi, 4ull * y.fo * y.ldi, tc_bn_for(y.fo));
             // input gradient: A = dZ [Np x fo] (in G2), B = W copies [K][fi][fo]
@@ -519,8 +551,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
             ok = ok && tc_make_map(&m[4], ctx->at<float>(p.o_w_hi[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
             ok = ok && tc_make_map(&m[5], ctx->at<float>(p.o_w_lo[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
             // weight gradient: 32-row tiles of H^(l) and of dZ (in G2)
-            ok = ok && tc_make_map(&m[6], ctx->H(l), y.fi, p.Np, 0, 4ull * y.ldi, 0, 32, true);
-            ok = ok && tc_make_map(&m[7], ctx->at<float>(p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 32, true);
+            ok = ok && tc_make_map(&m[6], Hin, y.fi, p.Np, 0, 4ull * y.ldi, 0, 32, true);
+            ok = ok && tc_make_map(&m[7], ctx->at<float>(agg_first ? p.o_G1 : p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 32, true);
         }
         if (!ok) return fail(ctx, GAD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     }
@@ -690,6 +722,7 @@ int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels) {
             return launch_gather_rows(ctx->at<float>(p.o_stage), p.dims[0], ctx->at<int32_t>(p.o_gid), p.Np, ctx->H(0), p.ld[0],
                                       ctx->stream);
         });
+        ctx->P_valid = false;   // A~ H^(0) is aggregated again by the next forward pass
     }
     if (labels) {
         GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage_lab, labels, 4 * (size_t)p.n, cudaMemcpyHostToDevice, ctx->stream));

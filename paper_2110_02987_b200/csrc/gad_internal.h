@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cmath>
 #include <string>
 #include <vector>
 
@@ -99,6 +100,31 @@ struct Epilogue {            // of the forward SpMM: bias, ReLU, dropout
     int32_t layer;
 };
 
+// What a finishing kernel gets: where the biases are and how ReLU / dropout apply on this layer and epoch.
+struct ActEpi {
+    const float* params;   // padded parameter blocks
+    long long pstride;     // floats between replicas
+    long long b_int;       // bias offset inside a block
+    int relu;              // 0 on the last layer
+    int drop;              // dropout is applied (rate > 0 on a layer with ReLU)
+    uint32_t thr;          // keep an element when the top 24 bits of its hash reach this
+    float scale;           // 1 / (1 - rate)
+    unsigned long long seed;
+    long long epoch;
+    int layer;
+    int col0;              // column of the operand's first column (column slabs)
+};
+inline ActEpi make_act(const Epilogue& e, int col0) {
+    ActEpi t{};
+    t.params = e.params; t.pstride = e.pstride; t.b_int = e.b_int + col0;
+    t.relu = e.relu; t.layer = e.layer;
+    t.drop = e.dropout > 0.f && e.relu;
+    t.thr = t.drop ? (uint32_t)std::floor((double)e.dropout * 16777216.0) : 0u;
+    t.scale = t.drop ? 1.f / (1.f - e.dropout) : 1.f;
+    t.seed = e.seed; t.epoch = e.epoch; t.col0 = col0;
+    return t;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Kernel launchers (each enqueues on `s` and returns the cudaGetLastError of its launches)
 // ---------------------------------------------------------------------------------------------
@@ -106,10 +132,10 @@ cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out,
                         const Epilogue* epi, cudaStream_t s);
 
 // mode 0: C = A * W_k (W row-major [Kd x N], ld ldw); mode 1: C = (A * W_k^T) masked by Hmask > 0, scaled
-// (W row-major [N x Kd]).  Tiles never cross a subgraph.
+// (W row-major [N x Kd]); mode 2: C = sigma(A * W_k + b_k) with dropout as `act` says.  Tiles never cross a subgraph.
 cudaError_t launch_gemm_rows_simt(int mode, const float* A, int lda, int Kd, const float* params, int64_t pstride,
                                   int64_t w_int, int ldw, int N, float* C, int ldc, const RowSpan* tiles,
-                                  int ntiles, const float* Hmask, int ldh, float scale, cudaStream_t s);
+                                  int ntiles, const float* Hmask, int ldh, float scale, const ActEpi* act, cudaStream_t s);
 
 // Tensor-core (tcgen05) version of launch_gemm_rows_simt.  The operands come through TMA descriptors made by
 // tc_make_map (A: [rows x Kd]; B, B_lo: [K][N][Kd] copies written by launch_split_weights); passes = 3 gives fp32
@@ -121,7 +147,7 @@ cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w
                                  float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, cudaStream_t s);
 cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* mapBlo, int mode, int passes, int Kd, int n_cols,
                                 float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
-                                int32_t* err, int num_sms, cudaStream_t s);
+                                const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s);
 
 // Tensor-core version of launch_gemm_tn_simt; mapH / mapZ are 32-row-box descriptors of H^(l) and dZ.
 cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,

@@ -5,19 +5,21 @@
 // "Grouped": every row tile / row chunk belongs to exactly one subgraph k and uses that replica's W_k.
 // All matrices keep zero-filled pad columns up to their leading dimension, so 16-byte loads never need a
 // column guard beyond "below the leading dimension".
+#include "epilogue.cuh"
 #include "gad_internal.h"
 
 namespace gad {
 
 // ---------------------------------------------------------------------------------------------
 // C[rows x N] = A[rows x Kd] * B, rows tiled by RowSpan.  MODE 0: B[kd][n] = W[kd*ldw + n];
-// MODE 1: B[kd][n] = W[n*ldw + kd] and the result is masked / scaled.
+// MODE 1: B[kd][n] = W[n*ldw + kd] and the result is masked / scaled.  MODE 2: as MODE 0, followed by bias, ReLU and
+// dropout (a layer that aggregates first finishes in its transform).
 // ---------------------------------------------------------------------------------------------
 template <int BM, int BN, int BK, int TM, int TN, int MODE>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN))
 gemm_rows_kernel(const float* __restrict__ A, int lda, int Kd, const float* __restrict__ params, long long pstride,
                  long long w_int, int ldw, int N, float* __restrict__ C, int ldc, const RowSpan* __restrict__ tiles,
-                 const float* __restrict__ Hmask, int ldh, float scale) {
+                 const float* __restrict__ Hmask, int ldh, float scale, ActEpi act) {
     constexpr int NT = (BM / TM) * (BN / TN);
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
@@ -41,7 +43,7 @@ gemm_rows_kernel(const float* __restrict__ A, int lda, int Kd, const float* __re
             if (r < t.nrows && k0 + kq < lda) v = *reinterpret_cast<const float4*>(A + (long long)(t.row0 + r) * lda + k0 + kq);
             As[kq + 0][r] = v.x; As[kq + 1][r] = v.y; As[kq + 2][r] = v.z; As[kq + 3][r] = v.w;
         }
-        if (MODE == 0) {
+        if (MODE != 1) {
             for (int i = tid; i < BK * (BN / 4); i += NT) {
                 int kk = i / (BN / 4), nq = (i % (BN / 4)) * 4;
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -88,6 +90,7 @@ gemm_rows_kernel(const float* __restrict__ A, int lda, int Kd, const float* __re
                 v.z = h.z > 0.f ? v.z * scale : 0.f;
                 v.w = h.w > 0.f ? v.w * scale : 0.f;
             }
+            if (MODE == 2) v = apply_act(v, act, t.k, row, n);
             *reinterpret_cast<float4*>(C + row * ldc + n) = v;
         }
     }
@@ -96,15 +99,19 @@ gemm_rows_kernel(const float* __restrict__ A, int lda, int Kd, const float* __re
 template <int BM, int BN, int BK, int TM, int TN>
 static cudaError_t launch_rows_cfg(int mode, const float* A, int lda, int Kd, const float* params, int64_t pstride,
                                    int64_t w_int, int ldw, int N, float* C, int ldc, const RowSpan* tiles, int ntiles,
-                                   const float* Hmask, int ldh, float scale, cudaStream_t s) {
+                                   const float* Hmask, int ldh, float scale, const ActEpi* act, cudaStream_t s) {
     dim3 grid((unsigned)ntiles, (unsigned)((ldc + BN - 1) / BN));
     constexpr int NT = (BM / TM) * (BN / TN);
+    const ActEpi none{};
     if (mode == 0)
         gemm_rows_kernel<BM, BN, BK, TM, TN, 0><<<grid, NT, 0, s>>>(A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles,
-                                                                    Hmask, ldh, scale);
-    else
+                                                                    Hmask, ldh, scale, none);
+    else if (mode == 1)
         gemm_rows_kernel<BM, BN, BK, TM, TN, 1><<<grid, NT, 0, s>>>(A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles,
-                                                                    Hmask, ldh, scale);
+                                                                    Hmask, ldh, scale, none);
+    else
+        gemm_rows_kernel<BM, BN, BK, TM, TN, 2><<<grid, NT, 0, s>>>(A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles,
+                                                                    Hmask, ldh, scale, *act);
     ++g_kernel_launches;
     return cudaGetLastError();
 }
@@ -112,13 +119,14 @@ static cudaError_t launch_rows_cfg(int mode, const float* A, int lda, int Kd, co
 // Row tiles hold at most 128 rows (the tile table is built with that height).
 cudaError_t launch_gemm_rows_simt(int mode, const float* A, int lda, int Kd, const float* params, int64_t pstride,
                                   int64_t w_int, int ldw, int N, float* C, int ldc, const RowSpan* tiles, int ntiles,
-                                  const float* Hmask, int ldh, float scale, cudaStream_t s) {
+                                  const float* Hmask, int ldh, float scale, const ActEpi* act, cudaStream_t s) {
     if (ntiles <= 0) return cudaSuccess;
+    if (mode == 2 && !act) return cudaErrorInvalidValue;
     if (ldc > 64)
-        return launch_rows_cfg<128, 128, 16, 8, 8>(mode, A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles, ntiles, Hmask, ldh, scale, s);
+        return launch_rows_cfg<128, 128, 16, 8, 8>(mode, A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles, ntiles, Hmask, ldh, scale, act, s);
     if (ldc > 32)
-        return launch_rows_cfg<128, 64, 16, 8, 4>(mode, A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles, ntiles, Hmask, ldh, scale, s);
-    return launch_rows_cfg<128, 32, 16, 4, 4>(mode, A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles, ntiles, Hmask, ldh, scale, s);
+        return launch_rows_cfg<128, 64, 16, 8, 4>(mode, A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles, ntiles, Hmask, ldh, scale, act, s);
+    return launch_rows_cfg<128, 32, 16, 4, 4>(mode, A, lda, Kd, params, pstride, w_int, ldw, N, C, ldc, tiles, ntiles, Hmask, ldh, scale, act, s);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -1,6 +1,8 @@
 // Grouped dense transforms on the 5th-generation tensor cores (tcgen05, accumulators in tensor memory):
 //   mode 0   Z_l  = H^(l) W_k^(l)                        (the H.W of the forward equation, Section 3.3)
 //   mode 1   dPre = (dZ_l W_k^(l)^T) masked by H^(l) > 0  (chain rule through the forward equation)
+//   mode 2   H^(l+1) = sigma((A~ H^(l)) W_k^(l) + b_k^(l)) with dropout: mode 0 finished in the epilogue, for a layer
+//            that aggregates before it transforms
 // Both are C[rows x N] = A[rows x Kd] * B_k^T with A row-major (Kd contiguous) and B_k stored as N rows of Kd
 // contiguous values, i.e. both operands K-major.  Row tiles never cross a subgraph, so a tile uses one replica's B.
 //
@@ -16,6 +18,7 @@
 // raises an error word, stops, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include "epilogue.cuh"
 #include "gad_internal.h"
 
 namespace gad {
@@ -133,6 +136,7 @@ struct TcArgs {
     float scale;
     int mode, passes;
     int32_t* err;
+    ActEpi act;   // mode 2
 };
 
 __global__ void __launch_bounds__(320, 1)
@@ -283,6 +287,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                     : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
+                float4 bias4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (a.mode == 2 && n < a.ldc) bias4 = load_bias(a.act, sp.k, n);
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN_MAX + c0), v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -300,6 +306,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         o[i].z = hm[i].z > 0.f ? o[i].z * a.scale : 0.f;
                         o[i].w = hm[i].w > 0.f ? o[i].w * a.scale : 0.f;
                     }
+                    if (a.mode == 2) o[i] = apply_act(o[i], bias4, a.act, (long long)sp.row0 + q * 32 + 4 * i + sub_r, n);
                 }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -563,8 +570,9 @@ cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w
 
 cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* mapBlo, int mode, int passes, int Kd, int n_cols,
                                 float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
-                                int32_t* err, int num_sms, cudaStream_t s) {
+                                const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s) {
     if (ntiles <= 0) return cudaSuccess;
+    if (mode == 2 && !act) return cudaErrorInvalidValue;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_ROWS);
@@ -574,6 +582,7 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
     TcArgs a;
     a.tiles = tiles; a.ntiles_rows = ntiles; a.BN = tc_bn_for(n_cols); a.ntn = (ldc + a.BN - 1) / a.BN; a.Kd = Kd;
     a.C = C; a.ldc = ldc; a.Hmask = Hmask; a.ldh = ldh; a.scale = scale; a.mode = mode; a.passes = passes; a.err = err;
+    a.act = act ? *act : ActEpi{};
     const long long total = (long long)ntiles * a.ntn;
     const unsigned grid = (unsigned)(total < num_sms ? total : num_sms);
     gemm_tc_kernel<<<grid, 320, SMEM_BYTES_ROWS, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),

@@ -8,28 +8,10 @@
 // (column, value) pairs and handed round with shuffles.  Rows come from a list binned by length (heaviest
 // first); long rows are cut into parts with a warp per part and a fixed-order sum of the parts through a scratch
 // buffer, so results never depend on scheduling.
+#include "epilogue.cuh"
 #include "gad_internal.h"
 
 namespace gad {
-
-__device__ __forceinline__ uint64_t mix64(uint64_t z) {
-    z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ULL;
-    z = (z ^ (z >> 27)) * 0x94d049bb133111ebULL;
-    return z ^ (z >> 31);
-}
-
-// Row part of the dropout hash: (seed, epoch, layer, row) -> 64 bits; the column is mixed in per element.
-__device__ __forceinline__ uint64_t dropout_row_key(uint64_t seed, int64_t epoch, int layer, int64_t row) {
-    const uint64_t G = 0x9e3779b97f4a7c15ULL;
-    uint64_t h = mix64(seed + G * (uint64_t)(1 + epoch));
-    h = mix64(h + G * (uint64_t)(1 + layer));
-    return mix64(h + G * (uint64_t)(1 + row));
-}
-__device__ __forceinline__ bool dropout_keep(uint64_t row_key, int col, uint32_t thr24) {
-    const uint64_t G = 0x9e3779b97f4a7c15ULL;
-    uint64_t h = mix64(row_key + G * (uint64_t)(1 + col));
-    return (uint32_t)(h >> 40) >= thr24;
-}
 
 __device__ __forceinline__ int find_sub(const int32_t* __restrict__ sub_off, int K, int row) {
     int lo = 0, hi = K;  // largest k with sub_off[k] <= row (empty subgraphs are skipped by the <=)
@@ -41,15 +23,9 @@ __device__ __forceinline__ int find_sub(const int32_t* __restrict__ sub_off, int
 }
 
 struct EpiDev {
-    const float* params;
-    long long pstride, b_int;
+    ActEpi act;
     const int32_t* sub_off;
-    int K, relu, layer, col0;
-    int drop;             // dropout is applied (rate > 0 on a layer with ReLU)
-    uint32_t thr;         // keep an element when the top 24 bits of its hash reach this
-    float scale;          // 1 / (1 - rate)
-    unsigned long long seed;
-    long long epoch;
+    int K;
 };
 
 template <int NV, bool EPI>
@@ -57,25 +33,10 @@ __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, i
                                            int ldo, const EpiDev& ep) {
     if (EPI) {
         const int k = find_sub(ep.sub_off, ep.K, row);
-        const float4* bias = reinterpret_cast<const float4*>(ep.params + (long long)k * ep.pstride + ep.b_int);
-        const bool drop = ep.drop != 0;
-        const float scale = ep.scale;
-        const uint32_t thr = ep.thr;
-        const uint64_t key = drop ? dropout_row_key(ep.seed, ep.epoch, ep.layer, row) : 0ull;
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
-            int v = gl + group * j;
-            if (v >= F4) continue;
-            float4 b = __ldg(bias + v);
-            float x[4] = {acc[j].x + b.x, acc[j].y + b.y, acc[j].z + b.z, acc[j].w + b.w};
-            if (ep.relu) {
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    x[t] = x[t] > 0.f ? x[t] : (x[t] <= 0.f ? 0.f : x[t]);   // ReLU that lets NaN through
-                    if (drop) x[t] = dropout_keep(key, ep.col0 + 4 * v + t, thr) ? x[t] * scale : 0.f;
-                }
-            }
-            acc[j] = make_float4(x[0], x[1], x[2], x[3]);
+            const int v = gl + group * j;
+            if (v < F4) acc[j] = apply_act(acc[j], ep.act, k, row, 4 * v);
         }
     }
 #pragma unroll
@@ -454,12 +415,8 @@ cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out,
         const int F4 = min(256, F4_all - c0);
         EpiDev ep{};
         if (epi) {
-            ep.params = epi->params; ep.pstride = epi->pstride; ep.b_int = epi->b_int + 4ll * c0;
-            ep.sub_off = epi->sub_off; ep.K = epi->K; ep.relu = epi->relu; ep.layer = epi->layer;
-            ep.drop = epi->dropout > 0.f && epi->relu;
-            ep.thr = ep.drop ? (uint32_t)floor((double)epi->dropout * 16777216.0) : 0u;
-            ep.scale = ep.drop ? 1.f / (1.f - epi->dropout) : 1.f;
-            ep.seed = epi->seed; ep.epoch = epi->epoch; ep.col0 = 4 * c0;
+            ep.act = make_act(*epi, 4 * c0);
+            ep.sub_off = epi->sub_off; ep.K = epi->K;
         }
         cudaError_t e = epi ? dispatch<true>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s)
                             : dispatch<false>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s);

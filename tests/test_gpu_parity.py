@@ -280,6 +280,27 @@ def test_set_inputs_replaces_features_and_labels(tiny):
         assert rel_err(g.get_grads(1), ref.get_grads(1)) <= TOL
 
 
+def test_kept_input_aggregation_follows_new_features(tiny):
+    """flags bit 1 keeps A~ H^(0) across epochs; new features must replace it."""
+    w = tiny
+    theta = glorot_params(w.dims, np.random.default_rng(8))
+    rng = np.random.default_rng(10)
+    X2 = rng.standard_normal(w.X.shape).astype(np.float32)
+    cp, cn, hp, hn = w.flat_partition()
+    st = orc().Store(w.n, w.rowptr, w.col, cp, cn, hp, hn)
+    ref = orc().Model(st, w.X, w.labels, w.split, w.dims, theta, lr=w.lr)
+    with pkg().from_workload(w, theta, flags=2) as g:
+        for _ in range(2):
+            assert np.max(np.abs(g.train_epoch() - ref.train_epoch())) <= 1e-5
+        ref2 = orc().Model(st, X2, w.labels, w.split, w.dims, ref.get_params(0), lr=w.lr)
+        for k in range(1, g.K):
+            ref2.set_params(k, ref.get_params(k))
+        g.set_inputs(X2, None)
+        for _ in range(2):
+            assert np.max(np.abs(g.train_epoch() - ref2.train_epoch())) <= 1e-5
+        assert rel_err(g.get_params(0), ref2.get_params(0)) <= TOL
+
+
 def test_non_finite_loss_is_reported_not_trapped(tiny):
     w = tiny
     theta = glorot_params(w.dims, np.random.default_rng(7))
@@ -316,11 +337,13 @@ def test_c2_two_epochs_full_size():
         assert np.max(np.abs(wg - wr)) <= 1e-6
 
 
-@pytest.mark.parametrize("gemm_mode,flags,tol", [(0, 0, TOL), (0, 1, TOL), (1, 0, 5e-2)])
+@pytest.mark.parametrize("gemm_mode,flags,tol", [(0, 0, TOL), (0, 1, TOL), (1, 0, 5e-2), (0, 2, TOL), (0, 3, TOL)])
 @pytest.mark.parametrize("dims", [(96, 160, 40, 8), (602, 256, 41), (20, 300, 130, 3)])
 def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
     """The grouped H.W transform on tensor cores (split-TF32: fp32 bar; single-pass TF32 operands: 5e-2 bar) and
-    on the FP32 ALUs (flags bit 0), over row tiles with ragged ends and feature widths that are not tile multiples."""
+    on the FP32 ALUs (flags bit 0), over row tiles with ragged ends and feature widths that are not tile multiples.
+    Layer 0 transforms first when F_0 > 2 F_1 (the 602-wide case) and aggregates first otherwise; flags bit 1 makes it
+    aggregate first everywhere and keeps the aggregated features between epochs."""
     case = small_random_case(21, n=900, K=3, p=0.01)
     g, ref, st = make_pair(case, dims, 21, lr=0.05, gemm_mode=gemm_mode, flags=flags)
     with g:
