@@ -45,12 +45,13 @@ int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_
 // group, per row), binned by floor(log2(entries)), heaviest bin first, ascending row id inside a bin.  Longer rows
 // are cut into parts of `part_entries` entries, one warp per part: parts = {row, first entry relative to the row,
 // entries, scratch slot}; fin = {row, first scratch slot, slots, 0} for every row that was cut.  The part length
-// starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most one scratch slot per two store rows.
+// starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most one scratch slot per two store rows;
+// a row that would still need more than kMaxSlotsPerRow parts gets longer parts of its own.
 // items = every part and every uncut row as {row, low 32 bits of the first entry's position in the store,
 // (high bits << 16) | entries, scratch slot or -1 for an uncut row}, subgraph by subgraph and longest first inside a
 // subgraph (same binning): the work list of
 // the one-warp-per-item kernel that serves operands of more than 64 columns.
-constexpr int64_t kMinPart = 64, kMaxPart = 1024;
+constexpr int64_t kMinPart = 64, kMaxPart = 1024, kMaxSlotsPerRow = 32;
 struct RowWork {
     std::vector<int32_t> perm;
     std::vector<int4> parts, fin, items;

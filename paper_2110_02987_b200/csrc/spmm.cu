@@ -2,12 +2,11 @@
 // aggregation half of the layer H^(l+1) = sigma(A~ (H^(l) W^(l)) + b) (Section 3.3, forward equation); run on
 // the transposed store it is the backward aggregation dZ = A~^T dPre.
 //
-// Work split: a warp owns one row and walks its entries; GROUP lanes (4..32) span the feature columns with NV
-// float4 accumulators each (16-byte loads of the dense operand), and when GROUP < 32 the warp's 32/GROUP
-// sub-groups take different entries of the row at the same time.  Entries are fetched 32 at a time as packed
-// (column, value) pairs and handed round with shuffles.  Rows come from a list binned by length (heaviest
-// first); long rows are cut into parts with a warp per part and a fixed-order sum of the parts through a scratch
-// buffer, so results never depend on scheduling.
+// Work list: every row, or every part of a row too long for one item, is an item {row, position of its first
+// entry, entries, scratch slot}; items are grouped by subgraph and sorted longest first inside one.  Operands wider
+// than 64 columns take a warp per item, narrower ones a group of 4, 8 or 16 lanes per item; every lane owns 16
+// bytes of each operand row it gathers.  The parts of a cut row go to scratch slots and a second kernel adds them
+// in part order, so results never depend on scheduling.
 #include "epilogue.cuh"
 #include "gad_internal.h"
 
@@ -46,146 +45,88 @@ __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, i
     }
 }
 
-// Entries [e0, e1) of one row accumulated by a whole warp.  The warp fetches 32 packed entries at a time (the
-// next batch is requested before the current one is consumed); with GROUP < 32 the 32/GROUP sub-groups take
-// different entries of the batch, each lane loading its own 16 bytes of the operand row, and the sub-group
-// sums are combined afterwards with a fixed butterfly.
-template <int NV, int GROUP>
-__device__ __forceinline__ void walk_entries(float4 (&acc)[NV], const uint2* __restrict__ ecv, long long e0, long long e1,
-                                             const float* __restrict__ Z, int ldz, int lane, int F4) {
-    constexpr int SG = 32 / GROUP;
-    const int gl = lane & (GROUP - 1), sg = lane / GROUP;
-    uint2 next = make_uint2(0u, 0u);
-    if (e0 + lane < e1) next = __ldg(ecv + e0 + lane);
-    for (long long e = e0; e < e1; e += 32) {
-        const uint2 mine = next;
-        if (e + 32 + lane < e1) next = __ldg(ecv + e + 32 + lane);
-        const int cnt = (int)min(32ll, e1 - e);
-        // U entries per sub-group are in flight together; a slot past the end of the batch re-reads the batch's
-        // first operand row with weight 0, so the loads stay unconditional and can all be issued at once
-        constexpr int U = NV <= 2 ? 4 : (NV <= 4 ? 2 : 1);
-        const int c_first = __shfl_sync(0xffffffffu, (int)mine.x, 0);
-        for (int t = 0; t < cnt; t += U * SG) {
-            int c[U];
-            float a[U];
+// Decoded item of the unified list.
+struct Item {
+    int row, len, slot;
+    const uint2* ent;
+};
+__device__ __forceinline__ Item load_item(const int4* __restrict__ items, int idx, const uint2* __restrict__ ecv) {
+    const int4 it = __ldg(items + idx);   // {row, entry position low, (position high << 16) | entries, scratch slot or -1}
+    Item r;
+    r.row = it.x; r.len = (int)((uint32_t)it.z & 0xFFFFu); r.slot = it.w;
+    r.ent = ecv + (((long long)((uint32_t)it.z >> 16) << 32) | (long long)(uint32_t)it.y);
+    return r;
+}
+
+// ---- operands of at most 64 columns: GROUP lanes per item, 32 / GROUP items per warp ----
+//
+// A group fetches a batch of entries at a time (the next batch is requested before this one is used), hands them
+// round with shuffles and has all their operand rows in flight before the multiply-adds; a slot past the end of the
+// item re-reads the item's own operand row with weight 0.  A last batch at most half full takes a half batch.
+#ifndef GAD_SPMM_NBATCH
+#define GAD_SPMM_NBATCH 8
+#endif
+#ifndef GAD_SPMM_NMINB
+#define GAD_SPMM_NMINB 3
+#endif
+constexpr int kNarrowBatch = GAD_SPMM_NBATCH;
+template <int GROUP> struct NarrowCfg { static constexpr int EPL = kNarrowBatch / GROUP > 0 ? kNarrowBatch / GROUP : 1; };
+
+template <int GROUP, int NB>
+__device__ __forceinline__ void narrow_batch(float4& acc, const uint2 (&mine)[NarrowCfg<GROUP>::EPL], unsigned gmask,
+                                             const char* zl, uint32_t ldzb) {
+    float4 z[NB];
+    float a[NB];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int src = t + u * SG + sg;   // entry of the batch this sub-group takes
-                c[u] = __shfl_sync(0xffffffffu, (int)mine.x, src & 31);
-                a[u] = __uint_as_float(__shfl_sync(0xffffffffu, mine.y, src & 31));
-                if (src >= cnt) { a[u] = 0.f; c[u] = c_first; }
-            }
-            float4 z[U][NV];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const float4* zr = reinterpret_cast<const float4*>(Z + (long long)c[u] * ldz);
-#pragma unroll
-                for (int j = 0; j < NV; ++j) {
-                    const int v = gl + GROUP * j;
-                    z[u][j] = v < F4 ? __ldg(zr + v) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int j = 0; j < NV; ++j) {
-                    acc[j].x = fmaf(a[u], z[u][j].x, acc[j].x);
-                    acc[j].y = fmaf(a[u], z[u][j].y, acc[j].y);
-                    acc[j].z = fmaf(a[u], z[u][j].z, acc[j].z);
-                    acc[j].w = fmaf(a[u], z[u][j].w, acc[j].w);
-                }
-        }
+    for (int t = 0; t < NB; ++t) {
+        const uint32_t c = __shfl_sync(gmask, mine[t / GROUP].x, t % GROUP, GROUP);
+        a[t] = __uint_as_float(__shfl_sync(gmask, mine[t / GROUP].y, t % GROUP, GROUP));
+        z[t] = __ldg(reinterpret_cast<const float4*>(zl + (unsigned long long)c * ldzb));
     }
-    if (SG > 1) {
 #pragma unroll
-        for (int j = 0; j < NV; ++j)
-#pragma unroll
-            for (int o = GROUP; o < 32; o <<= 1) {
-                acc[j].x += __shfl_xor_sync(0xffffffffu, acc[j].x, o);
-                acc[j].y += __shfl_xor_sync(0xffffffffu, acc[j].y, o);
-                acc[j].z += __shfl_xor_sync(0xffffffffu, acc[j].z, o);
-                acc[j].w += __shfl_xor_sync(0xffffffffu, acc[j].w, o);
-            }
+    for (int t = 0; t < NB; ++t) {
+        acc.x = fmaf(a[t], z[t].x, acc.x);
+        acc.y = fmaf(a[t], z[t].y, acc.y);
+        acc.z = fmaf(a[t], z[t].z, acc.z);
+        acc.w = fmaf(a[t], z[t].w, acc.w);
     }
 }
 
-// Narrow operands (at most 16 float4 per row): GROUP lanes per short row, 32/GROUP rows per warp.  A group fetches
-// GROUP entries at a time and has all of their operand rows in flight together; a slot past the end of the row
-// re-reads the row's own operand row (its self-loop is in the sum anyway) with weight 0.
 template <int GROUP, bool EPI>
-__global__ void __launch_bounds__(256) spmm_rows_narrow_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
-                                                               const int32_t* __restrict__ rows, int nrows,
-                                                               const float* __restrict__ Z, int ldz, float* __restrict__ out,
-                                                               int ldo, int F4, EpiDev ep) {
+__global__ void __launch_bounds__(256, GAD_SPMM_NMINB)
+spmm_items_narrow_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z, int ldz,
+                         float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
+    constexpr int NB = kNarrowBatch, EPL = NarrowCfg<GROUP>::EPL;   // entries per batch, entries a lane fetches per batch
     const int lane = threadIdx.x & 31, gl = lane & (GROUP - 1);
-    const unsigned gmask = ((1u << GROUP) - 1u) << (lane & ~(GROUP - 1));
-    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;
-    if (slot >= nrows) return;
-    const int row = rows[slot];
-    const long long e0 = rowptr[row], e1 = rowptr[row + 1];
+    const unsigned gmask = (GROUP == 32 ? 0xffffffffu : ((1u << GROUP) - 1u)) << (lane & ~(GROUP - 1));
+    const long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;
+    if (idx >= nitems) return;   // the whole group leaves together
+    const Item it = load_item(items, (int)idx, ecv);
+    const uint2 pad = make_uint2((uint32_t)it.row, 0u);
+    const char* zl = reinterpret_cast<const char*>(Z) + 16ll * min(gl, F4 - 1);   // lanes past the last column read it again
+    const uint32_t ldzb = 4u * (uint32_t)ldz;
     float4 acc[1] = {make_float4(0.f, 0.f, 0.f, 0.f)};
-    for (long long e = e0; e < e1; e += GROUP) {
-        uint2 mine = make_uint2((uint32_t)row, 0u);
-        if (e + gl < e1) mine = __ldg(ecv + e + gl);
-        float4 z[GROUP];
-        float a[GROUP];
+    uint2 next[EPL];
 #pragma unroll
-        for (int t = 0; t < GROUP; ++t) {
-            const int c = __shfl_sync(gmask, (int)mine.x, t, GROUP);
-            a[t] = __uint_as_float(__shfl_sync(gmask, mine.y, t, GROUP));
-            z[t] = gl < F4 ? __ldg(reinterpret_cast<const float4*>(Z + (long long)c * ldz) + gl) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int t = 0; t < GROUP; ++t) {
-            acc[0].x = fmaf(a[t], z[t].x, acc[0].x);
-            acc[0].y = fmaf(a[t], z[t].y, acc[0].y);
-            acc[0].z = fmaf(a[t], z[t].z, acc[0].z);
-            acc[0].w = fmaf(a[t], z[t].w, acc[0].w);
-        }
+    for (int i = 0; i < EPL; ++i) {
+        const int e = gl + GROUP * i;
+        next[i] = (e < NB && e < it.len) ? __ldg(it.ent + e) : pad;
     }
-    finish_row<1, EPI>(acc, row, gl, GROUP, F4, out, ldo, ep);
-}
-
-// One warp per row of the binned list.
-template <int NV, int GROUP, bool EPI>
-__global__ void __launch_bounds__(256) spmm_rows_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
-                                                        const int32_t* __restrict__ rows, int nrows,
-                                                        const float* __restrict__ Z, int ldz, float* __restrict__ out,
-                                                        int ldo, int F4, EpiDev ep) {
-    const int lane = threadIdx.x & 31;
-    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (slot >= nrows) return;
-    const int row = rows[slot];
-    float4 acc[NV];
+    for (int b = 0; b < it.len; b += NB) {
+        uint2 mine[EPL];
 #pragma unroll
-    for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    walk_entries<NV, GROUP>(acc, ecv, rowptr[row], rowptr[row + 1], Z, ldz, lane, F4);
-    if (lane < GROUP) finish_row<NV, EPI>(acc, row, lane, GROUP, F4, out, ldo, ep);
-}
-
-// Long rows are cut into parts; one warp per part, its partial row goes to the part's scratch slot and
-// spmm_finish_kernel adds a row's slots in part order.  No barrier, no shared memory: a warp leaves as soon as
-// its own entries are done.
-template <int NV, int GROUP>
-__global__ void __launch_bounds__(256) spmm_parts_kernel(const int64_t* __restrict__ rowptr, const uint2* __restrict__ ecv,
-                                                         const int4* __restrict__ parts, int nparts,
-                                                         const float* __restrict__ Z, int ldz, int ldo, int F4,
-                                                         float* __restrict__ scratch) {
-    const int lane = threadIdx.x & 31;
-    const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (slot >= nparts) return;
-    const int4 pt = parts[slot];   // {row, first entry (relative to the row), entries, scratch slot}
-    const long long e0 = rowptr[pt.x] + pt.y;
-    float4 acc[NV];
-#pragma unroll
-    for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    walk_entries<NV, GROUP>(acc, ecv, e0, e0 + pt.z, Z, ldz, lane, F4);
-    if (lane < GROUP) {
-#pragma unroll
-        for (int j = 0; j < NV; ++j) {
-            int v = lane + GROUP * j;
-            if (v < F4) reinterpret_cast<float4*>(scratch + (long long)pt.w * ldo)[v] = acc[j];
+        for (int i = 0; i < EPL; ++i) {
+            mine[i] = next[i];
+            const int e = gl + GROUP * i;
+            next[i] = (e < NB && b + NB + e < it.len) ? __ldg(it.ent + b + NB + e) : pad;
         }
+        if (it.len - b > NB / 2) narrow_batch<GROUP, NB>(acc[0], mine, gmask, zl, ldzb);
+        else narrow_batch<GROUP, NB / 2>(acc[0], mine, gmask, zl, ldzb);
+    }
+    if (it.slot >= 0) {
+        if (gl < F4) reinterpret_cast<float4*>(scratch + (long long)it.slot * ldo)[gl] = acc[0];
+    } else {
+        finish_row<1, EPI>(acc, it.row, gl, GROUP, F4, out, ldo, ep);
     }
 }
 
@@ -200,8 +141,8 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    // four slots are loaded together and added in slot order (a slot past the last one counts as zero)
-    constexpr int Q = NV <= 2 ? 4 : (NV <= 4 ? 2 : 1);
+    // several slots are loaded together and added in slot order (a slot past the last one counts as zero)
+    constexpr int Q = NV == 1 ? 16 : (NV == 2 ? 8 : (NV <= 4 ? 4 : 2));
     for (int p = 0; p < f.z; p += Q) {
         float4 t[Q][NV];
 #pragma unroll
@@ -313,9 +254,9 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
     const int idx = blockIdx.x * kItemWarps + warp;
     if (idx >= nitems) return;
     uint2* stage = stage_all[warp];
-    const int4 it = __ldg(items + idx);   // {row, entry position low, (position high << 16) | entries, scratch slot or -1}
-    const int row = it.x, len = (int)((uint32_t)it.z & 0xFFFFu);
-    const uint2* ent = ecv + (((long long)((uint32_t)it.z >> 16) << 32) | (long long)(uint32_t)it.y);
+    const Item item = load_item(items, idx, ecv);
+    const int row = item.row, len = item.len;
+    const uint2* ent = item.ent;
     const uint2 pad = make_uint2((uint32_t)row, 0u);
     // lanes past the last column read the last one (their sums are never stored)
     ZLane<NV, OFF32> zl;
@@ -342,11 +283,11 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
         for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU, OFF32>(acc, stage + t, zl);
         gather_tail<NV, UU / 2, OFF32>(acc, stage + t, cnt - t, zl);
     }
-    if (it.w >= 0) {
+    if (item.slot >= 0) {
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
             const int v = lane + 32 * j;
-            if (v < F4) reinterpret_cast<float4*>(scratch + (long long)it.w * ldo)[v] = acc[j];
+            if (v < F4) reinterpret_cast<float4*>(scratch + (long long)item.slot * ldo)[v] = acc[j];
         }
     } else {
         finish_row<NV, EPI>(acc, row, lane, 32, F4, out, ldo, ep);
@@ -372,23 +313,13 @@ static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, floa
         }
         return cudaGetLastError();
     }
-    if (A.nparts > 0) {  // long rows first: they are the longest items of work
-        spmm_parts_kernel<NV, GROUP><<<(unsigned)((A.nparts + 7) / 8), 256, 0, s>>>(A.rowptr, A.ecv, A.parts, A.nparts, Z, ldz, ldo, F4,
-                                                                                   A.scratch);
+    if (A.nitems > 0) {
+        const unsigned grid = (unsigned)(((long long)A.nitems * GROUP + 255) / 256);
+        spmm_items_narrow_kernel<GROUP, EPI><<<grid, 256, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
         ++g_kernel_launches;
     }
     if (A.nfin > 0) {
         spmm_finish_kernel<NV, GROUP, EPI><<<(unsigned)((A.nfin + 7) / 8), 256, 0, s>>>(A.fin, A.nfin, A.scratch, out, ldo, F4, ep);
-        ++g_kernel_launches;
-    }
-    if (A.nperm > 0) {
-        if constexpr (GROUP < 32) {
-            const unsigned grid = (unsigned)(((long long)A.nperm * GROUP + 255) / 256);
-            spmm_rows_narrow_kernel<GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
-        } else {
-            const unsigned grid = (unsigned)((A.nperm + 7) / 8);
-            spmm_rows_kernel<NV, GROUP, EPI><<<grid, 256, 0, s>>>(A.rowptr, A.ecv, A.perm, A.nperm, Z, ldz, out, ldo, F4, ep);
-        }
         ++g_kernel_launches;
     }
     return cudaGetLastError();

@@ -241,12 +241,19 @@ int64_t part_entries_for(const std::vector<int64_t>& rowptr) {
     return part;
 }
 
+// Part length of one cut row: the store's part length, or longer so that the row has at most kMaxSlotsPerRow parts
+// (the parts of a hub row then end inside the main kernel instead of as a long serial sum in the finishing one).
+static int64_t row_part_entries(int64_t len, int64_t part) {
+    const int64_t want = round_up((len + kMaxSlotsPerRow - 1) / kMaxSlotsPerRow, 32);
+    return std::min<int64_t>(std::max(part, want), 65535 / 32 * 32);
+}
+
 int64_t count_slots(const std::vector<int64_t>& rowptr) {
     const int64_t part = part_entries_for(rowptr);
     int64_t slots = 0;
     for (size_t r = 0; r + 1 < rowptr.size(); ++r) {
         const int64_t len = rowptr[r + 1] - rowptr[r];
-        if (len > part) slots += (len + part - 1) / part;
+        if (len > part) { const int64_t pl = row_part_entries(len, part); slots += (len + pl - 1) / pl; }
     }
     return slots;
 }
@@ -268,10 +275,11 @@ void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& su
     for (int64_t r = 0; r < Np; ++r) {
         const int64_t len = rowptr[r + 1] - rowptr[r];
         if (len <= part) { out.perm[(size_t)start[bin_of(len)]++] = (int32_t)r; continue; }
-        const int64_t np = (len + part - 1) / part;
+        const int64_t pl = row_part_entries(len, part);
+        const int64_t np = (len + pl - 1) / pl;
         out.fin.push_back(make_int4((int)r, (int)out.slots, (int)np, 0));
         for (int64_t q = 0; q < np; ++q)
-            out.parts.push_back(make_int4((int)r, (int)(q * part), (int)std::min(part, len - q * part), (int)(out.slots + q)));
+            out.parts.push_back(make_int4((int)r, (int)(q * pl), (int)std::min(pl, len - q * pl), (int)(out.slots + q)));
         out.slots += np;
     }
     // the unified list: subgraph by subgraph (the operand rows one subgraph gathers stay together in L2), parts
