@@ -29,7 +29,10 @@ UNIT = "epochs/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/; keyed by (workload, profile entry).  A kernel changed since its capture
 # has no entry (reported as null).
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # spmm_items_kernel (76.8 MB read + 32.9 MB written) + spmm_finish_kernel (14.9 MB read), profiles/spmm_items_c2.md
+    ("c2", "spmm_fwd_l0"): 124.6e6,
+}
 
 
 def measured_peaks():
@@ -92,6 +95,22 @@ class ClockSampler:
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def max_over_ranks(ms, world, device="cpu"):
+    """The slowest rank's time: every rank contributes its own device time and receives the maximum."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(steps, world, ms):
+    """Whole-job epochs/s of `world` independent replicas that each ran `steps` epochs in `ms` (max over ranks)."""
+    return world * steps / (ms * 1e-3)
 
 
 def describe(w):
@@ -255,11 +274,8 @@ def main():
     launches = pkg.launch_count() - l0
     ms = e0.elapsed_time(e1)
     loss = g.get_loss()
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, world, "cuda")
+    value = job_value(args.steps, world, ms)
 
     # ---- per-kernel timing (CUDA events on the library's stream, same steps) --------------------------
     g.profile_enable(True)
@@ -307,11 +323,8 @@ def main():
     e1.record()
     barrier()
     ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e = {"value": world * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
+    ms_e2e = max_over_ranks(ms_e2e, world, "cuda")
+    e2e = {"value": job_value(e2e_steps, world, ms_e2e), "unit": UNIT, "steps": e2e_steps,
            "h2d_bytes_per_step": int(Xp.numel() * 4 + yp.numel() * 4), "d2h_bytes_per_step": int((g.K + 1) * 4)}
 
     ws_mb = g.workspace_bytes / 1e6
