@@ -74,8 +74,8 @@ typedef struct {
     float lr;             /* eta of the update equation (Section 3.3 / 3.4.2)                                 */
     float dropout;        /* probability of dropping a hidden unit after the ReLU, in [0,1); 0 = none         */
     uint64_t seed;        /* seed of the dropout mask and of the default initialisation                       */
-    int32_t gemm_mode;    /* 0: fp32-accurate transform (SIMT, or split-TF32 tensor cores);                   *
-                           * 1: bf16 operands with fp32 accumulation on tensor cores                          */
+    int32_t gemm_mode;    /* 0: fp32-accurate transform (SIMT, or tensor cores with every operand split in two);  *
+                           * 1: reduced-precision operands (one TF32 pass) with fp32 accumulation on tensor cores */
     int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form (GAD_ERR_UNSUPPORTED)       */
     float beta;           /* beta of the importance weight (Section 3.4.1); the paper uses 1                  */
     int32_t weighted;     /* 1: weighted global consensus (Section 3.4.2); 0: plain average (Definition 3)    */

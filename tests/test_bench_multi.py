@@ -23,17 +23,16 @@ def _rank(rank, world, port, out):
     import bench
     dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
     ms = bench.max_over_ranks(10.0 + 5.0 * rank, world)        # rank 1 is the slow one
-    out[rank] = (ms, bench.job_value(20, world, ms))
+    with open(os.path.join(out, "rank%d.json" % rank), "w") as fh:
+        json.dump([ms, bench.job_value(20, world, ms)], fh)
     dist.barrier()
     dist.destroy_process_group()
 
 
-def test_two_ranks_agree_on_the_slowest_time_and_sum_the_work():
+def test_two_ranks_agree_on_the_slowest_time_and_sum_the_work(tmp_path):
     world = 2
-    with mp.Manager() as m:
-        out = m.dict()
-        mp.spawn(_rank, args=(world, _free_port(), out), nprocs=world, join=True)
-        got = dict(out)
+    mp.spawn(_rank, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    got = [json.load(open(tmp_path / ("rank%d.json" % r))) for r in range(world)]
     assert got[0] == got[1]
     ms, value = got[0]
     assert ms == 15.0

@@ -61,8 +61,8 @@ def check_store(g, st):
 def grad_tol(g, ref, tol):
     """Tolerance for gradients.  A hidden unit whose pre-activation is zero within rounding can land on different
     sides of the ReLU in fp32 and in the fp64 oracle; both results are valid, but such a unit changes its gradient
-    path by a finite amount.  Units like that must be genuine ties (magnitude <= 1e-5 of the layer's largest
-    value); when there are any, the gradient comparison is relaxed to 5e-2, otherwise it is `tol`."""
+    path by a finite amount.  Units like that must be genuine ties (magnitude <= max(1e-5, tol / 10) of the layer's
+    largest value); when there are any, the gradient comparison is relaxed to max(2 tol, 5e-2), otherwise it is `tol`."""
     ties, worst = 0, 0.0
     for l in range(1, len(g.dims) - 1):
         a, b = g.get_activation(l), ref.activation(l)
