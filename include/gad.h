@@ -154,9 +154,18 @@ int gad_get_store(gad_ctx* ctx, int64_t* rowptr, int32_t* col, float* val, int32
 int gad_get_activation(gad_ctx* ctx, int32_t l, float* out);
 
 /* Replaces the node features and/or labels (either may be NULL), host arrays of the shapes given to
- * gad_create.  The copies are enqueued on the stream from the caller's buffers, which must stay valid until
- * the stream has passed them (pinned memory makes the copy asynchronous). */
+ * gad_create.  The host-to-device copies go out on a second stream that the context owns, into one of two staging
+ * buffers, so they may overlap an epoch already enqueued on the context's stream; the reordering into store rows
+ * then runs on the context's stream, after the copy, and every later call sees the new inputs.  The caller's
+ * buffers must stay valid until a call that waits (gad_synchronize, gad_get_loss, ...) has returned; pinned memory
+ * makes the copy asynchronous.  Not part of the paper's algorithm: it is how a training loop streams inputs. */
 int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels);
+
+/* For a loop that never waits inside a step: enqueues the copy of the K+1 losses of the most recent epoch
+ * (layout of gad_get_loss) into loss_out, host memory that must be pinned and stay valid until gad_synchronize has
+ * returned.  No check for non-finite values is made.  gad_synchronize waits for both of the context's streams. */
+int gad_read_loss_async(gad_ctx* ctx, float* loss_out);
+int gad_synchronize(gad_ctx* ctx);
 
 /* Epoch counter (it indexes the dropout mask); set it to resume a run. */
 int gad_get_epoch(const gad_ctx* ctx, int64_t* epoch);

@@ -23,7 +23,7 @@ ERRORS = {-1: "GAD_ERR_ARG", -2: "GAD_ERR_RANGE", -3: "GAD_ERR_UNSORTED", -4: "G
 SYMBOLS = (
     "gad_workspace_bytes", "gad_create", "gad_train_epoch", "gad_get_loss", "gad_forward", "gad_subgraph_weights",
     "gad_consensus", "gad_get_params", "gad_set_params", "gad_get_grads", "gad_param_count", "gad_store_sizes",
-    "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
+    "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_read_loss_async", "gad_synchronize", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
     "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_subgraph_weights_static", "gad_launch_count",
     "gad_last_error", "gad_destroy",
 )
@@ -193,13 +193,20 @@ class Gad:
     def train_epoch(self, loss_out=None, wait=True):
         """gad_train_epoch.  With wait=True returns the float32 [K+1] losses (and waits for the stream); with
         wait=False only enqueues the epoch and returns None.  ``loss_out`` may be a preallocated float32 [K+1]
-        array (e.g. a view of pinned memory)."""
+        array (e.g. a view of pinned memory); with wait=False it must be pinned and receives the losses once the
+        stream gets there (gad_read_loss_async; call synchronize() before reading it)."""
         if not wait:
             self._ck(self._L.gad_train_epoch(self._h, None))
+            if loss_out is not None:
+                self._ck(self._L.gad_read_loss_async(self._h, _ptr(loss_out, C.c_float)))
             return None
         out = loss_out if loss_out is not None else np.zeros(self.K + 1, dtype=np.float32)
         self._ck(self._L.gad_train_epoch(self._h, _ptr(out, C.c_float)))
         return out
+
+    def synchronize(self):
+        """gad_synchronize: waits for everything enqueued on the context's two streams."""
+        self._ck(self._L.gad_synchronize(self._h))
 
     def get_loss(self):
         out = np.zeros(self.K + 1, dtype=np.float32)

@@ -42,7 +42,7 @@ struct Plan {
     size_t o_rowptr, o_ecv, o_perm, o_parts, o_fin, o_items, o_trowptr, o_tecv, o_tperm, o_tparts, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
         o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_dw_chunks, o_dw_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
         o_dw_partial, o_cs_partial, o_loss_partial, o_zeta_partial, o_zeta, o_loss, o_flags, o_zeta_f, o_w_f, o_stage,
-        o_stage_lab;
+        o_stage_lab, o_stage2, o_stage_lab2;
     std::vector<size_t> o_H, o_w_hi, o_w_lo, o_wt_hi, o_wt_lo;   // per layer
 };
 
@@ -137,6 +137,8 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_zeta = take(cur, 8 * (size_t)K); p.o_loss = take(cur, 4 * (size_t)(K + 1)); p.o_flags = take(cur, 16);
     p.o_zeta_f = take(cur, 4 * (size_t)K); p.o_w_f = take(cur, 4 * (size_t)K);
     p.o_stage = take(cur, 4 * (size_t)n * (size_t)std::max(p.dims[0], p.dims[p.L])); p.o_stage_lab = take(cur, 4 * (size_t)n);
+    // second staging pair: the copy of the next inputs may run while the previous ones are still being gathered
+    p.o_stage2 = take(cur, 4 * (size_t)n * (size_t)p.dims[0]); p.o_stage_lab2 = take(cur, 4 * (size_t)n);
     p.o_w_hi.resize(p.L); p.o_w_lo.resize(p.L); p.o_wt_hi.resize(p.L); p.o_wt_lo.resize(p.L);
     for (int l = 0; l < p.L; ++l) {
         const Layer& y = p.layers[l];
@@ -166,6 +168,9 @@ struct gad_ctx {
     bool profiling = false;
     std::vector<ProfEntry> prof;
     std::vector<float> host_block;  // staging for parameter pack / unpack
+    cudaStream_t copy_stream = nullptr;   // host -> device copies of gad_set_inputs
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_gathered[2] = {nullptr, nullptr};
+    int stage_idx = 0;              // staging pair the next gad_set_inputs uses
     bool hoist = false;             // keep A~ H^(0) across epochs (config flag bit 1)
     bool P_valid = false;           // A~ H^(0) matches the current features
     bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
@@ -445,6 +450,11 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->ws = (char*)workspace;
     ctx->cfg = *cfg;
     ctx->hoist = (cfg->flags & 2) != 0;
+    GAD_CK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+        GAD_CK(cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming));
+        GAD_CK(cudaEventCreateWithFlags(&ctx->ev_gathered[i], cudaEventDisableTiming));
+    }
     HostStore st;
     int rc = build_store(g, part, true, st, ctx->err);
     if (rc != GAD_OK) return fail(ctx, rc, ctx->err);
@@ -716,21 +726,44 @@ int gad_get_activation(gad_ctx* ctx, int32_t l, float* out) {
 int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels) {
     if (!ctx) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
+    if (!X && !labels) return GAD_OK;
+    // The copy goes out on its own stream into one of two staging pairs, so it can overlap the epoch that is still
+    // running on the context's stream; the gathers then run on the context's stream, after the copy.
+    const int b = ctx->stage_idx;
+    const size_t o_x = b ? p.o_stage2 : p.o_stage, o_l = b ? p.o_stage_lab2 : p.o_stage_lab;
+    GAD_CK(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_gathered[b], 0));   // the pair's previous contents have been consumed
+    if (X) GAD_CK(cudaMemcpyAsync(ctx->ws + o_x, X, 4 * (size_t)p.n * p.dims[0], cudaMemcpyHostToDevice, ctx->copy_stream));
+    if (labels) GAD_CK(cudaMemcpyAsync(ctx->ws + o_l, labels, 4 * (size_t)p.n, cudaMemcpyHostToDevice, ctx->copy_stream));
+    GAD_CK(cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
+    GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_copied[b], 0));
     if (X) {
-        GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage, X, 4 * (size_t)p.n * p.dims[0], cudaMemcpyHostToDevice, ctx->stream));
         GAD_RUN("gather_features", -1, 8.0 * p.Np * p.dims[0], 0.0, [&] {
-            return launch_gather_rows(ctx->at<float>(p.o_stage), p.dims[0], ctx->at<int32_t>(p.o_gid), p.Np, ctx->H(0), p.ld[0],
+            return launch_gather_rows(ctx->at<float>(o_x), p.dims[0], ctx->at<int32_t>(p.o_gid), p.Np, ctx->H(0), p.ld[0],
                                       ctx->stream);
         });
         ctx->P_valid = false;   // A~ H^(0) is aggregated again by the next forward pass
     }
     if (labels) {
-        GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage_lab, labels, 4 * (size_t)p.n, cudaMemcpyHostToDevice, ctx->stream));
         GAD_RUN("gather_labels", -1, 8.0 * p.Np, 0.0, [&] {
-            return launch_gather_labels(ctx->at<int32_t>(p.o_stage_lab), ctx->at<int32_t>(p.o_gid), p.Np, ctx->at<int32_t>(p.o_label),
+            return launch_gather_labels(ctx->at<int32_t>(o_l), ctx->at<int32_t>(p.o_gid), p.Np, ctx->at<int32_t>(p.o_label),
                                         ctx->stream);
         });
     }
+    GAD_CK(cudaEventRecord(ctx->ev_gathered[b], ctx->stream));
+    ctx->stage_idx ^= 1;
+    return GAD_OK;
+}
+
+int gad_read_loss_async(gad_ctx* ctx, float* loss_out) {
+    if (!ctx || !loss_out) return GAD_ERR_ARG;
+    GAD_CK(cudaMemcpyAsync(loss_out, ctx->ws + ctx->p.o_loss, 4 * (size_t)(ctx->p.K + 1), cudaMemcpyDeviceToHost, ctx->stream));
+    return GAD_OK;
+}
+
+int gad_synchronize(gad_ctx* ctx) {
+    if (!ctx) return GAD_ERR_ARG;
+    GAD_CK(cudaStreamSynchronize(ctx->copy_stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
     return GAD_OK;
 }
 
@@ -803,6 +836,11 @@ void gad_destroy(gad_ctx* ctx) {
     if (!ctx) return;
     for (auto& e : ctx->prof)
         for (auto& pr : e.pending) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
+    if (ctx->copy_stream) { cudaStreamSynchronize(ctx->copy_stream); cudaStreamDestroy(ctx->copy_stream); }
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
+        if (ctx->ev_gathered[i]) cudaEventDestroy(ctx->ev_gathered[i]);
+    }
     delete ctx;
 }
 

@@ -12,9 +12,9 @@
 // epoch by a small kernel; A tiles are split in shared memory by four warps of the GEMM kernel.  With passes = 1
 // only A B is issued on the unsplit operands (TF32 operand precision).
 //
-// One persistent CTA per SM, 10 warps: warp 0 issues TMA loads (128B-swizzled tiles) through a 3-stage ring,
-// warps 2-5 split the A tile, warp 1 issues tcgen05.mma, warps 6-9 drain the accumulator (tcgen05.ld) while
-// the MMA warp already fills the second accumulator.  Every mbarrier wait is bounded: on a time-out the CTA
+// One persistent CTA per SM, 18 warps: warp 0 issues TMA loads (128B-swizzled tiles) through a 3-stage ring,
+// warps 2-9 split the A tile, warp 1 issues tcgen05.mma, warps 10-17 drain the accumulator (tcgen05.ld, two warps
+// per quarter of the tensor-memory lanes) while the MMA warp already fills the second accumulator.  Every mbarrier wait is bounded: on a time-out the CTA
 // raises an error word, stops, frees its tensor memory and returns.
 #include <cuda.h>
 
@@ -30,7 +30,11 @@ constexpr int A_BYTES = BM * BK * 4;                      // 16 KiB
 constexpr int B_BYTES = BN_MAX * BK * 4;                  // 16 KiB
 constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;    // A_hi | A_lo | B_hi | B_lo
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
-constexpr int EPI_BYTES = 4 * 32 * 33 * 4;                // per-warp transpose tiles of the epilogue
+constexpr int EPI_WARPS = 8;                              // two per quarter of the tensor-memory lanes
+constexpr int EPI_BYTES = EPI_WARPS * 32 * 33 * 4;        // per-warp transpose tiles of the epilogue
+constexpr int SPLIT_WARPS = 8;                            // warps that split the A tile
+constexpr int EPI_WARP0 = 2 + SPLIT_WARPS;                // first epilogue warp (a multiple of 2, see the lane quarters)
+constexpr int ROWS_THREADS = 32 * (EPI_WARP0 + EPI_WARPS);
 constexpr int SMEM_BYTES_ROWS = SMEM_BYTES + EPI_BYTES;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int TMEM_COLS = 2 * BN_MAX;
@@ -139,7 +143,7 @@ struct TcArgs {
     ActEpi act;   // mode 2
 };
 
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(ROWS_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmBlo, const TcArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -155,12 +159,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     auto tempty = [&](int i) { return bars + 8u * (3 * STAGES + 2 + i); };
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    float* epi_sm = reinterpret_cast<float*>(sm + STAGES * STAGE_BYTES + 256);   // 4 warps x 32 x 33 floats
+    float* epi_sm = reinterpret_cast<float*>(sm + STAGES * STAGE_BYTES + 256);   // EPI_WARPS x 32 x 33 floats
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), 128); mbar_init(empty(s), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 128); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), 32 * SPLIT_WARPS); mbar_init(empty(s), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 32 * EPI_WARPS); }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -229,7 +233,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mma_commit(tfull(acc));           // accumulator complete
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
-    } else if (warp >= 2 && warp <= 5) {
+    } else if (warp >= 2 && warp < EPI_WARP0) {
         // ---------------- A split: hi = x rounded to TF32, lo = x - hi ----------------
         const int tt = threadIdx.x - 64;
         int stage = 0;
@@ -242,8 +246,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     float4* hi = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES);
                     float4* lo = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES + A_BYTES);
 #pragma unroll 4
-                    for (int j = 0; j < A_BYTES / 16 / 128; ++j) {
-                        const int i = tt + 128 * j;
+                    for (int j = 0; j < A_BYTES / 16 / (32 * SPLIT_WARPS); ++j) {
+                        const int i = tt + 32 * SPLIT_WARPS * j;
                         const float4 v = hi[i];
                         float4 h, l;
                         h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
@@ -259,9 +263,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= EPI_WARP0) {
         // ---------------- epilogue: tensor memory -> registers -> global ----------------
-        const int q = warp & 3;                    // this warp may read tensor-memory lanes 32q .. 32q+31
+        // this warp may read tensor-memory lanes 32q .. 32q+31; the two warps of a quarter take alternate
+        // blocks of 32 columns
+        const int q = warp & 3, half = (warp - EPI_WARP0) >> 2;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -272,9 +278,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // A thread receives one accumulator row (32 columns at a time); the warp turns its 32 x 32 block through
             // shared memory so that 8 lanes write 128 contiguous bytes of one output row.
-            float* tr = epi_sm + (warp - 6) * (32 * 33);
+            float* tr = epi_sm + (warp - EPI_WARP0) * (32 * 33);
             const int sub_r = lane >> 3, sub_c = (lane & 7) * 4;
-            for (int c0 = 0; c0 < a.BN && n0 + c0 < a.ldc; c0 += 32) {
+            for (int c0 = 32 * half; c0 < a.BN && n0 + c0 < a.ldc; c0 += 64) {
                 const int n = n0 + c0 + sub_c;
                 // the eight mask loads of this lane go out together, ahead of the accumulator read and of any store
                 float4 hm[8];
@@ -380,7 +386,8 @@ __device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr) {
            ((uint64_t)1 << 61);
 }
 
-__global__ void __launch_bounds__(256, 1)
+constexpr int TN_THREADS = 512;   // warp 0: TMA, warp 1: MMA, warps 2..15: operand split, warps 8..15 also drain the accumulator
+__global__ void __launch_bounds__(TN_THREADS, 1)
 gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmZ, const TnArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -394,7 +401,7 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     const uint32_t tfull = bars + 8u * (3 * STAGES);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    constexpr int NSPLIT = 192;   // threads of warps 2..7
+    constexpr int NSPLIT = TN_THREADS - 64;   // threads of warps 2..15
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -490,14 +497,15 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
     }
-    // epilogue by warps 4..7 once every MMA has completed
-    if (warp >= 4) {
-        const int q = warp & 3;
+    // epilogue by warps 8..15 (two per quarter of the tensor-memory lanes, alternate blocks of 32 columns) once
+    // every MMA has completed
+    if (warp >= 8) {
+        const int q = warp & 3, half = (warp - 8) >> 2;
         const bool done = mbar_wait(tfull, 0, abort_flag, a.err, 16);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int m = m0 + q * 32 + lane;
         float* P = a.partial + (long long)(blockIdx.x / tiles_per_chunk) * a.pstride_chunk;
-        for (int c0 = 0; c0 < a.BN && n0 + c0 < a.ldw; c0 += 32) {
+        for (int c0 = 32 * half; c0 < a.BN && n0 + c0 < a.ldw; c0 += 64) {
             uint32_t v[32];
             tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -585,7 +593,7 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
     a.act = act ? *act : ActEpi{};
     const long long total = (long long)ntiles * a.ntn;
     const unsigned grid = (unsigned)(total < num_sms ? total : num_sms);
-    gemm_tc_kernel<<<grid, 320, SMEM_BYTES_ROWS, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
+    gemm_tc_kernel<<<grid, ROWS_THREADS, SMEM_BYTES_ROWS, s>>>(*reinterpret_cast<const CUtensorMap*>(mapA), *reinterpret_cast<const CUtensorMap*>(mapB),
                                                  *reinterpret_cast<const CUtensorMap*>(mapBlo), a);
     ++g_kernel_launches;
     return cudaGetLastError();
@@ -604,7 +612,7 @@ cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, in
     a.chunks = chunks; a.BN = tc_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;
     a.partial = partial; a.pstride_chunk = (long long)M * ldw; a.passes = passes; a.err = err;
     const unsigned grid = (unsigned)((long long)nchunks * a.ntm * a.ntn);
-    gemm_tn_tc_kernel<<<grid, 256, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapH), *reinterpret_cast<const CUtensorMap*>(mapZ), a);
+    gemm_tn_tc_kernel<<<grid, TN_THREADS, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapH), *reinterpret_cast<const CUtensorMap*>(mapZ), a);
     ++g_kernel_launches;
     return cudaGetLastError();
 }

@@ -26,6 +26,33 @@ __device__ __forceinline__ bool cta_arrive_last(unsigned* counter, unsigned expe
     return last;
 }
 
+// Sum over the chunks [c0, c1) of src[c * stride + j], for one column j, as the finishing CTA does it: the chunk
+// range is cut into `nseg` equal segments, segment `seg` is added in chunk order by the calling thread (up to
+// eight loads in flight), and the caller then adds the segment sums in segment order.  The order of the additions
+// depends only on (c0, c1, nseg).
+template <class T>
+__device__ __forceinline__ T segment_sum(const T* src, long long stride, long long j, int c0, int c1, int seg, int nseg) {
+    const int len = (c1 - c0 + nseg - 1) / nseg;
+    int c = c0 + seg * len;
+    const int e = min(c1, c + len);
+    T s = (T)0;
+    for (; c + 8 <= e; c += 8) {
+        T v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = __ldcg(src + (long long)(c + u) * stride + j);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
+    }
+    for (; c < e; ++c) s += __ldcg(src + (long long)c * stride + j);
+    return s;
+}
+// Columns are handled 256 / nseg at a time; nseg = 256 / (columns rounded up to a power of two), at least 1.
+__device__ __forceinline__ int segments_for(int cols) {
+    int p = 1;
+    while (p < cols && p < 256) p <<= 1;
+    return 256 / p;
+}
+
 struct LossTail {
     const int32_t* chunk_ptr;   // [K+1]
     int K;
@@ -35,13 +62,20 @@ struct LossTail {
     unsigned* counter;
 };
 
-// One thread per subgraph adds that subgraph's chunk sums in chunk order; thread 0 then adds the K subgraph sums
-// in ascending k for the global loss sum_k |T_k| L_k / sum_k |T_k|.
+// The chunk sums are first brought into shared memory by the whole CTA (4096 at a time); one thread per subgraph
+// then adds its subgraph's sums in chunk order, and thread 0 adds the K subgraph sums in ascending k for the global
+// loss sum_k |T_k| L_k / sum_k |T_k|.
 __device__ __forceinline__ void loss_finalize(const float* loss_partial, const float* __restrict__ inv_ntrain, const LossTail& t) {
+    __shared__ float stage[4096];
     __shared__ float sums[1024];
+    const int nchunks = t.chunk_ptr[t.K];
+    const bool staged = nchunks <= 4096;
+    if (staged)
+        for (int c = threadIdx.x; c < nchunks; c += blockDim.x) stage[c] = __ldcg(loss_partial + c);
+    __syncthreads();
     for (int k = threadIdx.x; k < t.K; k += blockDim.x) {
         float s = 0.f;
-        for (int c = t.chunk_ptr[k]; c < t.chunk_ptr[k + 1]; ++c) s += __ldcg(loss_partial + c);
+        for (int c = t.chunk_ptr[k]; c < t.chunk_ptr[k + 1]; ++c) s += staged ? stage[c] : __ldcg(loss_partial + c);
         if (k < 1024) sums[k] = s;
         t.loss[k] = s * inv_ntrain[k];
         if (!isfinite(s)) atomicExch(t.nonfinite, 1);
@@ -52,7 +86,7 @@ __device__ __forceinline__ void loss_finalize(const float* loss_partial, const f
         for (int k = 0; k < t.K; ++k) {
             if (k < 1024) { s += sums[k]; continue; }
             float sk = 0.f;
-            for (int c = t.chunk_ptr[k]; c < t.chunk_ptr[k + 1]; ++c) sk += __ldcg(loss_partial + c);
+            for (int c = t.chunk_ptr[k]; c < t.chunk_ptr[k + 1]; ++c) sk += staged ? stage[c] : __ldcg(loss_partial + c);
             s += sk;
         }
         t.loss[t.K] = s * t.inv_total;
@@ -241,21 +275,23 @@ __global__ void __launch_bounds__(256) colsum_chunks_kernel(const float* __restr
         }
         __syncthreads();
     }
-    // the last CTA of this subgraph adds the subgraph's chunk sums in chunk order
+    // the last CTA of this subgraph adds the subgraph's chunk sums: segments of the chunk range in parallel, then
+    // the segment sums in order
     const int c0 = chunk_ptr[c.k], c1 = chunk_ptr[c.k + 1];
     if (!cta_arrive_last(counters + c.k, (unsigned)(c1 - c0))) return;
-    for (int j = threadIdx.x; j < ld; j += blockDim.x) {
-        float s = 0.f;
-        int cc = c0;
-        for (; cc + 8 <= c1; cc += 8) {   // eight chunks' values requested together, added in chunk order
-            float v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = __ldcg(partial + (long long)(cc + u) * pstride_chunk + j);
-#pragma unroll
-            for (int u = 0; u < 8; ++u) s += v[u];
+    float* seg_sm = reinterpret_cast<float*>(sm);   // 256 floats of the 4 KiB tile above
+    const int nseg = segments_for(ld), per = 256 / nseg;
+    const int jl = threadIdx.x % per, seg = threadIdx.x / per;
+    for (int j0 = 0; j0 < ld; j0 += per) {
+        const int j = j0 + jl;
+        seg_sm[threadIdx.x] = j < ld ? segment_sum(partial, pstride_chunk, j, c0, c1, seg, nseg) : 0.f;
+        __syncthreads();
+        if (seg == 0 && j < ld) {
+            float t = seg_sm[jl];
+            for (int q = 1; q < nseg; ++q) t += seg_sm[q * per + jl];
+            out[(long long)c.k * ostride + off + j] = t;
         }
-        for (; cc < c1; ++cc) s += __ldcg(partial + (long long)cc * pstride_chunk + j);
-        out[(long long)c.k * ostride + off + j] = s;
+        __syncthreads();
     }
 }
 // Column sums of G over every subgraph's rows: out[k][off + j] = sum over the rows of subgraph k of G[row][j], j < ld.
@@ -308,32 +344,30 @@ __device__ __forceinline__ void zeta_finalize(int k, const double* partial, int 
                                               const int32_t* __restrict__ sub_off, const int64_t* __restrict__ deg_sum,
                                               const int64_t* __restrict__ deg_sq, float beta, double* __restrict__ zeta) {
     __shared__ double red[256];
+    __shared__ double seg_a[256], seg_b[256];
     const long long n = sub_off[k + 1] - sub_off[k];
     const bool uniform = deg_sum[k] == 0;
     const double D = uniform ? (double)n : (double)deg_sum[k];
     double q = 0.0;
-    if (n > 0)
-        for (int f = threadIdx.x; f < F; f += blockDim.x) {
-            double a = 0.0, b = 0.0;
-            const int c1 = chunk_ptr[k + 1];
-            int c = chunk_ptr[k];
-            for (; c + 8 <= c1; c += 8) {   // eight chunks' values requested together, added in chunk order
-                double va[8], vb[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    va[u] = __ldcg(partial + (long long)(c + u) * 2 * ld + f);
-                    vb[u] = __ldcg(partial + (long long)(c + u) * 2 * ld + ld + f);
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) { a += va[u]; b += vb[u]; }
+    if (n > 0) {
+        // segments of the chunk range in parallel, the segment sums then added in order, per feature
+        const int c0 = chunk_ptr[k], c1 = chunk_ptr[k + 1];
+        const int nseg = segments_for(F), per = 256 / nseg;
+        const int fl = threadIdx.x % per, seg = threadIdx.x / per;
+        for (int f0 = 0; f0 < F; f0 += per) {
+            const int f = f0 + fl;
+            seg_a[threadIdx.x] = f < F ? segment_sum(partial, 2ll * ld, f, c0, c1, seg, nseg) : 0.0;
+            seg_b[threadIdx.x] = f < F ? segment_sum(partial, 2ll * ld, (long long)ld + f, c0, c1, seg, nseg) : 0.0;
+            __syncthreads();
+            if (seg == 0 && f < F) {
+                double a = seg_a[fl], b = seg_b[fl];
+                for (int t = 1; t < nseg; ++t) { a += seg_a[t * per + fl]; b += seg_b[t * per + fl]; }
+                const double m1 = a / D;
+                q += b / D - m1 * m1;
             }
-            for (; c < c1; ++c) {
-                a += __ldcg(partial + (long long)c * 2 * ld + f);
-                b += __ldcg(partial + (long long)c * 2 * ld + ld + f);
-            }
-            const double m1 = a / D;
-            q += b / D - m1 * m1;
+            __syncthreads();
         }
+    }
     red[threadIdx.x] = q;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {

@@ -280,6 +280,33 @@ def test_set_inputs_replaces_features_and_labels(tiny):
         assert rel_err(g.get_grads(1), ref.get_grads(1)) <= TOL
 
 
+def test_pipelined_inputs_and_asynchronous_loss_reads(tiny):
+    """A loop that never waits inside a step: inputs alternate between two pinned buffers (the copies go out on the
+    context's second stream into alternating staging buffers), losses come back asynchronously."""
+    import torch
+    w = tiny
+    theta = glorot_params(w.dims, np.random.default_rng(11))
+    rng = np.random.default_rng(12)
+    Xs = [w.X, rng.standard_normal(w.X.shape).astype(np.float32), rng.standard_normal(w.X.shape).astype(np.float32)]
+    pinned = [torch.from_numpy(x).pin_memory() for x in Xs]
+    labels = torch.from_numpy(w.labels).pin_memory()
+    losses = torch.zeros((5, w.K + 1), dtype=torch.float32).pin_memory()
+    cp, cn, hp, hn = w.flat_partition()
+    st = orc().Store(w.n, w.rowptr, w.col, cp, cn, hp, hn)
+    with pkg().from_workload(w, theta) as g:
+        for i in range(5):
+            g.set_inputs(pinned[i % 3], labels)
+            g.train_epoch(loss_out=losses[i].numpy(), wait=False)
+        g.synchronize()
+        params = theta
+        for i in range(5):
+            ref = orc().Model(st, Xs[i % 3], w.labels, w.split, w.dims, params, lr=w.lr)
+            want = ref.train_epoch()
+            params = ref.get_params(0)      # identical replicas after the weighted consensus
+            assert np.max(np.abs(losses[i].numpy() - want)) <= 1e-5, "step %d" % i
+        assert rel_err(g.get_params(0), params) <= TOL
+
+
 def test_kept_input_aggregation_follows_new_features(tiny):
     """flags bit 1 keeps A~ H^(0) across epochs; new features must replace it."""
     w = tiny
