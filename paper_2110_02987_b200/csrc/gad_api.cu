@@ -169,6 +169,8 @@ struct gad_ctx {
     std::vector<ProfEntry> prof;
     std::vector<float> host_block;  // staging for parameter pack / unpack
     cudaStream_t copy_stream = nullptr;   // host -> device copies of gad_set_inputs
+    cudaStream_t side_stream = nullptr;   // small kernels of an epoch that depend on little (operand split, zeta, bias gradients)
+    cudaEvent_t ev_fork = nullptr, ev_split = nullptr, ev_g1 = nullptr, ev_bias = nullptr, ev_join = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_gathered[2] = {nullptr, nullptr};
     int stage_idx = 0;              // staging pair the next gad_set_inputs uses
     bool hoist = false;             // keep A~ H^(0) across epochs (config flag bit 1)
@@ -234,7 +236,19 @@ int run(gad_ctx* ctx, const char* name, int layer, double bytes, double flops, F
 
 double spmm_bytes(const Plan& p, int F) { return 8.0 * p.nnz + 8.0 * p.Np + 8.0 * (double)p.Np * F; }
 
-int forward_pass(gad_ctx* ctx, bool train) {
+// Inside a training epoch the kernels that depend on little (operand split of the weights, zeta, bias gradients) go
+// to a second stream and run beside the aggregation / transform sequence; events order them against it.  While
+// per-kernel timing is on everything stays on the context's stream, where the timing events are recorded.
+cudaStream_t side_of(gad_ctx* ctx) { return ctx->profiling ? ctx->stream : ctx->side_stream; }
+// Work enqueued on `to` after this call starts only when the work enqueued on `from` so far has finished.
+int hand_over(gad_ctx* ctx, cudaStream_t from, cudaStream_t to, cudaEvent_t ev) {
+    if (from == to) return GAD_OK;
+    GAD_CK(cudaEventRecord(ev, from));
+    GAD_CK(cudaStreamWaitEvent(to, ev, 0));
+    return GAD_OK;
+}
+
+int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
     const Plan& p = ctx->p;
     float* Z = ctx->at<float>(p.o_G2);
     const float* params = ctx->at<float>(p.o_params);
@@ -245,9 +259,11 @@ int forward_pass(gad_ctx* ctx, bool train) {
             GAD_RUN("split_weights", l, 20.0 * p.K * y.fi * y.fo, 0.0, [&] {
                 return launch_split_weights(params, p.pstride, y.w_int, y.fi, y.fo, y.ldw, y.ldi, p.K, ctx->at<float>(p.o_w_hi[l]),
                                             ctx->at<float>(p.o_w_lo[l]), ctx->at<float>(p.o_wt_hi[l]), ctx->at<float>(p.o_wt_lo[l]),
-                                            ctx->stream);
+                                            ss);
             });
         }
+    bool split_pending = ctx->use_tc && ss != ctx->stream;   // the first transform waits for the split operands
+    if (split_pending) GAD_CK(cudaEventRecord(ctx->ev_split, ss));
     for (int l = 0; l < p.L; ++l) {
         const Layer& y = p.layers[l];
         Epilogue ep{params, p.pstride, y.b_int, ctx->at<int32_t>(p.o_sub_off), p.K, l < p.L - 1 ? 1 : 0,
@@ -261,6 +277,7 @@ int forward_pass(gad_ctx* ctx, bool train) {
                 ctx->P_valid = true;
             }
             const ActEpi act = make_act(ep, 0);
+            if (split_pending) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
             GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
                 if (ctx->use_tc)
                     return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 2, passes, y.fi, y.fo,
@@ -271,6 +288,7 @@ int forward_pass(gad_ctx* ctx, bool train) {
             });
             continue;
         }
+        if (split_pending) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
         GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
             if (ctx->use_tc)
                 return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 0, passes, y.fi, y.fo, Z,
@@ -285,19 +303,19 @@ int forward_pass(gad_ctx* ctx, bool train) {
     return GAD_OK;
 }
 
-int zeta_pass(gad_ctx* ctx) {
+int zeta_pass(gad_ctx* ctx, cudaStream_t s) {
     const Plan& p = ctx->p;
     GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 1), 4.0 * p.Np * p.dims[0], [&] {
         return launch_zeta(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
                            (int)p.chunks.size(), ctx->at<int32_t>(p.o_chunk_ptr), ctx->at<int32_t>(p.o_sub_off),
                            ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_deg_sq), ctx->cfg.beta,
                            ctx->at<double>(p.o_zeta_partial), ctx->at<unsigned>(p.o_counters) + 1 + p.K, ctx->at<double>(p.o_zeta),
-                           ctx->stream);
+                           s);
     });
     return GAD_OK;
 }
 
-int backward_pass(gad_ctx* ctx) {
+int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
     const Plan& p = ctx->p;
     float* G1 = ctx->at<float>(p.o_G1);
     float* G2 = ctx->at<float>(p.o_G2);
@@ -312,10 +330,14 @@ int backward_pass(gad_ctx* ctx) {
     const float scale = ctx->cfg.dropout > 0.f ? 1.f / (1.f - ctx->cfg.dropout) : 1.f;
     for (int l = p.L - 1; l >= 0; --l) {
         const Layer& y = p.layers[l];
+        // db reads dPre (G1) beside the kernels that follow; the next writer of G1 waits for it
+        int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_g1);
+        if (rc != GAD_OK) return rc;
         GAD_RUN("bias_grad", l, 4.0 * p.Np * y.fo, 1.0 * p.Np * y.fo, [&] {
             return launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr,
-                                        ctx->at<unsigned>(p.o_counters) + 1, grads, p.pstride, y.b_int, ctx->stream);
+                                        ctx->at<unsigned>(p.o_counters) + 1, grads, p.pstride, y.b_int, ss);
         });
+        if (ss != ctx->stream) GAD_CK(cudaEventRecord(ctx->ev_bias, ss));
         const bool agg_first = l == 0 && p.agg_first0;   // then dW = (A~ X)^T dPre and nothing flows further back
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
@@ -331,6 +353,7 @@ int backward_pass(gad_ctx* ctx) {
             return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, dw_chunk_ptr, p.K, grads, p.pstride,
                                         y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
         });
+        if (l > 0 && ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
         if (l > 0)
             GAD_RUN("gemm_dh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
                 if (ctx->use_tc)
@@ -451,6 +474,9 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->cfg = *cfg;
     ctx->hoist = (cfg->flags & 2) != 0;
     GAD_CK(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    GAD_CK(cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t* e : {&ctx->ev_fork, &ctx->ev_split, &ctx->ev_g1, &ctx->ev_bias, &ctx->ev_join})
+        GAD_CK(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
     for (int i = 0; i < 2; ++i) {
         GAD_CK(cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming));
         GAD_CK(cudaEventCreateWithFlags(&ctx->ev_gathered[i], cudaEventDisableTiming));
@@ -597,8 +623,11 @@ int gad_get_loss(gad_ctx* ctx, float* loss_out) {
 int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
     if (!ctx) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
-    int rc = forward_pass(ctx, true);
+    cudaStream_t ss = side_of(ctx);
+    int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_fork);   // this epoch's side work follows everything enqueued so far
     if (rc != GAD_OK) return rc;
+    if ((rc = forward_pass(ctx, true, ss)) != GAD_OK) return rc;
+    if (ss != ctx->stream && (rc = zeta_pass(ctx, ss)) != GAD_OK) return rc;   // beside the forward pass
     const int C = p.dims[p.L];
     GAD_RUN("softmax_xent", -1, 8.0 * p.Np * C, 0.0, [&] {
         return launch_softmax_xent(ctx->H(p.L), p.ld[p.L], C, ctx->at<int32_t>(p.o_label), ctx->at<uint8_t>(p.o_train),
@@ -607,8 +636,9 @@ int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
                                    ctx->ntrain_total > 0 ? 1.f / (float)ctx->ntrain_total : 0.f, ctx->at<float>(p.o_loss),
                                    ctx->at<int32_t>(p.o_flags), ctx->at<unsigned>(p.o_counters), ctx->stream);
     });
-    if ((rc = backward_pass(ctx)) != GAD_OK) return rc;
-    if ((rc = zeta_pass(ctx)) != GAD_OK) return rc;
+    if ((rc = backward_pass(ctx, ss)) != GAD_OK) return rc;
+    if (ss == ctx->stream && (rc = zeta_pass(ctx, ss)) != GAD_OK) return rc;
+    if ((rc = hand_over(ctx, ss, ctx->stream, ctx->ev_join)) != GAD_OK) return rc;
     GAD_RUN("sgd_consensus", -1, 12.0 * p.K * p.Pint, 4.0 * p.K * p.Pint, [&] {
         return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
                                     ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->stream);
@@ -621,7 +651,7 @@ int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
 int gad_forward(gad_ctx* ctx, float* logits_out) {
     if (!ctx || !logits_out) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
-    int rc = forward_pass(ctx, false);
+    int rc = forward_pass(ctx, false, ctx->stream);
     if (rc != GAD_OK) return rc;
     const int C = p.dims[p.L];
     GAD_CK(cudaMemsetAsync(ctx->ws + p.o_stage, 0, 4 * (size_t)p.n * C, ctx->stream));
@@ -635,7 +665,7 @@ int gad_forward(gad_ctx* ctx, float* logits_out) {
 int gad_subgraph_weights(gad_ctx* ctx, float* zeta_out, float* w_out) {
     if (!ctx) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
-    int rc = zeta_pass(ctx);
+    int rc = zeta_pass(ctx, ctx->stream);
     if (rc != GAD_OK) return rc;
     GAD_CK(launch_weights(ctx->at<double>(p.o_zeta), p.K, ctx->cfg.weighted, ctx->at<float>(p.o_zeta_f), ctx->at<float>(p.o_w_f),
                           ctx->stream));
@@ -648,7 +678,7 @@ int gad_subgraph_weights(gad_ctx* ctx, float* zeta_out, float* w_out) {
 int gad_consensus(gad_ctx* ctx) {
     if (!ctx) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
-    int rc = zeta_pass(ctx);
+    int rc = zeta_pass(ctx, ctx->stream);
     if (rc != GAD_OK) return rc;
     GAD_RUN("consensus", -1, 8.0 * p.K * p.Pint, 2.0 * p.K * p.Pint, [&] {
         return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, 0.f,
@@ -763,6 +793,7 @@ int gad_read_loss_async(gad_ctx* ctx, float* loss_out) {
 int gad_synchronize(gad_ctx* ctx) {
     if (!ctx) return GAD_ERR_ARG;
     GAD_CK(cudaStreamSynchronize(ctx->copy_stream));
+    GAD_CK(cudaStreamSynchronize(ctx->side_stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));
     return GAD_OK;
 }
@@ -837,6 +868,9 @@ void gad_destroy(gad_ctx* ctx) {
     for (auto& e : ctx->prof)
         for (auto& pr : e.pending) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
     if (ctx->copy_stream) { cudaStreamSynchronize(ctx->copy_stream); cudaStreamDestroy(ctx->copy_stream); }
+    if (ctx->side_stream) { cudaStreamSynchronize(ctx->side_stream); cudaStreamDestroy(ctx->side_stream); }
+    for (cudaEvent_t e : {ctx->ev_fork, ctx->ev_split, ctx->ev_g1, ctx->ev_bias, ctx->ev_join})
+        if (e) cudaEventDestroy(e);
     for (int i = 0; i < 2; ++i) {
         if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
         if (ctx->ev_gathered[i]) cudaEventDestroy(ctx->ev_gathered[i]);
