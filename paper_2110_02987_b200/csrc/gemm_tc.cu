@@ -29,7 +29,9 @@ constexpr int BM = 128, BK = 32, STAGES = 3, BN_MAX = 128;
 constexpr int A_BYTES = BM * BK * 4;                      // 16 KiB
 constexpr int B_BYTES = BN_MAX * BK * 4;                  // 16 KiB
 constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;    // A_hi | A_lo | B_hi | B_lo
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int RING_BYTES = STAGES * STAGE_BYTES;           // the rows kernel cuts this into 3 .. 6 stages
+constexpr int MAX_STAGES = 6;
+constexpr int SMEM_BYTES = RING_BYTES + 1024 + 256;
 constexpr int EPI_WARPS = 8;                              // two per quarter of the tensor-memory lanes
 constexpr int EPI_BYTES = EPI_WARPS * 32 * 33 * 4;        // per-warp transpose tiles of the epilogue
 constexpr int SPLIT_WARPS = 8;                            // warps that split the A tile
@@ -151,20 +153,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
     uint8_t* sm = smem_raw + pad;                 // 1024-byte aligned: the 128B swizzle pattern repeats every 1024 bytes
     const uint32_t sm_addr = raw_addr + pad;
-    const uint32_t bars = sm_addr + STAGES * STAGE_BYTES;
+    // The ring holds as many stages as fit: a stage is A (and its low half when splitting) plus the B tile(s) of
+    // BN rows, so narrow outputs and the single-pass mode get a deeper ring.
+    const uint32_t b_bytes = (uint32_t)a.BN * BK * 4;
+    const uint32_t off_b = a.passes > 1 ? 2u * A_BYTES : (uint32_t)A_BYTES;
+    const uint32_t stage_bytes = off_b + (a.passes > 1 ? 2u : 1u) * b_bytes;
+    const int nst = min(MAX_STAGES, (int)(RING_BYTES / stage_bytes));
+    const uint32_t bars = sm_addr + RING_BYTES;
     auto full = [&](int s) { return bars + 8u * s; };
-    auto xfull = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto empty = [&](int s) { return bars + 8u * (2 * STAGES + s); };
-    auto tfull = [&](int i) { return bars + 8u * (3 * STAGES + i); };
-    auto tempty = [&](int i) { return bars + 8u * (3 * STAGES + 2 + i); };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
+    auto xfull = [&](int s) { return bars + 8u * (MAX_STAGES + s); };
+    auto empty = [&](int s) { return bars + 8u * (2 * MAX_STAGES + s); };
+    auto tfull = [&](int i) { return bars + 8u * (3 * MAX_STAGES + i); };
+    auto tempty = [&](int i) { return bars + 8u * (3 * MAX_STAGES + 2 + i); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + RING_BYTES + 8 * (3 * MAX_STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
-    float* epi_sm = reinterpret_cast<float*>(sm + STAGES * STAGE_BYTES + 256);   // EPI_WARPS x 32 x 33 floats
+    float* epi_sm = reinterpret_cast<float*>(sm + RING_BYTES + 256);   // EPI_WARPS x 32 x 33 floats
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), 32 * SPLIT_WARPS); mbar_init(empty(s), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), 32 * EPI_WARPS); }
+        // one arrival per splitting / draining warp
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), SPLIT_WARPS); mbar_init(empty(s), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(tfull(i), 1); mbar_init(tempty(i), EPI_WARPS); }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -179,7 +188,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int ntiles = a.ntiles_rows * a.ntn;
     const int nkb = (a.Kd + BK - 1) / BK;
-    const uint32_t b_bytes = (uint32_t)a.BN * BK * 4;
     const uint32_t tx_bytes = A_BYTES + (a.passes > 1 ? 2u : 1u) * b_bytes;
 
     if (warp == 0 && lane == 0) {
@@ -193,11 +201,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int kb = 0; kb < nkb; ++kb) {
                 if (!(ok = mbar_wait(empty(stage), phase ^ 1u, abort_flag, a.err, 1))) break;
                 mbar_expect_tx(full(stage), tx_bytes);
-                const uint32_t base = sm_addr + stage * STAGE_BYTES;
+                const uint32_t base = sm_addr + stage * stage_bytes;
                 tma_load_2d(base, &tmA, kb * BK, sp.row0, full(stage));
-                tma_load_3d(base + 2 * A_BYTES, &tmB, kb * BK, n0, sp.k, full(stage));
-                if (a.passes > 1) tma_load_3d(base + 2 * A_BYTES + B_BYTES, &tmBlo, kb * BK, n0, sp.k, full(stage));
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                tma_load_3d(base + off_b, &tmB, kb * BK, n0, sp.k, full(stage));
+                if (a.passes > 1) tma_load_3d(base + off_b + b_bytes, &tmBlo, kb * BK, n0, sp.k, full(stage));
+                if (++stage == nst) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1 && lane == 0) {
@@ -214,20 +222,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 3))) break;
                 if (!(ok = mbar_wait(xfull(stage), phase, abort_flag, a.err, 4))) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t base = sm_addr + stage * STAGE_BYTES;
+                const uint32_t base = sm_addr + stage * stage_bytes;
                 const uint64_t a_hi = smem_desc(base), a_lo = smem_desc(base + A_BYTES);
-                const uint64_t b_hi = smem_desc(base + 2 * A_BYTES), b_lo = smem_desc(base + 2 * A_BYTES + B_BYTES);
+                const uint64_t b_hi = smem_desc(base + off_b), b_lo = smem_desc(base + off_b + b_bytes);
+                // One thread issues every MMA, so the instructions between two MMAs are the cost: the common case of a
+                // full block of four K steps is unrolled with constant descriptor offsets (8 TF32 values = 32 bytes = 2
+                // descriptor units along K).
                 const int nks = min(BK / 8, (a.Kd - kb * BK + 7) / 8);
-                for (int ks = 0; ks < nks; ++ks) {
-                    const uint64_t adv = (uint64_t)(ks * 32 >> 4);   // 8 TF32 values = 32 bytes along K
-                    mma_tf32(d, a_hi + adv, b_hi + adv, idesc, (kb | ks) != 0 ? 1u : 0u);
+                if (nks == BK / 8) {
                     if (a.passes > 1) {
-                        mma_tf32(d, a_hi + adv, b_lo + adv, idesc, 1u);
-                        mma_tf32(d, a_lo + adv, b_hi + adv, idesc, 1u);
+#pragma unroll
+                        for (int ks = 0; ks < BK / 8; ++ks) {
+                            mma_tf32(d, a_hi + 2 * ks, b_hi + 2 * ks, idesc, ks == 0 ? (kb != 0 ? 1u : 0u) : 1u);
+                            mma_tf32(d, a_hi + 2 * ks, b_lo + 2 * ks, idesc, 1u);
+                            mma_tf32(d, a_lo + 2 * ks, b_hi + 2 * ks, idesc, 1u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < BK / 8; ++ks)
+                            mma_tf32(d, a_hi + 2 * ks, b_hi + 2 * ks, idesc, ks == 0 ? (kb != 0 ? 1u : 0u) : 1u);
+                    }
+                } else {
+                    for (int ks = 0; ks < nks; ++ks) {
+                        const uint64_t adv = (uint64_t)(2 * ks);
+                        mma_tf32(d, a_hi + adv, b_hi + adv, idesc, (kb | ks) != 0 ? 1u : 0u);
+                        if (a.passes > 1) {
+                            mma_tf32(d, a_hi + adv, b_lo + adv, idesc, 1u);
+                            mma_tf32(d, a_lo + adv, b_hi + adv, idesc, 1u);
+                        }
                     }
                 }
                 mma_commit(empty(stage));     // the stage may be refilled once these MMAs have read it
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                if (++stage == nst) { stage = 0; phase ^= 1u; }
             }
             if (!ok) break;
             mma_commit(tfull(acc));           // accumulator complete
@@ -241,10 +267,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 5))) break;
+                // (the vote keeps the warp together: lanes may see a time-out or an abort at different polls)
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait(full(stage), phase, abort_flag, a.err, 5)))) break;
                 if (a.passes > 1) {
-                    float4* hi = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES);
-                    float4* lo = reinterpret_cast<float4*>(sm + stage * STAGE_BYTES + A_BYTES);
+                    float4* hi = reinterpret_cast<float4*>(sm + stage * stage_bytes);
+                    float4* lo = reinterpret_cast<float4*>(sm + stage * stage_bytes + A_BYTES);
 #pragma unroll 4
                     for (int j = 0; j < A_BYTES / 16 / (32 * SPLIT_WARPS); ++j) {
                         const int i = tt + 32 * SPLIT_WARPS * j;
@@ -259,8 +286,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
                 }
-                mbar_arrive(xfull(stage));
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(xfull(stage));
+                if (++stage == nst) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp >= EPI_WARP0) {
@@ -274,7 +302,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
             const RowSpan sp = a.tiles[t / a.ntn];
             const int n0 = (t % a.ntn) * a.BN;
-            if (!(ok = mbar_wait(tfull(acc), acc_phase, abort_flag, a.err, 6))) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(tfull(acc), acc_phase, abort_flag, a.err, 6)))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // A thread receives one accumulator row (32 columns at a time); the warp turns its 32 x 32 block through
             // shared memory so that 8 lanes write 128 contiguous bytes of one output row.
@@ -322,7 +350,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __syncwarp();
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            mbar_arrive(tempty(acc));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -331,7 +360,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // shared memory is released.
     __syncthreads();
     if (*abort_flag && threadIdx.x == 0)
-        for (int s = 0; s < STAGES; ++s)
+        for (int s = 0; s < nst; ++s)
             for (uint32_t i = 0; i < 4096u; ++i)
                 if (mbar_try_wait(full(s), 0) || mbar_try_wait(full(s), 1)) break;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -450,14 +479,25 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t base = sm_addr + stage * STAGE_BYTES;
             const int nks = min(BK / 8, (c.nrows - kb * BK + 7) / 8);
-            for (int ks = 0; ks < nks; ++ks) {
-                const uint32_t off = (uint32_t)ks * 1024u;   // next group of 8 rows
-                const uint64_t a_hi = smem_desc_mn(base + off), a_lo = smem_desc_mn(base + A_BYTES + off);
-                const uint64_t b_hi = smem_desc_mn(base + 2 * A_BYTES + off), b_lo = smem_desc_mn(base + 2 * A_BYTES + B_BYTES + off);
-                mma_tf32(tmem_base, a_hi, b_hi, idesc, (kb | ks) != 0 ? 1u : 0u);
-                if (a.passes > 1) {
-                    mma_tf32(tmem_base, a_hi, b_lo, idesc, 1u);
-                    mma_tf32(tmem_base, a_lo, b_hi, idesc, 1u);
+            const uint64_t a_hi = smem_desc_mn(base), a_lo = smem_desc_mn(base + A_BYTES);
+            const uint64_t b_hi = smem_desc_mn(base + 2 * A_BYTES), b_lo = smem_desc_mn(base + 2 * A_BYTES + B_BYTES);
+            // the next group of 8 rows is 1024 bytes = 64 descriptor units further on; a full block is unrolled so that
+            // the issuing thread spends few instructions between two MMAs
+            if (nks == BK / 8 && a.passes > 1) {
+#pragma unroll
+                for (int ks = 0; ks < BK / 8; ++ks) {
+                    mma_tf32(tmem_base, a_hi + 64 * ks, b_hi + 64 * ks, idesc, ks == 0 ? (kb != 0 ? 1u : 0u) : 1u);
+                    mma_tf32(tmem_base, a_hi + 64 * ks, b_lo + 64 * ks, idesc, 1u);
+                    mma_tf32(tmem_base, a_lo + 64 * ks, b_hi + 64 * ks, idesc, 1u);
+                }
+            } else {
+                for (int ks = 0; ks < nks; ++ks) {
+                    const uint64_t adv = (uint64_t)(64 * ks);
+                    mma_tf32(tmem_base, a_hi + adv, b_hi + adv, idesc, (kb | ks) != 0 ? 1u : 0u);
+                    if (a.passes > 1) {
+                        mma_tf32(tmem_base, a_hi + adv, b_lo + adv, idesc, 1u);
+                        mma_tf32(tmem_base, a_lo + adv, b_hi + adv, idesc, 1u);
+                    }
                 }
             }
             mma_commit(empty(stage));
