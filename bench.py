@@ -30,8 +30,8 @@ UNIT = "epochs/s"
 # capture summarised under profiles/; keyed by (workload, profile entry).  A kernel changed since its capture
 # has no entry (reported as null).
 NCU_TRAFFIC = {
-    # spmm_items_kernel (76.8 MB read + 32.9 MB written) + spmm_finish_kernel (14.9 MB read), profiles/spmm_items_c2.md
-    ("c2", "spmm_fwd_l0"): 124.6e6,
+    # spmm_items_kernel (76.8 MB read + 33.6 MB written) + spmm_finish_kernel (14.9 MB read), profiles/spmm_items_c2.md
+    ("c2", "spmm_fwd_l0"): 125.3e6,
 }
 
 
@@ -215,6 +215,7 @@ def main():
     ap.add_argument("--K", type=int, default=8)
     ap.add_argument("--gemm-mode", type=int, default=0)
     ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--zeta-mode", type=int, default=0, help="1: literal pairwise importance weights (O(n^2 F) per subgraph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernels", action="store_true", help="also print the per-kernel table to stderr")
     args = ap.parse_args()
@@ -250,7 +251,7 @@ def main():
     # Replicas only: every rank runs the whole K-subgraph job on its own GPU (no collective on the data path).
     w = make_workload(args.workload, **args.wl_kw)
     theta = glorot_params(w.dims, np.random.default_rng(0))
-    g = pkg.from_workload(w, theta, gemm_mode=args.gemm_mode, flags=args.flags)
+    g = pkg.from_workload(w, theta, gemm_mode=args.gemm_mode, flags=args.flags, zeta_mode=args.zeta_mode)
 
     def barrier():
         torch.cuda.synchronize()

@@ -33,6 +33,8 @@ struct Plan {
     int32_t maxld = 0;
     std::vector<RowSpan> tiles, chunks, dw_chunks, core_spans;
     std::vector<int32_t> chunk_ptr, dw_chunk_ptr;   // [K+1]
+    std::vector<int64_t> pair_ptr;    // [K+1] tiles of pairs per subgraph (zeta_mode 1), else empty
+    size_t o_pair_ptr = 0, o_pair_partial = 0;
     int64_t dw_partial = 0;           // floats per chunk
     bool agg_first0 = false;          // layer 0 aggregates before it transforms
     size_t o_P = 0;                   // A~ H^(0)  [Np x ld0], only with agg_first0
@@ -59,8 +61,13 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         if (cfg->dims[l] < 1) { err = "layer size must be positive"; return GAD_ERR_ARG; }
     if (!(cfg->dropout >= 0.f && cfg->dropout < 1.f)) { err = "dropout must be in [0,1)"; return GAD_ERR_ARG; }
     if (cfg->gemm_mode != 0 && cfg->gemm_mode != 1) { err = "gemm_mode must be 0 or 1"; return GAD_ERR_ARG; }
-    if (cfg->zeta_mode == 1) { err = "zeta_mode 1 (pairwise form) is not implemented"; return GAD_ERR_UNSUPPORTED; }
-    if (cfg->zeta_mode != 0) { err = "zeta_mode must be 0 or 1"; return GAD_ERR_ARG; }
+    if (cfg->zeta_mode != 0 && cfg->zeta_mode != 1) { err = "zeta_mode must be 0 or 1"; return GAD_ERR_ARG; }
+    if (cfg->zeta_mode == 1)   // O(n'^2 F_0) pairs per subgraph
+        for (int32_t k = 0; k < K; ++k)
+            if (sub_off[k + 1] - sub_off[k] > kZetaPairMaxRows) {
+                err = "zeta_mode 1 (pairwise form) takes subgraphs of at most " + std::to_string(kZetaPairMaxRows) + " rows";
+                return GAD_ERR_UNSUPPORTED;
+            }
     if (!(cfg->beta > 0.f)) { err = "beta must be positive"; return GAD_ERR_ARG; }
     p.n = n; p.K = K; p.L = cfg->L; p.nnz = nnz; p.Np = sub_off[K]; p.slots = slots;
     p.dims.assign(cfg->dims, cfg->dims + cfg->L + 1);
@@ -147,6 +154,12 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     }
     p.o_counters = take(cur, 4 * (size_t)(1 + 2 * K));
     if (p.agg_first0) p.o_P = take(cur, 4 * Np * (size_t)p.ld[0]);
+    if (cfg->zeta_mode == 1) {
+        p.pair_ptr.assign(K + 1, 0);
+        for (int32_t k = 0; k < K; ++k) p.pair_ptr[k + 1] = p.pair_ptr[k] + zeta_pair_tiles(sub_off[k + 1] - sub_off[k]);
+        p.o_pair_ptr = take(cur, 8 * (size_t)(K + 1));
+        p.o_pair_partial = take(cur, 8 * (size_t)p.pair_ptr[K]);
+    }
     p.bytes = cur;
     return GAD_OK;
 }
@@ -305,6 +318,16 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
 
 int zeta_pass(gad_ctx* ctx, cudaStream_t s) {
     const Plan& p = ctx->p;
+    if (ctx->cfg.zeta_mode == 1) {
+        const double pairs = 64.0 * 64.0 * (double)p.pair_ptr[p.K];
+        GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 1), 3.0 * pairs * p.dims[0], [&] {
+            return launch_zeta_pair(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<int32_t>(p.o_sub_off),
+                                    ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_pair_ptr), p.pair_ptr[p.K], p.K, ctx->cfg.beta,
+                                    ctx->at<double>(p.o_pair_partial), ctx->at<unsigned>(p.o_counters) + 1 + p.K,
+                                    ctx->at<double>(p.o_zeta), s);
+        });
+        return GAD_OK;
+    }
     GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 1), 4.0 * p.Np * p.dims[0], [&] {
         return launch_zeta(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
                            (int)p.chunks.size(), ctx->at<int32_t>(p.o_chunk_ptr), ctx->at<int32_t>(p.o_sub_off),
@@ -530,7 +553,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         (rc = upload(ctx, p.o_deg_sq, deg_sq)) || (rc = upload(ctx, p.o_inv_ntrain, inv_ntrain)) ||
         (rc = upload(ctx, p.o_tiles, p.tiles)) || (rc = upload(ctx, p.o_chunks, p.chunks)) ||
         (rc = upload(ctx, p.o_chunk_ptr, p.chunk_ptr)) || (rc = upload(ctx, p.o_dw_chunks, p.dw_chunks)) ||
-        (rc = upload(ctx, p.o_dw_chunk_ptr, p.dw_chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)))
+        (rc = upload(ctx, p.o_dw_chunk_ptr, p.dw_chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)) ||
+        (rc = upload(ctx, p.o_pair_ptr, p.pair_ptr)))
         return rc;
     // features: graph order -> staging -> store-row order with zero pad columns
     GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage, X, 4 * (size_t)g->n * p.dims[0], cudaMemcpyHostToDevice, ctx->stream));

@@ -181,6 +181,14 @@ cudaError_t launch_zeta(const float* X, int ld, int F, const int32_t* deg, const
                         const int32_t* chunk_ptr, const int32_t* sub_off, const int64_t* deg_sum, const int64_t* deg_sq,
                         float beta, double* partial, unsigned* counters, double* zeta, cudaStream_t s);
 
+// zeta_k in the literal pairwise form, sum_{i<j} p_i p_j / (|x_i - x_j| + beta), 64 x 64 tiles of pairs (one CTA each,
+// pair_ptr[k] = first tile of subgraph k); counters: one per subgraph; partial: one double per tile.
+constexpr int64_t kZetaPairMaxRows = 32768;
+int64_t zeta_pair_tiles(int64_t rows);
+cudaError_t launch_zeta_pair(const float* X, int ld, int F, const int32_t* deg, const int32_t* sub_off, const int64_t* deg_sum,
+                             const int64_t* pair_ptr, int64_t npairs, int K, float beta, double* partial, unsigned* counters,
+                             double* zeta, cudaStream_t s);
+
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, cudaStream_t s);
 cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s);

@@ -40,7 +40,7 @@ def make_pair(case, dims, seed=0, X=None, **kw):
     cp, cn = flat(core)
     hp, hn = flat(halo)
     st = orc().Store(n, rowptr, col, cp, cn, hp, hn, weights=w)
-    okw = {k: v for k, v in kw.items() if k in ("lr", "dropout", "seed", "beta", "weighted")}
+    okw = {k: v for k, v in kw.items() if k in ("lr", "dropout", "seed", "beta", "weighted", "zeta_mode")}
     ref = orc().Model(st, X, y, split, dims, theta, **okw)
     g = pkg().Gad(n, rowptr, col, cp, cn, hp, hn, X, y, split, dims, init_params=theta, weights=w, **kw)
     return g, ref, st
@@ -177,6 +177,34 @@ def test_importance_weights_and_consensus(tiny):
         assert rel_err(g.get_params(0), first) <= 1e-6              # a second consensus changes nothing
     with pkg().from_workload(tiny, theta, weighted=False) as g:
         assert np.allclose(g.subgraph_weights()[1], 0.25)
+
+
+@pytest.mark.parametrize("seed,n,K,F", [(0, 70, 3, 6), (1, 700, 2, 37), (2, 3000, 3, 64), (3, 1500, 1, 130)])
+def test_pairwise_importance_weights(seed, n, K, F):
+    """zeta_mode 1: the printed formula taken literally, sum_{i<j} p_i p_j / (|x_i - x_j| + beta), over tiles of
+    64 x 64 pairs with ragged last tiles, against the oracle's double loop; then an epoch whose consensus uses them."""
+    case = small_random_case(seed, n=n, K=K, p=min(0.15, 8.0 / n))
+    g, ref, st = make_pair(case, (F, 8, 3), seed, lr=0.1, zeta_mode=1)
+    with g:
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(zg - zr)) <= 2e-6 * np.max(zr)
+        assert np.max(np.abs(wg - wr)) <= 2e-6
+        check_epoch(g, ref)
+
+
+def test_pairwise_importance_of_identical_points_is_the_closed_form():
+    """All features equal: every distance is 0 and zeta = S / beta with S = (1 - sum p^2) / 2."""
+    case = small_random_case(5, n=300, K=2, p=0.05)
+    n = case[0]
+    X = np.ones((n, 12), dtype=np.float32) * 0.75
+    g, ref, st = make_pair(case, (12, 5, 3), 5, X=X, zeta_mode=1, beta=0.5)
+    with g:
+        zg, _ = g.subgraph_weights()
+    for k in range(st.K):
+        d = st.deg[st.sub_off[k]:st.sub_off[k + 1]].astype(np.float64)
+        p = d / d.sum() if d.sum() > 0 else np.full(len(d), 1.0 / len(d))
+        assert abs(zg[k] - 0.5 * (1.0 - np.sum(p * p)) / 0.5) <= 1e-6
 
 
 def test_large_feature_offsets_do_not_break_the_variance_statistics():
