@@ -41,7 +41,7 @@ struct Plan {
     size_t o_counters = 0;            // arrival counters: [loss | K column sums | K zeta]
     size_t bytes = 0;
     // offsets into the workspace
-    size_t o_rowptr, o_ecv, o_perm, o_parts, o_fin, o_items, o_trowptr, o_tecv, o_tperm, o_tparts, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
+    size_t o_rowptr, o_ecv, o_fin, o_items, o_trowptr, o_tecv, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
         o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_dw_chunks, o_dw_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
         o_dw_partial, o_cs_partial, o_loss_partial, o_zeta_partial, o_zeta, o_loss, o_flags, o_zeta_f, o_w_f, o_stage,
         o_stage_lab, o_stage2, o_stage_lab2;
@@ -120,10 +120,10 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_rowptr = take(cur, 8 * (Np + 1)); p.o_ecv = take(cur, 8 * (size_t)nnz);
     // work lists: one part per scratch slot, at most one cut row per kMinPart entries
     const size_t max_parts = (size_t)(slots + 1), max_fin = (size_t)(nnz / kMinPart + 1);
-    p.o_perm = take(cur, 4 * Np); p.o_parts = take(cur, 16 * max_parts); p.o_fin = take(cur, 16 * max_fin);
+    p.o_fin = take(cur, 16 * max_fin);
     p.o_items = take(cur, 16 * (Np + max_parts));
     p.o_trowptr = take(cur, 8 * (Np + 1)); p.o_tecv = take(cur, 8 * (size_t)nnz);
-    p.o_tperm = take(cur, 4 * Np); p.o_tparts = take(cur, 16 * max_parts); p.o_tfin = take(cur, 16 * max_fin);
+    p.o_tfin = take(cur, 16 * max_fin);
     p.o_titems = take(cur, 16 * (Np + max_parts));
     p.o_sub_off = take(cur, 4 * (size_t)(K + 1)); p.o_gid = take(cur, 4 * Np); p.o_deg = take(cur, 4 * Np);
     p.o_label = take(cur, 4 * Np); p.o_train = take(cur, Np);
@@ -416,7 +416,7 @@ uint64_t host_mix64(uint64_t z) {
 
 int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col,
                   const std::vector<float>& val,
-                  size_t o_rowptr, size_t o_ecv, size_t o_perm, size_t o_parts, size_t o_fin, size_t o_items, SparseDev& out) {
+                  size_t o_rowptr, size_t o_ecv, size_t o_fin, size_t o_items, SparseDev& out) {
     const Plan& p = ctx->p;
     std::vector<uint2> ecv(col.size());
     for (size_t e = 0; e < col.size(); ++e) {
@@ -427,12 +427,8 @@ int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::
     RowWork work;
     bin_rows(rowptr, sub_off, work);
     if (work.slots > p.slots) return fail(ctx, GAD_ERR_OOM, "SpMM scratch slots exceed the planned count");
-    const std::vector<int32_t>& perm = work.perm;
     GAD_CK(cudaMemcpyAsync(ctx->ws + o_rowptr, rowptr.data(), 8 * rowptr.size(), cudaMemcpyHostToDevice, ctx->stream));
     if (!ecv.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_ecv, ecv.data(), 8 * ecv.size(), cudaMemcpyHostToDevice, ctx->stream));
-    if (!perm.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_perm, perm.data(), 4 * perm.size(), cudaMemcpyHostToDevice, ctx->stream));
-    if (!work.parts.empty())
-        GAD_CK(cudaMemcpyAsync(ctx->ws + o_parts, work.parts.data(), 16 * work.parts.size(), cudaMemcpyHostToDevice, ctx->stream));
     if (!work.fin.empty())
         GAD_CK(cudaMemcpyAsync(ctx->ws + o_fin, work.fin.data(), 16 * work.fin.size(), cudaMemcpyHostToDevice, ctx->stream));
     if (!work.items.empty())
@@ -440,15 +436,11 @@ int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::
     GAD_CK(cudaStreamSynchronize(ctx->stream));  // the host vectors above go out of scope
     out.rowptr = ctx->at<int64_t>(o_rowptr);
     out.ecv = ctx->at<uint2>(o_ecv);
-    out.perm = ctx->at<int32_t>(o_perm);
-    out.parts = ctx->at<int4>(o_parts);
     out.fin = ctx->at<int4>(o_fin);
     out.items = ctx->at<int4>(o_items);
     out.nitems = (int32_t)work.items.size();
     out.nrows = (int64_t)rowptr.size() - 1;
     out.scratch = ctx->at<float>(p.o_spmm_scratch);
-    out.nperm = (int32_t)perm.size();
-    out.nparts = (int32_t)work.parts.size();
     out.nfin = (int32_t)work.fin.size();
     return GAD_OK;
 }
@@ -522,10 +514,10 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->sub_off = st.sub_off;
     ctx->gid = st.gid;
 
-    rc = upload_sparse(ctx, st.sub_off, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_perm, p.o_parts, p.o_fin, p.o_items, ctx->A);
+    rc = upload_sparse(ctx, st.sub_off, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_fin, p.o_items, ctx->A);
     if (rc != GAD_OK) return rc;
     if (!st.symmetric) {
-        rc = upload_sparse(ctx, st.sub_off, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tperm, p.o_tparts, p.o_tfin, p.o_titems, ctx->At);
+        rc = upload_sparse(ctx, st.sub_off, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tfin, p.o_titems, ctx->At);
         if (rc != GAD_OK) return rc;
     }
     // per-row labels and loss mask, per-subgraph degree sums and training counts

@@ -41,16 +41,15 @@ int build_store(const gad_csr* g, const gad_partition* part, bool values, HostSt
 // Sizes only (for gad_workspace_bytes): rows, entries, and the SpMM scratch slots of the worse orientation.
 int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_t* nnz, int64_t* slots, std::string& err);
 
-// Work lists of the SpMM launch.  Rows of at most `part_entries` entries go to `perm` (one warp, or one lane
-// group, per row), binned by floor(log2(entries)), heaviest bin first, ascending row id inside a bin.  Longer rows
-// are cut into parts of `part_entries` entries, one warp per part: parts = {row, first entry relative to the row,
-// entries, scratch slot}; fin = {row, first scratch slot, slots, 0} for every row that was cut.  The part length
-// starts at kMinPart and doubles (up to kMaxPart) until the cut rows need at most one scratch slot per two store rows;
-// a row that would still need more than kMaxSlotsPerRow parts gets longer parts of its own.
-// items = every part and every uncut row as {row, low 32 bits of the first entry's position in the store,
-// (high bits << 16) | entries, scratch slot or -1 for an uncut row}, subgraph by subgraph and longest first inside a
-// subgraph (same binning): the work list of
-// the one-warp-per-item kernel that serves operands of more than 64 columns.
+// Work lists of the SpMM launch (host side).  A row of at most `part_entries` entries is one item; a longer row is
+// cut into parts of `part_entries` entries, each an item with a scratch slot of its own, and gets an entry
+// fin = {row, first scratch slot, slots, 0}.  The part length starts at kMinPart and doubles (up to kMaxPart)
+// until the cut rows need at most one scratch slot per two store rows; a row that would still need more than
+// kMaxSlotsPerRow parts gets longer parts of its own.
+// items = {row, low 32 bits of the first entry's position in the store, (high bits << 16) | entries, scratch slot
+// or -1 for an uncut row}, subgraph by subgraph and inside a subgraph binned by floor(log2(entries)), longest bin
+// first, ascending row inside a bin.  `perm` (uncut rows in that order) and `parts` are the intermediate lists the
+// items are built from.
 constexpr int64_t kMinPart = 64, kMaxPart = 1024, kMaxSlotsPerRow = 32;
 struct RowWork {
     std::vector<int32_t> perm;
@@ -66,14 +65,12 @@ int64_t count_slots(const std::vector<int64_t>& rowptr);
 // Device views
 // ---------------------------------------------------------------------------------------------
 struct SparseDev {
-    const int64_t* rowptr = nullptr;  // [Np+1]
+    const int64_t* rowptr = nullptr;  // [Np+1] (kept for the accessors; the kernels read the work list)
     const uint2* ecv = nullptr;       // [nnz] packed (column, value bits)
-    const int32_t* perm = nullptr;    // binned short rows
-    const int4* parts = nullptr;      // parts of the long rows
     const int4* fin = nullptr;        // rows made of several parts
     const int4* items = nullptr;      // parts and uncut rows together, longest first
     float* scratch = nullptr;         // [slots x leading dimension of the output] partial rows
-    int32_t nperm = 0, nparts = 0, nfin = 0, nitems = 0;
+    int32_t nfin = 0, nitems = 0;
     int64_t nrows = 0;                // rows (and columns) of the store
 };
 
