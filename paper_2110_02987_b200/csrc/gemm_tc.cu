@@ -39,7 +39,8 @@ constexpr int EPI_WARP0 = 2 + SPLIT_WARPS;                // first epilogue warp
 constexpr int ROWS_THREADS = 32 * (EPI_WARP0 + EPI_WARPS);
 constexpr int SMEM_BYTES_ROWS = SMEM_BYTES + EPI_BYTES;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
-constexpr int TMEM_COLS = 2 * BN_MAX;
+constexpr int ACC_COLS = 256;                             // widest output tile of the rows kernel (one MMA: N <= 256)
+constexpr int TMEM_COLS = 2 * ACC_COLS;                   // two accumulators: all 512 columns of the SM's tensor memory
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -217,7 +218,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
             if (!(ok = mbar_wait(tempty(acc), acc_phase ^ 1u, abort_flag, a.err, 2))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t d = tmem_base + (uint32_t)(acc * BN_MAX);
+            const uint32_t d = tmem_base + (uint32_t)(acc * ACC_COLS);
             for (int kb = 0; kb < nkb; ++kb) {
                 if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 3))) break;
                 if (!(ok = mbar_wait(xfull(stage), phase, abort_flag, a.err, 4))) break;
@@ -324,7 +325,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float4 bias4 = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (a.mode == 2 && n < a.ldc) bias4 = load_bias(a.act, sp.k, n);
                 uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN_MAX + c0), v);
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS + c0), v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int j = 0; j < 32; ++j) tr[lane * 33 + j] = __uint_as_float(v[j]);
@@ -586,7 +587,10 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
-int tc_bn_for(int n_cols) { return n_cols <= 16 ? 16 : n_cols <= 32 ? 32 : n_cols <= 64 ? 64 : 128; }
+// Output columns per tile: one MMA covers up to 256, and an M = 128, K = 8 TF32 MMA costs about the same for any N, so
+// the widest tile that the ring still holds twice is the cheapest.  The weight-gradient kernel stays at 128.
+int tc_bn_for(int n_cols) { return n_cols <= 16 ? 16 : n_cols <= 32 ? 32 : n_cols <= 64 ? 64 : n_cols <= 128 ? 128 : 256; }
+static int tn_bn_for(int n_cols) { return tc_bn_for(n_cols) < 128 ? tc_bn_for(n_cols) : 128; }
 
 // fp32 tensor [outer (z)] x [rows (y)] x [inner (x)], box = 32 floats x box_rows x 1, zero fill outside.  K-major
 // operand tiles use the 128-byte swizzle of 16-byte units; MN-major TF32 tiles need the 128-byte swizzle of
@@ -649,7 +653,7 @@ cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, in
         configured = true;
     }
     TnArgs a;
-    a.chunks = chunks; a.BN = tc_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;
+    a.chunks = chunks; a.BN = tn_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;
     a.partial = partial; a.pstride_chunk = (long long)M * ldw; a.passes = passes; a.err = err;
     const unsigned grid = (unsigned)((long long)nchunks * a.ntm * a.ntn);
     gemm_tn_tc_kernel<<<grid, TN_THREADS, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapH), *reinterpret_cast<const CUtensorMap*>(mapZ), a);
