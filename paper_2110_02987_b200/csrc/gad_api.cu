@@ -95,9 +95,12 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     int64_t R = round_up(std::max<int64_t>(1, (p.Np + target - 1) / target), 32);
     R = std::min<int64_t>(std::max<int64_t>(R, 128), 16384);
     // The weight gradient has a long reduction per output tile, so it gets longer chunks: about one CTA per SM (a
-    // single wave: every CTA pays the pipeline fill once) over the layer with the most output tiles (128 x 128 each).
+    // single wave: every CTA pays the pipeline fill once) over the layer with the most output tiles (128 rows x up to 256 columns each).
     int64_t max_tiles = 1;
-    for (const Layer& y : p.layers) max_tiles = std::max<int64_t>(max_tiles, ((y.fi + 127) / 128) * (int64_t)((y.ldw + 127) / 128));
+    for (const Layer& y : p.layers) {
+        const int bn = tc_bn_for(y.fo);
+        max_tiles = std::max<int64_t>(max_tiles, ((y.fi + 127) / 128) * (int64_t)((y.ldw + bn - 1) / bn));
+    }
     int64_t Rdw = round_up(std::max<int64_t>(1, p.Np * max_tiles / std::max<int64_t>(74, 148 - K)), 32);
     // (not longer than 4096 rows: the CTAs that share a chunk then stay close enough to share it in L2)
     Rdw = std::min<int64_t>(std::max<int64_t>(Rdw, 256), 4096);

@@ -424,24 +424,29 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
     uint8_t* sm = smem_raw + pad;
     const uint32_t sm_addr = raw_addr + pad;
-    const uint32_t bars = sm_addr + STAGES * STAGE_BYTES;
+    // a stage holds the H tile and its low half (16 KiB each) and the dZ tile of BN columns with its low half
+    const int nb_blocks = (a.BN + 31) / 32;                    // 32-value blocks of the B tile
+    const uint32_t b_bytes = (uint32_t)nb_blocks * 4096u;
+    const uint32_t stage_bytes = 2u * A_BYTES + 2u * b_bytes;
+    const int nst = min(MAX_STAGES, (int)(RING_BYTES / stage_bytes));
+    const uint32_t bars = sm_addr + RING_BYTES;
     auto full = [&](int s) { return bars + 8u * s; };
-    auto xfull = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto empty = [&](int s) { return bars + 8u * (2 * STAGES + s); };
-    const uint32_t tfull = bars + 8u * (3 * STAGES);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * STAGE_BYTES + 8 * (3 * STAGES + 4));
+    auto xfull = [&](int s) { return bars + 8u * (MAX_STAGES + s); };
+    auto empty = [&](int s) { return bars + 8u * (2 * MAX_STAGES + s); };
+    const uint32_t tfull = bars + 8u * (3 * MAX_STAGES);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + RING_BYTES + 8 * (3 * MAX_STAGES + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
     constexpr int NSPLIT = TN_THREADS - 64;   // threads of warps 2..15
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), NSPLIT); mbar_init(empty(s), 1); }
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), NSPLIT); mbar_init(empty(s), 1); }
         mbar_init(tfull, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN_MAX) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(ACC_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -454,7 +459,6 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     const int tile = blockIdx.x % tiles_per_chunk;
     const int m0 = (tile / a.ntn) * BM, n0 = (tile % a.ntn) * a.BN;
     const int nkb = (c.nrows + BK - 1) / BK;
-    const int nb_blocks = (a.BN + 31) / 32;                    // 32-value blocks of the B tile
     const uint32_t tx_bytes = (uint32_t)(4 + nb_blocks) * 4096u;
     bool ok = true;
 
@@ -464,11 +468,11 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
         for (int kb = 0; kb < nkb; ++kb) {
             if (!(ok = mbar_wait(empty(stage), phase ^ 1u, abort_flag, a.err, 11))) break;
             mbar_expect_tx(full(stage), tx_bytes);
-            const uint32_t base = sm_addr + stage * STAGE_BYTES;
+            const uint32_t base = sm_addr + stage * stage_bytes;
             const int r = c.row0 + kb * BK;
             for (int j = 0; j < 4; ++j) tma_load_2d(base + j * 4096, &tmH, m0 + 32 * j, r, full(stage));
             for (int j = 0; j < nb_blocks; ++j) tma_load_2d(base + 2 * A_BYTES + j * 4096, &tmZ, n0 + 32 * j, r, full(stage));
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
     } else if (warp == 1 && lane == 0) {
         int stage = 0;
@@ -478,10 +482,10 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 13))) break;
             if (!(ok = mbar_wait(xfull(stage), phase, abort_flag, a.err, 14))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t base = sm_addr + stage * STAGE_BYTES;
+            const uint32_t base = sm_addr + stage * stage_bytes;
             const int nks = min(BK / 8, (c.nrows - kb * BK + 7) / 8);
             const uint64_t a_hi = smem_desc_mn(base), a_lo = smem_desc_mn(base + A_BYTES);
-            const uint64_t b_hi = smem_desc_mn(base + 2 * A_BYTES), b_lo = smem_desc_mn(base + 2 * A_BYTES + B_BYTES);
+            const uint64_t b_hi = smem_desc_mn(base + 2 * A_BYTES), b_lo = smem_desc_mn(base + 2 * A_BYTES + b_bytes);
             // the next group of 8 rows is 1024 bytes = 64 descriptor units further on; a full block is unrolled so that
             // the issuing thread spends few instructions between two MMAs
             if (nks == BK / 8 && a.passes > 1) {
@@ -502,7 +506,7 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
                 }
             }
             mma_commit(empty(stage));
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
         if (ok) mma_commit(tfull);
     } else if (warp >= 2) {
@@ -515,13 +519,13 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 15))) break;
             const int rows_valid = min(BK, c.nrows - kb * BK);
             if (a.passes > 1 || rows_valid < BK) {
-                uint8_t* sb = sm + stage * STAGE_BYTES;
+                uint8_t* sb = sm + stage * stage_bytes;
                 for (int i = tt; i < nf4; i += NSPLIT) {
                     const int blk = i >> 8, in = i & 255;                         // block of 32 values, float4 inside it
                     const int row = in >> 3;                                      // 8 float4 per 128-byte row
                     const int byte_off = (blk < 4 ? blk * 4096 : 2 * A_BYTES + (blk - 4) * 4096) + in * 16;
                     float4* hi = reinterpret_cast<float4*>(sb + byte_off);
-                    float4* lo = reinterpret_cast<float4*>(sb + byte_off + (blk < 4 ? A_BYTES : B_BYTES));
+                    float4* lo = reinterpret_cast<float4*>(sb + byte_off + (blk < 4 ? (uint32_t)A_BYTES : b_bytes));
                     float4 v = *hi;
                     if (row >= rows_valid) v = make_float4(0.f, 0.f, 0.f, 0.f);
                     float4 h, l;
@@ -535,7 +539,7 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             mbar_arrive(xfull(stage));
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
     }
     // epilogue by warps 8..15 (two per quarter of the tensor-memory lanes, alternate blocks of 32 columns) once
@@ -566,7 +570,7 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     __syncthreads();
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(BN_MAX) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(ACC_COLS) : "memory");
     }
 }
 
@@ -588,9 +592,8 @@ EncodeTiledFn encode_fn() {
 }  // namespace
 
 // Output columns per tile: one MMA covers up to 256, and an M = 128, K = 8 TF32 MMA costs about the same for any N, so
-// the widest tile that the ring still holds twice is the cheapest.  The weight-gradient kernel stays at 128.
+// the widest tile that the ring still holds twice is the cheapest.
 int tc_bn_for(int n_cols) { return n_cols <= 16 ? 16 : n_cols <= 32 ? 32 : n_cols <= 64 ? 64 : n_cols <= 128 ? 128 : 256; }
-static int tn_bn_for(int n_cols) { return tc_bn_for(n_cols) < 128 ? tc_bn_for(n_cols) : 128; }
 
 // fp32 tensor [outer (z)] x [rows (y)] x [inner (x)], box = 32 floats x box_rows x 1, zero fill outside.  K-major
 // operand tiles use the 128-byte swizzle of 16-byte units; MN-major TF32 tiles need the 128-byte swizzle of
@@ -653,7 +656,7 @@ cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, in
         configured = true;
     }
     TnArgs a;
-    a.chunks = chunks; a.BN = tn_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;
+    a.chunks = chunks; a.BN = tc_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;
     a.partial = partial; a.pstride_chunk = (long long)M * ldw; a.passes = passes; a.err = err;
     const unsigned grid = (unsigned)((long long)nchunks * a.ntm * a.ntn);
     gemm_tn_tc_kernel<<<grid, TN_THREADS, SMEM_BYTES, s>>>(*reinterpret_cast<const CUtensorMap*>(mapH), *reinterpret_cast<const CUtensorMap*>(mapZ), a);
