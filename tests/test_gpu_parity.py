@@ -239,6 +239,61 @@ def test_single_replica_and_degenerate_subgraphs():
         assert zg[1] == 0.0 and wg[1] == 0.0
 
 
+def test_many_subgraphs_and_a_deep_network():
+    """K = 40 small subgraphs (several row tiles and chunks end inside a subgraph of a few rows) and L = 5 layers."""
+    case = small_random_case(31, n=600, K=40, p=0.02)
+    g, ref, st = make_pair(case, (20, 24, 40, 16, 12, 5), 31, lr=0.05)
+    with g:
+        check_store(g, st)
+        check_epoch(g, ref)
+        check_epoch(g, ref)
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("dims", [(24, 40, 6), (100, 20, 6)])
+def test_dropout_through_both_layer_orders_and_transform_paths(flags, dims):
+    """Dropout after the ReLU when layer 0 aggregates first (mask applied in the transform's epilogue: tensor-core
+    kernel, or the FP32-ALU one with flags bit 0) and when it transforms first (mask applied in the SpMM epilogue)."""
+    case = small_random_case(33, n=500, K=3, p=0.02)
+    g, ref, st = make_pair(case, dims, 33, lr=0.05, dropout=0.4, flags=flags)
+    with g:
+        for _ in range(2):
+            lg, lr = g.train_epoch(), ref.train_epoch()
+            assert np.max(np.abs(lg - lr)) <= 1e-4
+            h1g, h1r = g.get_activation(1), ref.activation(1)
+            assert np.array_equal(h1g == 0, h1r == 0)
+            assert rel_err(h1g, h1r) <= TOL
+        for k in range(g.K):
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+
+
+def test_wide_input_aggregated_first():
+    """F_0 = 1100 > 1024 aggregated first (two column slabs in the SpMM, a 1100-deep reduction in the transform)."""
+    case = small_random_case(35, n=400, K=2, p=0.03)
+    g, ref, st = make_pair(case, (1100, 600, 4), 35, lr=0.02)
+    with g:
+        check_epoch(g, ref)
+
+
+def test_pairwise_importance_with_degenerate_subgraphs():
+    """zeta_mode 1 with an empty subgraph (zeta 0), a single-row subgraph (no pair: zeta 0) and a subgraph without edges
+    (uniform p)."""
+    n = 40
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    src = np.array([0, 1, 1, 2, 2, 3], dtype=np.int64)
+    dst = np.array([1, 0, 2, 1, 3, 2], dtype=np.int32)
+    np.cumsum(np.bincount(src, minlength=n), out=rowptr[1:])
+    core = [np.arange(0, 10, dtype=np.int32), np.empty(0, np.int32), np.array([10], dtype=np.int32), np.arange(20, 40, dtype=np.int32)]
+    halo = [np.empty(0, np.int32)] * 4
+    g, ref, st = make_pair((n, rowptr, dst, None, core, halo), (5, 4, 3), 37, zeta_mode=1)
+    with g:
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert zg[1] == 0.0 and zg[2] == 0.0
+        assert np.max(np.abs(zg - zr)) <= 1e-6 and np.max(np.abs(wg - wr)) <= 1e-6
+        check_epoch(g, ref)
+
+
 def test_isolated_nodes_and_no_edges():
     n = 40
     rowptr = np.zeros(n + 1, dtype=np.int64)
