@@ -39,6 +39,11 @@ struct Plan {
     bool agg_first0 = false;          // layer 0 aggregates before it transforms
     size_t o_P = 0;                   // A~ H^(0)  [Np x ld0], only with agg_first0
     size_t o_counters = 0;            // arrival counters: [loss | K column sums | K zeta]
+    // layers of at most 16 output columns take the streaming FP32 kernels (flag bit 2 switches them off)
+    std::vector<uint8_t> narrow;      // [L]
+    std::vector<RowSpan> nchunks;     // their row chunks: about three CTAs per SM, never across subgraphs
+    std::vector<int32_t> nchunk_ptr;  // [K+1]
+    size_t o_nchunks = 0, o_nchunk_ptr = 0, o_nw_partial = 0;
     size_t bytes = 0;
     // offsets into the workspace
     size_t o_rowptr, o_ecv, o_fin, o_items, o_trowptr, o_tecv, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
@@ -157,6 +162,26 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     }
     p.o_counters = take(cur, 4 * (size_t)(1 + 2 * K));
     if (p.agg_first0) p.o_P = take(cur, 4 * Np * (size_t)p.ld[0]);
+    p.narrow.assign(p.L, 0);
+    int64_t narrow_partial = 0;
+    for (int l = 0; l < p.L; ++l) {
+        const Layer& y = p.layers[l];
+        const bool agg_first = l == 0 && p.agg_first0;
+        p.narrow[l] = (cfg->flags & 5) == 0 && !agg_first && narrow_supported(y.ldi, y.ldo);
+        if (p.narrow[l]) narrow_partial = std::max(narrow_partial, (int64_t)y.fi * y.ldw);
+    }
+    if (narrow_partial > 0) {
+        const int64_t Rn = std::max<int64_t>(64, round_up((p.Np + 443) / 444, 32));
+        p.nchunk_ptr.assign(K + 1, 0);
+        for (int32_t k = 0; k < K; ++k) {
+            for (int64_t r = sub_off[k]; r < sub_off[k + 1]; r += Rn)
+                p.nchunks.push_back(RowSpan{(int32_t)r, (int32_t)std::min<int64_t>(Rn, sub_off[k + 1] - r), k, 0});
+            p.nchunk_ptr[k + 1] = (int32_t)p.nchunks.size();
+        }
+        p.o_nchunks = take(cur, sizeof(RowSpan) * p.nchunks.size());
+        p.o_nchunk_ptr = take(cur, 4 * (size_t)(K + 1));
+        p.o_nw_partial = take(cur, 4 * p.nchunks.size() * (size_t)narrow_partial);
+    }
     if (cfg->zeta_mode == 1) {
         p.pair_ptr.assign(K + 1, 0);
         for (int32_t k = 0; k < K; ++k) p.pair_ptr[k + 1] = p.pair_ptr[k] + zeta_pair_tiles(sub_off[k + 1] - sub_off[k]);
@@ -304,8 +329,11 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
             });
             continue;
         }
-        if (split_pending) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
+        if (split_pending && !(ctx->use_tc && p.narrow[l])) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
         GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+            if (ctx->use_tc && p.narrow[l])
+                return launch_narrow_fwd(ctx->H(l), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, ctx->at<RowSpan>(p.o_nchunks),
+                                         (int)p.nchunks.size(), Z, y.ldo, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
             if (ctx->use_tc)
                 return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 0, passes, y.fi, y.fo, Z,
                                            y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr,
@@ -368,6 +396,20 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                     [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
+        if (l > 0 && ctx->use_tc && p.narrow[l]) {
+            // one pass over H^(l) and dZ gives both dW and dPre of the layer below (it writes G1: the column sums come first)
+            if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
+            GAD_RUN("gemm_dwdh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 8.0 * p.K * y.fi * y.fo, 4.0 * p.Np * y.fi * y.fo, [&] {
+                cudaError_t e = launch_narrow_bwd(ctx->H(l), y.ldi, y.fi, G2, y.ldo, params, p.pstride, y.w_int, y.ldw,
+                                                  ctx->at<RowSpan>(p.o_nchunks), (int)p.nchunks.size(), scale, G1,
+                                                  ctx->at<float>(p.o_nw_partial), (int64_t)y.fi * y.ldw,
+                                                  ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
+                if (e != cudaSuccess) return e;
+                return launch_reduce_chunks(ctx->at<float>(p.o_nw_partial), (int64_t)y.fi * y.ldw, ctx->at<int32_t>(p.o_nchunk_ptr), p.K,
+                                            grads, p.pstride, y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
+            });
+            continue;
+        }
         GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
             cudaError_t e =
                 ctx->use_tc ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
@@ -549,7 +591,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         (rc = upload(ctx, p.o_tiles, p.tiles)) || (rc = upload(ctx, p.o_chunks, p.chunks)) ||
         (rc = upload(ctx, p.o_chunk_ptr, p.chunk_ptr)) || (rc = upload(ctx, p.o_dw_chunks, p.dw_chunks)) ||
         (rc = upload(ctx, p.o_dw_chunk_ptr, p.dw_chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)) ||
-        (rc = upload(ctx, p.o_pair_ptr, p.pair_ptr)))
+        (rc = upload(ctx, p.o_pair_ptr, p.pair_ptr)) || (rc = upload(ctx, p.o_nchunks, p.nchunks)) ||
+        (rc = upload(ctx, p.o_nchunk_ptr, p.nchunk_ptr)))
         return rc;
     // features: graph order -> staging -> store-row order with zero pad columns
     GAD_CK(cudaMemcpyAsync(ctx->ws + p.o_stage, X, 4 * (size_t)g->n * p.dims[0], cudaMemcpyHostToDevice, ctx->stream));

@@ -1,0 +1,344 @@
+// Transforms of a layer with at most 16 output columns (a classifier layer: the paper's datasets have 3 .. 41
+// classes), on the FP32 ALUs.  With so few columns the product H W costs 2 * 16 flops per loaded value: the layer is
+// a stream over H^(l), bound by HBM, and a tensor-core tile (M = 128 at the price of any N) has nothing to offer.
+//
+//   forward    Z_l = H^(l) W_k^(l)                                   (the H.W of the forward equation, Section 3.3)
+//   backward   dW_k^(l) = H^(l)^T dZ_l   and   dPre_(l-1) = (dZ_l W_k^(l)^T) masked by H^(l) > 0, in ONE pass over
+//              H^(l) and dZ_l (chain rule through the forward equation)
+//
+// A CTA of four warps owns a run of rows of one subgraph (a chunk) and streams it through a three-stage ring in
+// shared memory: one thread issues bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) of the next
+// row blocks of H^(l) and dZ_l while the warps work on the current one.  A lane owns four columns of H^(l) (a warp a
+// slab of 128 columns, wider layers spread their slabs over the warps) and keeps its 4 x 16 block of W_k^(l), and in
+// the backward kernel of dW, in registers for the whole chunk.  Chunk results of dW are added per subgraph in chunk
+// order by reduce_chunks, so nothing depends on scheduling.  Every mbarrier wait is bounded: on a time-out the CTA
+// raises the error word and returns.
+#include <algorithm>
+
+#include "gad_internal.h"
+
+namespace gad {
+
+namespace {
+
+constexpr int kWarps = 4, kStages = 3;
+constexpr uint32_t kWaitLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_expect(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.b32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i)
+        if (bar_try(bar, parity)) return true;
+    return false;
+}
+// Contiguous global -> shared copy of `bytes` (a multiple of 16, both addresses 16-byte aligned).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Rows per ring stage: a stage holds 4096 floats of H^(l) per 128-column slab set.
+__host__ __device__ inline int block_rows(int nslab) { return 32 / nslab; }
+
+struct Ring {
+    uint32_t bar0;       // shared address of the first stage's mbarrier (8 bytes each)
+    const float* A;      // H^(l) rows of the chunk
+    const float* B;      // dZ_l rows of the chunk, or null
+    int lda, ldb, nrows, BR;
+    uint32_t a_addr, b_addr, stage_a_bytes, stage_b_bytes;
+    __device__ __forceinline__ void issue(int b) const {
+        const int s = b % kStages, nb = min(BR, nrows - b * BR);
+        const uint32_t ab = (uint32_t)nb * (uint32_t)lda * 4u, bb = B ? (uint32_t)nb * (uint32_t)ldb * 4u : 0u;
+        const uint32_t bar = bar0 + 8u * (uint32_t)s;
+        bar_expect(bar, ab + bb);
+        bulk_load(a_addr + s * stage_a_bytes, A + (long long)b * BR * lda, ab, bar);
+        if (B) bulk_load(b_addr + s * stage_b_bytes, B + (long long)b * BR * ldb, bb, bar);
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// backward: dW partial of the chunk, and dPre_(l-1) rows
+// ---------------------------------------------------------------------------------------------
+template <int NQ>
+__global__ void __launch_bounds__(32 * kWarps, 3)
+narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __restrict__ dZ, int ldz, const float* __restrict__ params,
+                  long long pstride, long long w_int, int ldw, const RowSpan* __restrict__ chunks, float scale, float* __restrict__ dPre,
+                  float* __restrict__ partial, long long partial_stride, int nslab, int32_t* __restrict__ err) {
+    constexpr int NP = 4 * NQ;
+    extern __shared__ __align__(128) unsigned char narrow_smem[];
+    __shared__ __align__(8) unsigned long long bars[kStages];
+    const RowSpan ch = chunks[blockIdx.x];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int slab = warp % nslab, rg = warp / nslab, nrg = kWarps / nslab;
+    const int ldh4 = ldh >> 2, col4 = 32 * slab + lane, col = 4 * col4;
+    const bool live = col4 < ldh4;
+    const int BR = block_rows(nslab);
+    const int nblk = (ch.nrows + BR - 1) / BR;
+    Ring ring;
+    ring.A = H + (long long)ch.row0 * ldh; ring.B = dZ + (long long)ch.row0 * ldz;
+    ring.lda = ldh; ring.ldb = ldz; ring.nrows = ch.nrows; ring.BR = BR;
+    ring.stage_a_bytes = (uint32_t)BR * ldh * 4u; ring.stage_b_bytes = (uint32_t)BR * ldz * 4u;
+    ring.a_addr = smem_addr(narrow_smem);
+    ring.b_addr = ring.a_addr + kStages * ring.stage_a_bytes;
+    ring.bar0 = smem_addr(&bars[0]);
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) bar_init(ring.bar0 + 8u * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        for (int b = 0; b < min(kStages, nblk); ++b) ring.issue(b);
+
+    // this lane's block of W_k: rows col .. col+3, all NP columns
+    float Wr[4][NP], acc[4][NP];
+    {
+        const float* W = params + (long long)ch.k * pstride + w_int;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                const float4 t = (live && col + j < fi) ? __ldg(reinterpret_cast<const float4*>(W + (long long)(col + j) * ldw) + q)
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                Wr[j][4 * q] = t.x; Wr[j][4 * q + 1] = t.y; Wr[j][4 * q + 2] = t.z; Wr[j][4 * q + 3] = t.w;
+            }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int n = 0; n < NP; ++n) acc[j][n] = 0.f;
+    }
+    const float4* As = reinterpret_cast<const float4*>(narrow_smem);
+    const float4* Bs = reinterpret_cast<const float4*>(narrow_smem + kStages * ring.stage_a_bytes);
+    const int a_stage4 = (int)(ring.stage_a_bytes >> 4), b_stage4 = (int)(ring.stage_b_bytes >> 4);
+    for (int b = 0; b < nblk; ++b) {
+        const int s = b % kStages;
+        const bool ok = bar_wait(ring.bar0 + 8u * (uint32_t)s, (uint32_t)(b / kStages) & 1u);
+        if (__syncthreads_or(!ok)) {   // a copy never arrived: report it and stop
+            if (threadIdx.x == 0) atomicExch(err, 90);
+            return;
+        }
+        const int nb = min(BR, ch.nrows - b * BR);
+        const float4* Ab = As + s * a_stage4;
+        const float4* Bb = Bs + s * b_stage4;
+        for (int r = rg; r < nb; r += nrg) {
+            const float4 h4 = live ? Ab[r * ldh4 + col4] : make_float4(0.f, 0.f, 0.f, 0.f);
+            float dz[NP];
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                const float4 t = Bb[r * NQ + q];
+                dz[4 * q] = t.x; dz[4 * q + 1] = t.y; dz[4 * q + 2] = t.z; dz[4 * q + 3] = t.w;
+            }
+            const float h[4] = {h4.x, h4.y, h4.z, h4.w};
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int n = 0; n < NP; ++n) {
+                    v[j] = fmaf(dz[n], Wr[j][n], v[j]);
+                    acc[j][n] = fmaf(h[j], dz[n], acc[j][n]);
+                }
+            if (live) {
+                float4 o;
+                o.x = h[0] > 0.f ? v[0] * scale : 0.f; o.y = h[1] > 0.f ? v[1] * scale : 0.f;
+                o.z = h[2] > 0.f ? v[2] * scale : 0.f; o.w = h[3] > 0.f ? v[3] * scale : 0.f;
+                reinterpret_cast<float4*>(dPre + (long long)(ch.row0 + b * BR + r) * ldh)[col4] = o;
+            }
+        }
+        __syncthreads();   // the stage has been read by every warp
+        if (threadIdx.x == 0 && b + kStages < nblk) ring.issue(b + kStages);
+    }
+    // dW of the chunk: the row groups of a slab added in order (through the ring's memory, now idle)
+    float* red = reinterpret_cast<float*>(narrow_smem);   // [warp][4 * NP][32 lanes]
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int n = 0; n < NP; ++n) red[(warp * 4 * NP + j * NP + n) * 32 + lane] = acc[j][n];
+    __syncthreads();
+    float* out = partial + (long long)blockIdx.x * partial_stride;
+    for (int e = threadIdx.x; e < nslab * 4 * NP * 32; e += 32 * kWarps) {
+        const int sl = e / (4 * NP * 32), jn = (e / 32) % (4 * NP), ln = e & 31;
+        float sum = 0.f;
+        for (int g = 0; g < nrg; ++g) sum += red[((g * nslab + sl) * 4 * NP + jn) * 32 + ln];
+        const int c = 128 * sl + 4 * ln + jn / NP, n = jn % NP;
+        if (c < fi) out[(long long)c * ldw + n] = sum;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// forward: Z rows of the chunk
+// ---------------------------------------------------------------------------------------------
+// NP: the output columns rounded up to a power of two; a warp takes 32 / NP rows at a time so that the sums of
+// one step are 32 values, spread over the 32 lanes by a halving exchange (lane i ends with value i).
+template <int NP>
+__global__ void __launch_bounds__(32 * kWarps, 3)
+narrow_fwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __restrict__ params, long long pstride, long long w_int,
+                  int ldw, const RowSpan* __restrict__ chunks, float* __restrict__ Z, int ldz, int nslab, int32_t* __restrict__ err) {
+    constexpr int RPI = 32 / NP;
+    extern __shared__ __align__(128) unsigned char narrow_smem[];
+    __shared__ __align__(8) unsigned long long bars[kStages];
+    const RowSpan ch = chunks[blockIdx.x];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int slab = warp % nslab, rg = warp / nslab, nrg = kWarps / nslab;
+    const int ldh4 = ldh >> 2, col4 = 32 * slab + lane, col = 4 * col4;
+    const bool live = col4 < ldh4;
+    const int BR = block_rows(nslab);
+    const int nblk = (ch.nrows + BR - 1) / BR;
+    Ring ring;
+    ring.A = H + (long long)ch.row0 * ldh; ring.B = nullptr;
+    ring.lda = ldh; ring.ldb = 0; ring.nrows = ch.nrows; ring.BR = BR;
+    ring.stage_a_bytes = (uint32_t)BR * ldh * 4u; ring.stage_b_bytes = 0;
+    ring.a_addr = smem_addr(narrow_smem);
+    ring.b_addr = 0;
+    ring.bar0 = smem_addr(&bars[0]);
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) bar_init(ring.bar0 + 8u * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        for (int b = 0; b < min(kStages, nblk); ++b) ring.issue(b);
+
+    float Wr[4][NP];
+    {
+        const float* W = params + (long long)ch.k * pstride + w_int;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int q = 0; q < NP / 4; ++q) {
+                const float4 t = (live && col + j < fi && 4 * q < ldw) ? __ldg(reinterpret_cast<const float4*>(W + (long long)(col + j) * ldw) + q)
+                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                Wr[j][4 * q] = t.x; Wr[j][4 * q + 1] = t.y; Wr[j][4 * q + 2] = t.z; Wr[j][4 * q + 3] = t.w;
+            }
+    }
+    const float4* As = reinterpret_cast<const float4*>(narrow_smem);
+    const int a_stage4 = (int)(ring.stage_a_bytes >> 4);
+    // per-slab sums of a block, two buffers (a warp may be one block ahead of the slowest reader)
+    float* red = reinterpret_cast<float*>(narrow_smem + kStages * ring.stage_a_bytes);   // [2][nslab][32 rows x NP]
+    for (int b = 0; b < nblk; ++b) {
+        const int s = b % kStages;
+        const bool ok = bar_wait(ring.bar0 + 8u * (uint32_t)s, (uint32_t)(b / kStages) & 1u);
+        if (__syncthreads_or(!ok)) {
+            if (threadIdx.x == 0) atomicExch(err, 91);
+            return;
+        }
+        const int nb = min(BR, ch.nrows - b * BR);
+        const float4* Ab = As + s * a_stage4;
+        float* rb = red + (b & 1) * nslab * 32 * NP + slab * 32 * NP;
+        for (int g = rg; g * RPI < nb; g += nrg) {
+            float x[32];
+#pragma unroll
+            for (int rr = 0; rr < RPI; ++rr) {
+                const int r = g * RPI + rr;
+                const float4 h = (live && r < nb) ? Ab[r * ldh4 + col4] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int n = 0; n < NP; ++n)
+                    x[rr * NP + n] = fmaf(h.w, Wr[3][n], fmaf(h.z, Wr[2][n], fmaf(h.y, Wr[1][n], h.x * Wr[0][n])));
+            }
+            // halving exchange: after the step with distance d a lane keeps the half of its values selected by that
+            // bit of its index; lane i ends with the sum over all lanes of value i
+#pragma unroll
+            for (int d = 16, n = 32; d >= 1; d >>= 1, n >>= 1) {
+                const bool up = (lane & d) != 0;
+#pragma unroll
+                for (int i = 0; i < n / 2; ++i) {
+                    const float send = up ? x[i] : x[i + n / 2];
+                    const float keep = up ? x[i + n / 2] : x[i];
+                    x[i] = keep + __shfl_xor_sync(0xffffffffu, send, d);
+                }
+            }
+            rb[g * 32 + lane] = x[0];   // value (row g * RPI + lane / NP, column lane % NP)
+        }
+        __syncthreads();   // the stage has been read and the slab sums of the block are written
+        if (threadIdx.x == 0 && b + kStages < nblk) ring.issue(b + kStages);
+        const float* r0 = red + (b & 1) * nslab * 32 * NP;
+        for (int e = threadIdx.x; e < nb * NP; e += 32 * kWarps) {
+            float sum = 0.f;
+            for (int sl = 0; sl < nslab; ++sl) sum += r0[sl * 32 * NP + e];
+            const int r = e / NP, n = e % NP;
+            if (n < ldz) Z[(long long)(ch.row0 + b * BR + r) * ldz + n] = sum;
+        }
+    }
+}
+
+}  // namespace
+
+bool narrow_supported(int ldi, int ldo) { return ldo >= 4 && ldo <= 16 && ldi >= 4 && ldi <= 128 * kWarps; }
+
+// Room for the ring beyond the default 48 KB, and the shared-memory share of the SM set for three resident CTAs.
+template <class Kernel>
+static cudaError_t prepare(Kernel kernel) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+}
+
+static int slabs_for(int ldi) { const int s = (ldi + 127) / 128; return s <= 1 ? 1 : (s <= 2 ? 2 : 4); }
+
+cudaError_t launch_narrow_fwd(const float* H, int ldh, int fi, const float* params, int64_t pstride, int64_t w_int, int ldw,
+                              const RowSpan* chunks, int nchunks, float* Z, int ldz, int32_t* err, cudaStream_t s) {
+    if (nchunks <= 0) return cudaSuccess;
+    const int nslab = slabs_for(ldh), BR = block_rows(nslab);
+    const int np = ldz <= 4 ? 4 : (ldz <= 8 ? 8 : 16);
+    const size_t smem = (size_t)kStages * BR * ldh * 4 + 2ull * nslab * 32 * np * 4;
+    auto go = [&](auto kernel) -> cudaError_t {
+        static bool prepared = false;   // per instantiation
+        if (!prepared) {
+            cudaError_t e = prepare(kernel);
+            if (e != cudaSuccess) return e;
+            prepared = true;
+        }
+        kernel<<<(unsigned)nchunks, 32 * kWarps, smem, s>>>(H, ldh, fi, params, pstride, w_int, ldw, chunks, Z, ldz, nslab, err);
+        ++g_kernel_launches;
+        return cudaGetLastError();
+    };
+    return np == 4 ? go(narrow_fwd_kernel<4>) : (np == 8 ? go(narrow_fwd_kernel<8>) : go(narrow_fwd_kernel<16>));
+}
+
+cudaError_t launch_narrow_bwd(const float* H, int ldh, int fi, const float* dZ, int ldz, const float* params, int64_t pstride,
+                              int64_t w_int, int ldw, const RowSpan* chunks, int nchunks, float scale, float* dPre, float* partial,
+                              int64_t partial_stride, int32_t* err, cudaStream_t s) {
+    if (nchunks <= 0) return cudaSuccess;
+    const int nslab = slabs_for(ldh), BR = block_rows(nslab), nq = ldz / 4;
+    size_t smem = (size_t)kStages * BR * (ldh + ldz) * 4;
+    smem = std::max(smem, (size_t)kWarps * 4 * ldz * 32 * 4);   // the exchange of the dW blocks at the end
+    auto go = [&](auto kernel) -> cudaError_t {
+        static bool prepared = false;   // per instantiation
+        if (!prepared) {
+            cudaError_t e = prepare(kernel);
+            if (e != cudaSuccess) return e;
+            prepared = true;
+        }
+        kernel<<<(unsigned)nchunks, 32 * kWarps, smem, s>>>(H, ldh, fi, dZ, ldz, params, pstride, w_int, ldw, chunks, scale, dPre, partial,
+                                                            partial_stride, nslab, err);
+        ++g_kernel_launches;
+        return cudaGetLastError();
+    };
+    switch (nq) {
+        case 1: return go(narrow_bwd_kernel<1>);
+        case 2: return go(narrow_bwd_kernel<2>);
+        case 3: return go(narrow_bwd_kernel<3>);
+        default: return go(narrow_bwd_kernel<4>);
+    }
+}
+
+}  // namespace gad

@@ -468,3 +468,27 @@ def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
             assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
             assert rel_err(g.get_params(k), ref.get_params(k)) <= tol
         assert rel_err(g.forward(), ref.forward_global(case[0])) <= tol
+
+
+@pytest.mark.parametrize("flags", [0, 4])
+@pytest.mark.parametrize("dims,dropout", [((40, 128, 16), 0.0), ((30, 200, 12), 0.0), ((24, 500, 7), 0.3), ((100, 8, 3), 0.0),
+                                          ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0)])
+def test_layers_of_at_most_sixteen_output_columns(flags, dims, dropout):
+    """Layers with at most 16 output columns run as streams on the FP32 ALUs (forward H.W; backward dW and the masked
+    input gradient in one pass), or with flags bit 2 through the tensor-core transforms like any other layer.  Input
+    widths of one, two and four 128-column slabs, ragged ones, one beyond the kernels' limit (516: tensor cores
+    again), a narrow layer in the middle of the network and one that is layer 0."""
+    case = small_random_case(31, n=1500, K=3, p=0.006)
+    g, ref, st = make_pair(case, dims, 31, lr=0.05, dropout=dropout, flags=flags)
+    with g:
+        for _ in range(2):
+            lg, lr = g.train_epoch(), ref.train_epoch()
+            assert np.max(np.abs(lg - lr)) <= 1e-4
+        L = len(dims) - 1
+        for l in range(1, L + 1):
+            assert rel_err(g.get_activation(l), ref.activation(l)) <= TOL, "activation %d" % l
+        gt = grad_tol(g, ref, TOL)
+        for k in range(g.K):
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+        assert rel_err(g.forward(), ref.forward_global(case[0])) <= TOL
