@@ -83,8 +83,9 @@ typedef struct {
     int32_t flags;        /* bit 0: force the SIMT transform even where a tensor-core kernel exists;
                              bit 1: layer 0 aggregates first and keeps A~ H^(0) from one epoch to the next (it
                              changes only with the features, i.e. with gad_set_inputs);
-                             bit 2: layers of at most 16 output columns also go through the tensor-core transforms
-                             instead of the streaming FP32 kernels written for them (for comparison)           */
+                             bit 2: the backward pass of a layer of at most 16 output columns also goes through the
+                             tensor-core transforms instead of the streaming FP32 kernel written for it (for
+                             comparison)                                                                      */
 } gad_config;
 
 /* Bytes of device workspace gad_create needs for these inputs.  Host-only; touches no GPU. */

@@ -39,7 +39,7 @@ struct Plan {
     bool agg_first0 = false;          // layer 0 aggregates before it transforms
     size_t o_P = 0;                   // A~ H^(0)  [Np x ld0], only with agg_first0
     size_t o_counters = 0;            // arrival counters: [loss | K column sums | K zeta]
-    // layers of at most 16 output columns take the streaming FP32 kernels (flag bit 2 switches them off)
+    // layers l >= 1 of at most 16 output columns take the streaming FP32 kernel on the way back (flag bit 2 switches it off)
     std::vector<uint8_t> narrow;      // [L]
     std::vector<RowSpan> nchunks;     // their row chunks: about three CTAs per SM, never across subgraphs
     std::vector<int32_t> nchunk_ptr;  // [K+1]
@@ -167,7 +167,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     for (int l = 0; l < p.L; ++l) {
         const Layer& y = p.layers[l];
         const bool agg_first = l == 0 && p.agg_first0;
-        p.narrow[l] = (cfg->flags & 5) == 0 && !agg_first && narrow_supported(y.ldi, y.ldo);
+        p.narrow[l] = (cfg->flags & 5) == 0 && l > 0 && !agg_first && narrow_supported(y.ldi, y.ldo);
         if (p.narrow[l]) narrow_partial = std::max(narrow_partial, (int64_t)y.fi * y.ldw);
     }
     if (narrow_partial > 0) {
@@ -329,11 +329,8 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
             });
             continue;
         }
-        if (split_pending && !(ctx->use_tc && p.narrow[l])) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
+        if (split_pending) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
         GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
-            if (ctx->use_tc && p.narrow[l])
-                return launch_narrow_fwd(ctx->H(l), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, ctx->at<RowSpan>(p.o_nchunks),
-                                         (int)p.nchunks.size(), Z, y.ldo, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
             if (ctx->use_tc)
                 return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 0, passes, y.fi, y.fo, Z,
                                            y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr,
@@ -396,7 +393,7 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                     [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
-        if (l > 0 && ctx->use_tc && p.narrow[l]) {
+        if (ctx->use_tc && p.narrow[l]) {
             // one pass over H^(l) and dZ gives both dW and dPre of the layer below (it writes G1: the column sums come first)
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
             GAD_RUN("gemm_dwdh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 8.0 * p.K * y.fi * y.fo, 4.0 * p.Np * y.fi * y.fo, [&] {

@@ -151,14 +151,11 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
 cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,
                               int nchunks, float* partial, int32_t* err, cudaStream_t s);
 
-// Transforms of a layer with at most 16 output columns, as streams on the FP32 ALUs (narrow.cu).  `chunks` are runs of
-// rows of one subgraph, one CTA each.  Forward: Z = H W_k.  Backward, in one pass over H and dZ: partial[chunk] =
-// H[chunk rows]^T dZ[chunk rows] ([fi x ldw], to be added per subgraph by launch_reduce_chunks) and dPre = (dZ W_k^T)
-// masked by H > 0, times `scale`.  H and dZ must be contiguous (leading dimension = row length).  err receives 90 / 91 if
-// a bounded wait runs out.
+// Backward transforms of a layer with at most 16 output columns as one stream on the FP32 ALUs (narrow.cu).  `chunks`
+// are runs of rows of one subgraph, one CTA each.  In one pass over H and dZ: partial[chunk] = H[chunk rows]^T dZ[chunk
+// rows] ([fi x ldw], to be added per subgraph by launch_reduce_chunks) and dPre = (dZ W_k^T) masked by H > 0, times
+// `scale`.  H and dZ must be contiguous (leading dimension = row length).  err receives 90 if a bounded wait runs out.
 bool narrow_supported(int ldi, int ldo);
-cudaError_t launch_narrow_fwd(const float* H, int ldh, int fi, const float* params, int64_t pstride, int64_t w_int, int ldw,
-                              const RowSpan* chunks, int nchunks, float* Z, int ldz, int32_t* err, cudaStream_t s);
 cudaError_t launch_narrow_bwd(const float* H, int ldh, int fi, const float* dZ, int ldz, const float* params, int64_t pstride,
                               int64_t w_int, int ldw, const RowSpan* chunks, int nchunks, float scale, float* dPre, float* partial,
                               int64_t partial_stride, int32_t* err, cudaStream_t s);

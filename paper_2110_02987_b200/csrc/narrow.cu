@@ -1,19 +1,22 @@
-// Transforms of a layer with at most 16 output columns (a classifier layer: the paper's datasets have 3 .. 41
-// classes), on the FP32 ALUs.  With so few columns the product H W costs 2 * 16 flops per loaded value: the layer is
-// a stream over H^(l), bound by HBM, and a tensor-core tile (M = 128 at the price of any N) has nothing to offer.
+// Backward transforms of a layer with at most 16 output columns (a classifier layer: the paper's datasets have
+// 3 .. 41 classes), on the FP32 ALUs:
 //
-//   forward    Z_l = H^(l) W_k^(l)                                   (the H.W of the forward equation, Section 3.3)
-//   backward   dW_k^(l) = H^(l)^T dZ_l   and   dPre_(l-1) = (dZ_l W_k^(l)^T) masked by H^(l) > 0, in ONE pass over
-//              H^(l) and dZ_l (chain rule through the forward equation)
+//   dW_k^(l) = H^(l)^T dZ_l   and   dPre_(l-1) = (dZ_l W_k^(l)^T) masked by H^(l) > 0
+//
+// in ONE pass over H^(l) and dZ_l (chain rule through the forward equation, Section 3.3).  With so few columns
+// both products cost 2 * 16 flops per loaded value of H^(l), and the tensor-core kernels, whose M = 128 tile costs
+// the same for any N, would read H^(l) twice for them.
 //
 // A CTA of four warps owns a run of rows of one subgraph (a chunk) and streams it through a three-stage ring in
 // shared memory: one thread issues bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) of the next
 // row blocks of H^(l) and dZ_l while the warps work on the current one.  A lane owns four columns of H^(l) (a warp a
-// slab of 128 columns, wider layers spread their slabs over the warps) and keeps its 4 x 16 block of W_k^(l), and in
-// the backward kernel of dW, in registers for the whole chunk.  Chunk results of dW are added per subgraph in chunk
+// slab of 128 columns, wider layers spread their slabs over the warps) and keeps its 4 x 16 blocks of W_k^(l) and of
+// dW in registers for the whole chunk.  Chunk results of dW are added per subgraph in chunk
 // order by reduce_chunks, so nothing depends on scheduling.  Every mbarrier wait is bounded: on a time-out the CTA
 // raises the error word and returns.
 #include <algorithm>
+#include <mutex>
+#include <set>
 
 #include "gad_internal.h"
 
@@ -183,136 +186,27 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// forward: Z rows of the chunk
-// ---------------------------------------------------------------------------------------------
-// NP: the output columns rounded up to a power of two; a warp takes 32 / NP rows at a time so that the sums of
-// one step are 32 values, spread over the 32 lanes by a halving exchange (lane i ends with value i).
-template <int NP>
-__global__ void __launch_bounds__(32 * kWarps, 3)
-narrow_fwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __restrict__ params, long long pstride, long long w_int,
-                  int ldw, const RowSpan* __restrict__ chunks, float* __restrict__ Z, int ldz, int nslab, int32_t* __restrict__ err) {
-    constexpr int RPI = 32 / NP;
-    extern __shared__ __align__(128) unsigned char narrow_smem[];
-    __shared__ __align__(8) unsigned long long bars[kStages];
-    const RowSpan ch = chunks[blockIdx.x];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int slab = warp % nslab, rg = warp / nslab, nrg = kWarps / nslab;
-    const int ldh4 = ldh >> 2, col4 = 32 * slab + lane, col = 4 * col4;
-    const bool live = col4 < ldh4;
-    const int BR = block_rows(nslab);
-    const int nblk = (ch.nrows + BR - 1) / BR;
-    Ring ring;
-    ring.A = H + (long long)ch.row0 * ldh; ring.B = nullptr;
-    ring.lda = ldh; ring.ldb = 0; ring.nrows = ch.nrows; ring.BR = BR;
-    ring.stage_a_bytes = (uint32_t)BR * ldh * 4u; ring.stage_b_bytes = 0;
-    ring.a_addr = smem_addr(narrow_smem);
-    ring.b_addr = 0;
-    ring.bar0 = smem_addr(&bars[0]);
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int s = 0; s < kStages; ++s) bar_init(ring.bar0 + 8u * s, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-    if (threadIdx.x == 0)
-        for (int b = 0; b < min(kStages, nblk); ++b) ring.issue(b);
-
-    float Wr[4][NP];
-    {
-        const float* W = params + (long long)ch.k * pstride + w_int;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int q = 0; q < NP / 4; ++q) {
-                const float4 t = (live && col + j < fi && 4 * q < ldw) ? __ldg(reinterpret_cast<const float4*>(W + (long long)(col + j) * ldw) + q)
-                                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-                Wr[j][4 * q] = t.x; Wr[j][4 * q + 1] = t.y; Wr[j][4 * q + 2] = t.z; Wr[j][4 * q + 3] = t.w;
-            }
-    }
-    const float4* As = reinterpret_cast<const float4*>(narrow_smem);
-    const int a_stage4 = (int)(ring.stage_a_bytes >> 4);
-    // per-slab sums of a block, two buffers (a warp may be one block ahead of the slowest reader)
-    float* red = reinterpret_cast<float*>(narrow_smem + kStages * ring.stage_a_bytes);   // [2][nslab][32 rows x NP]
-    for (int b = 0; b < nblk; ++b) {
-        const int s = b % kStages;
-        const bool ok = bar_wait(ring.bar0 + 8u * (uint32_t)s, (uint32_t)(b / kStages) & 1u);
-        if (__syncthreads_or(!ok)) {
-            if (threadIdx.x == 0) atomicExch(err, 91);
-            return;
-        }
-        const int nb = min(BR, ch.nrows - b * BR);
-        const float4* Ab = As + s * a_stage4;
-        float* rb = red + (b & 1) * nslab * 32 * NP + slab * 32 * NP;
-        for (int g = rg; g * RPI < nb; g += nrg) {
-            float x[32];
-#pragma unroll
-            for (int rr = 0; rr < RPI; ++rr) {
-                const int r = g * RPI + rr;
-                const float4 h = (live && r < nb) ? Ab[r * ldh4 + col4] : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int n = 0; n < NP; ++n)
-                    x[rr * NP + n] = fmaf(h.w, Wr[3][n], fmaf(h.z, Wr[2][n], fmaf(h.y, Wr[1][n], h.x * Wr[0][n])));
-            }
-            // halving exchange: after the step with distance d a lane keeps the half of its values selected by that
-            // bit of its index; lane i ends with the sum over all lanes of value i
-#pragma unroll
-            for (int d = 16, n = 32; d >= 1; d >>= 1, n >>= 1) {
-                const bool up = (lane & d) != 0;
-#pragma unroll
-                for (int i = 0; i < n / 2; ++i) {
-                    const float send = up ? x[i] : x[i + n / 2];
-                    const float keep = up ? x[i + n / 2] : x[i];
-                    x[i] = keep + __shfl_xor_sync(0xffffffffu, send, d);
-                }
-            }
-            rb[g * 32 + lane] = x[0];   // value (row g * RPI + lane / NP, column lane % NP)
-        }
-        __syncthreads();   // the stage has been read and the slab sums of the block are written
-        if (threadIdx.x == 0 && b + kStages < nblk) ring.issue(b + kStages);
-        const float* r0 = red + (b & 1) * nslab * 32 * NP;
-        for (int e = threadIdx.x; e < nb * NP; e += 32 * kWarps) {
-            float sum = 0.f;
-            for (int sl = 0; sl < nslab; ++sl) sum += r0[sl * 32 * NP + e];
-            const int r = e / NP, n = e % NP;
-            if (n < ldz) Z[(long long)(ch.row0 + b * BR + r) * ldz + n] = sum;
-        }
-    }
-}
-
 }  // namespace
 
 bool narrow_supported(int ldi, int ldo) { return ldo >= 4 && ldo <= 16 && ldi >= 4 && ldi <= 128 * kWarps; }
 
-// Room for the ring beyond the default 48 KB, and the shared-memory share of the SM set for three resident CTAs.
+// Room for the ring beyond the default 48 KB, and the shared-memory share of the SM set for three resident CTAs; once
+// per kernel (the instantiations share one function-pointer type, so they are told apart by address).
 template <class Kernel>
 static cudaError_t prepare(Kernel kernel) {
+    static std::mutex lock;
+    static std::set<const void*> done;
+    std::lock_guard<std::mutex> guard(lock);
+    if (done.count(reinterpret_cast<const void*>(kernel))) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    done.insert(reinterpret_cast<const void*>(kernel));
+    return cudaSuccess;
 }
 
 static int slabs_for(int ldi) { const int s = (ldi + 127) / 128; return s <= 1 ? 1 : (s <= 2 ? 2 : 4); }
-
-cudaError_t launch_narrow_fwd(const float* H, int ldh, int fi, const float* params, int64_t pstride, int64_t w_int, int ldw,
-                              const RowSpan* chunks, int nchunks, float* Z, int ldz, int32_t* err, cudaStream_t s) {
-    if (nchunks <= 0) return cudaSuccess;
-    const int nslab = slabs_for(ldh), BR = block_rows(nslab);
-    const int np = ldz <= 4 ? 4 : (ldz <= 8 ? 8 : 16);
-    const size_t smem = (size_t)kStages * BR * ldh * 4 + 2ull * nslab * 32 * np * 4;
-    auto go = [&](auto kernel) -> cudaError_t {
-        static bool prepared = false;   // per instantiation
-        if (!prepared) {
-            cudaError_t e = prepare(kernel);
-            if (e != cudaSuccess) return e;
-            prepared = true;
-        }
-        kernel<<<(unsigned)nchunks, 32 * kWarps, smem, s>>>(H, ldh, fi, params, pstride, w_int, ldw, chunks, Z, ldz, nslab, err);
-        ++g_kernel_launches;
-        return cudaGetLastError();
-    };
-    return np == 4 ? go(narrow_fwd_kernel<4>) : (np == 8 ? go(narrow_fwd_kernel<8>) : go(narrow_fwd_kernel<16>));
-}
 
 cudaError_t launch_narrow_bwd(const float* H, int ldh, int fi, const float* dZ, int ldz, const float* params, int64_t pstride,
                               int64_t w_int, int ldw, const RowSpan* chunks, int nchunks, float scale, float* dPre, float* partial,
@@ -322,12 +216,8 @@ cudaError_t launch_narrow_bwd(const float* H, int ldh, int fi, const float* dZ, 
     size_t smem = (size_t)kStages * BR * (ldh + ldz) * 4;
     smem = std::max(smem, (size_t)kWarps * 4 * ldz * 32 * 4);   // the exchange of the dW blocks at the end
     auto go = [&](auto kernel) -> cudaError_t {
-        static bool prepared = false;   // per instantiation
-        if (!prepared) {
-            cudaError_t e = prepare(kernel);
-            if (e != cudaSuccess) return e;
-            prepared = true;
-        }
+        cudaError_t e = prepare(kernel);
+        if (e != cudaSuccess) return e;
         kernel<<<(unsigned)nchunks, 32 * kWarps, smem, s>>>(H, ldh, fi, dZ, ldz, params, pstride, w_int, ldw, chunks, scale, dPre, partial,
                                                             partial_stride, nslab, err);
         ++g_kernel_launches;

@@ -474,10 +474,10 @@ def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
 @pytest.mark.parametrize("dims,dropout", [((40, 128, 16), 0.0), ((30, 200, 12), 0.0), ((24, 500, 7), 0.3), ((100, 8, 3), 0.0),
                                           ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0)])
 def test_layers_of_at_most_sixteen_output_columns(flags, dims, dropout):
-    """Layers with at most 16 output columns run as streams on the FP32 ALUs (forward H.W; backward dW and the masked
-    input gradient in one pass), or with flags bit 2 through the tensor-core transforms like any other layer.  Input
-    widths of one, two and four 128-column slabs, ragged ones, one beyond the kernels' limit (516: tensor cores
-    again), a narrow layer in the middle of the network and one that is layer 0."""
+    """The backward pass of a layer l >= 1 with at most 16 output columns runs as one stream on the FP32 ALUs (dW and
+    the masked input gradient in one pass over H and dZ), or with flags bit 2 through the tensor-core transforms like
+    any other layer.  Input widths of one, two and four 128-column slabs, ragged ones, one beyond the kernel's limit
+    (516: tensor cores again), a narrow layer in the middle of the network and one that is layer 0 (tensor cores)."""
     case = small_random_case(31, n=1500, K=3, p=0.006)
     g, ref, st = make_pair(case, dims, 31, lr=0.05, dropout=dropout, flags=flags)
     with g:
