@@ -202,6 +202,61 @@ def cpu_baseline(w, theta, budget_s=20.0):
             "sample": "%d whole epochs of the same workload after one warm-up epoch" % n}
 
 
+def run_micro_consensus(args):
+    """HBM-sized point for the update and consensus kernel: K = 8 replicas of one 4096 x 4096 layer (P = 16.8 M
+    parameters, 0.5 GB per set of copies) over a small graph.  Prints one JSON line: the kernel's time inside an epoch
+    (SGD step + weighted consensus: 12 K P bytes) and inside gad_consensus (consensus alone: 8 K P bytes), against the measured
+    copy rate."""
+    import torch
+    import __graft_entry__ as entry
+    from gad_synth.graphs import sbm_graph
+    from gad_synth.partition import contiguous_partition, one_hop_halo
+    from gad_synth import glorot_params
+    import paper_2110_02987_b200 as pkg
+    if not os.path.exists(pkg.LIB_PATH):
+        entry.build()
+    torch.cuda.set_device(0)
+    rng = np.random.default_rng(0)
+    K, D, bs = 8, int(args.F) if args.F > 128 else 4096, 128
+    rowptr, col, block = sbm_graph(K, bs, 0.05, 0.002, rng)
+    n = K * bs
+    X = rng.standard_normal((n, D), dtype=np.float32)
+    y = rng.integers(0, D, size=n).astype(np.int32)
+    split = np.zeros(n, dtype=np.uint8)
+    core = contiguous_partition(n, K)
+    halo = one_hop_halo(rowptr, col, core, frac_of_candidates=0.05)
+    cp = np.zeros(K + 1, dtype=np.int64); np.cumsum([len(c) for c in core], out=cp[1:])
+    hp = np.zeros(K + 1, dtype=np.int64); np.cumsum([len(h) for h in halo], out=hp[1:])
+    theta = glorot_params((D, D), rng)
+    g = pkg.Gad(n, rowptr, col, cp, np.concatenate(core).astype(np.int32), hp,
+                np.concatenate(halo).astype(np.int32) if hp[-1] else np.empty(0, np.int32), X, y, split, (D, D), init_params=theta)
+    hbm_peak, _, peak_kind = measured_peaks()
+    for _ in range(3):
+        g.train_epoch(wait=False)
+    g.profile_enable(True); g.profile_reset()
+    for _ in range(args.steps or 10):
+        g.train_epoch(wait=False)
+    prof = {e["name"]: e for e in g.profile_read()}
+    e = prof["sgd_consensus"]
+    ms_in = e["total_ms"] / e["launches"]
+    g.profile_reset()
+    for _ in range(20):
+        g.consensus()    # importance weights, then the weighted mean written to all copies
+    prof = {e["name"]: e for e in g.profile_read()}
+    g.profile_enable(False)
+    c = prof["consensus"]
+    ms_alone = c["total_ms"] / c["launches"]
+    P = g.P
+    line = {"micro": "consensus", "K": K, "P": P, "bytes_per_copy_set": 4 * K * P,
+            "sgd_consensus_in_epoch": {"ms": ms_in, "bytes": e["bytes_per_launch"], "GBps": e["bytes_per_launch"] / ms_in / 1e6,
+                                       "frac": e["bytes_per_launch"] / ms_in / 1e6 / hbm_peak},
+            "gad_consensus": {"ms": ms_alone, "bytes": 8.0 * K * P, "GBps": 8.0 * K * P / ms_alone / 1e6,
+                              "frac": 8.0 * K * P / ms_alone / 1e6 / hbm_peak},
+            "peak": hbm_peak, "peak_source": peak_kind, "unit": "GB/s"}
+    g.destroy()
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -218,7 +273,12 @@ def main():
     ap.add_argument("--zeta-mode", type=int, default=0, help="1: literal pairwise importance weights (O(n^2 F) per subgraph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernels", action="store_true", help="also print the per-kernel table to stderr")
+    ap.add_argument("--micro", default=None, choices=["consensus"],
+                    help="a single-kernel point instead of the epoch benchmark (consensus: K = 8 copies of a 4096 x 4096 layer)")
     args = ap.parse_args()
+    if args.micro == "consensus":
+        run_micro_consensus(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "gad" else args.warmup
     if args.steps is None:
         args.steps = (1000 if args.workload in ("c2", "tiny", "tiny_signal") else 20) if args.impl == "gad" else 3

@@ -112,8 +112,9 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
     if (threadIdx.x == 0)
         for (int b = 0; b < min(kStages, nblk); ++b) ring.issue(b);
 
-    // this lane's block of W_k: rows col .. col+3, all NP columns
-    float Wr[4][NP], acc[4][NP];
+    // this lane's block of W_k: rows col .. col+3, all NP columns, kept as pairs of neighbouring columns for the
+    // two-wide FP32 multiply-add (one instruction, two IEEE fused multiply-adds)
+    float2 Wp[4][NP / 2], accp[4][NP / 2];
     {
         const float* W = params + (long long)ch.k * pstride + w_int;
 #pragma unroll
@@ -122,12 +123,12 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
             for (int q = 0; q < NQ; ++q) {
                 const float4 t = (live && col + j < fi) ? __ldg(reinterpret_cast<const float4*>(W + (long long)(col + j) * ldw) + q)
                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
-                Wr[j][4 * q] = t.x; Wr[j][4 * q + 1] = t.y; Wr[j][4 * q + 2] = t.z; Wr[j][4 * q + 3] = t.w;
+                Wp[j][2 * q] = make_float2(t.x, t.y); Wp[j][2 * q + 1] = make_float2(t.z, t.w);
             }
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int n = 0; n < NP; ++n) acc[j][n] = 0.f;
+            for (int m = 0; m < NP / 2; ++m) accp[j][m] = make_float2(0.f, 0.f);
     }
     const float4* As = reinterpret_cast<const float4*>(narrow_smem);
     const float4* Bs = reinterpret_cast<const float4*>(narrow_smem + kStages * ring.stage_a_bytes);
@@ -144,21 +145,25 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
         const float4* Bb = Bs + s * b_stage4;
         for (int r = rg; r < nb; r += nrg) {
             const float4 h4 = live ? Ab[r * ldh4 + col4] : make_float4(0.f, 0.f, 0.f, 0.f);
-            float dz[NP];
+            float2 dzp[NP / 2];
 #pragma unroll
             for (int q = 0; q < NQ; ++q) {
                 const float4 t = Bb[r * NQ + q];
-                dz[4 * q] = t.x; dz[4 * q + 1] = t.y; dz[4 * q + 2] = t.z; dz[4 * q + 3] = t.w;
+                dzp[2 * q] = make_float2(t.x, t.y); dzp[2 * q + 1] = make_float2(t.z, t.w);
             }
             const float h[4] = {h4.x, h4.y, h4.z, h4.w};
-            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            float v[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < 4; ++j) {
+                const float2 hh = make_float2(h[j], h[j]);
+                float2 v2 = make_float2(0.f, 0.f);   // even and odd columns of the dot product, added at the end
 #pragma unroll
-                for (int n = 0; n < NP; ++n) {
-                    v[j] = fmaf(dz[n], Wr[j][n], v[j]);
-                    acc[j][n] = fmaf(h[j], dz[n], acc[j][n]);
+                for (int m = 0; m < NP / 2; ++m) {
+                    v2 = __ffma2_rn(dzp[m], Wp[j][m], v2);
+                    accp[j][m] = __ffma2_rn(hh, dzp[m], accp[j][m]);
                 }
+                v[j] = v2.x + v2.y;
+            }
             if (live) {
                 float4 o;
                 o.x = h[0] > 0.f ? v[0] * scale : 0.f; o.y = h[1] > 0.f ? v[1] * scale : 0.f;
@@ -174,7 +179,7 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
 #pragma unroll
     for (int j = 0; j < 4; ++j)
 #pragma unroll
-        for (int n = 0; n < NP; ++n) red[(warp * 4 * NP + j * NP + n) * 32 + lane] = acc[j][n];
+        for (int n = 0; n < NP; ++n) red[(warp * 4 * NP + j * NP + n) * 32 + lane] = (n & 1) ? accp[j][n / 2].y : accp[j][n / 2].x;
     __syncthreads();
     float* out = partial + (long long)blockIdx.x * partial_stride;
     for (int e = threadIdx.x; e < nslab * 4 * NP * 32; e += 32 * kWarps) {
