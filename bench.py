@@ -257,6 +257,76 @@ def run_micro_consensus(args):
     print(json.dumps(line))
 
 
+def run_sharded(args, w, theta, rank, world, local_rank):
+    """Algorithm 2's deployment shape: the K subgraphs spread over the ranks, every rank a context with its share,
+    one all-reduce (NCCL) of the consensus buffer per epoch.  Strong scaling: the whole job is K subgraphs however
+    many GPUs share it.  Prints the same JSON line with "scaling": "strong"."""
+    import torch
+    import torch.distributed as dist
+    import paper_2110_02987_b200 as pkg
+    mine = pkg.shard_subgraphs(w.K, world, rank)
+    sub = type(w)(**{**w.__dict__})
+    sub.core, sub.halo = [w.core[k] for k in mine], [w.halo[k] for k in mine]
+    g = pkg.from_workload(sub, theta, gemm_mode=args.gemm_mode, flags=args.flags, zeta_mode=args.zeta_mode)
+    sh = pkg.ShardedEpoch(g)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        sh.step(want_loss=False)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = pkg.launch_count()
+    with ClockSampler(local_rank) as clk:
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            sh.step(want_loss=False)
+        e1.record()
+        barrier()
+    launches = pkg.launch_count() - l0
+    ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    value = args.steps / (ms * 1e-3)
+    # end to end: features and labels from pinned memory and the global loss read back, every step
+    Xp = torch.from_numpy(w.X).pin_memory()
+    yp = torch.from_numpy(w.labels).pin_memory()
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        g.set_inputs(Xp, yp)
+        loss = sh.step(want_loss=True)
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        g.set_inputs(Xp, yp)
+        loss = sh.step(want_loss=True)
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    total_nnz = torch.tensor([float(g.nnz_prime)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(total_nnz)
+    n_prime, buf_bytes = g.n_prime, 4 * g.consensus_floats()
+    g.destroy()
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f32" if args.gemm_mode == 0 else "tf32 operands, f32 accumulate", "data": "synthetic",
+            "config": {"workload": describe(w), "parallelism": "K subgraphs over %d rank(s), k = rank mod N; one all-reduce of %d bytes per epoch"
+                       % (world, buf_bytes), "n_prime_rank0": n_prime, "nnz_prime": int(total_nnz.item())},
+            "edges_per_s": value * float(total_nnz.item()), "final_loss": float(loss), "clocks": clk.summary(),
+            "e2e": {"value": e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                    "h2d_bytes_per_step": int(Xp.numel() * 4 + yp.numel() * 4), "d2h_bytes_per_step": int((g.K + 1) * 4)},
+            "gpu_launches": int(launches)}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -273,6 +343,8 @@ def main():
     ap.add_argument("--zeta-mode", type=int, default=0, help="1: literal pairwise importance weights (O(n^2 F) per subgraph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernels", action="store_true", help="also print the per-kernel table to stderr")
+    ap.add_argument("--shard", action="store_true",
+                    help="spread the K subgraphs over the ranks (one all-reduce per epoch) instead of running N replicas of the job")
     ap.add_argument("--micro", default=None, choices=["consensus"],
                     help="a single-kernel point instead of the epoch benchmark (consensus: K = 8 copies of a 4096 x 4096 layer)")
     args = ap.parse_args()
@@ -308,9 +380,13 @@ def main():
         dist.barrier()
     pkg.load()
 
-    # Replicas only: every rank runs the whole K-subgraph job on its own GPU (no collective on the data path).
+    # Replicas only (the default): every rank runs the whole K-subgraph job on its own GPU (no collective on the data
+    # path).  --shard: the K subgraphs are spread over the ranks (k = rank, rank + N, ...), one all-reduce per epoch.
     w = make_workload(args.workload, **args.wl_kw)
     theta = glorot_params(w.dims, np.random.default_rng(0))
+    if args.shard:
+        run_sharded(args, w, theta, rank, world, local_rank)
+        return
     g = pkg.from_workload(w, theta, gemm_mode=args.gemm_mode, flags=args.flags, zeta_mode=args.zeta_mode)
 
     def barrier():

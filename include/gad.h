@@ -138,6 +138,46 @@ int gad_subgraph_weights(gad_ctx* ctx, float* zeta_out, float* w_out);
  * when weighted == 0).  Enqueued on the stream. */
 int gad_consensus(gad_ctx* ctx);
 
+/* ---- Algorithm 2 with the subgraphs spread over several contexts --------------------------------------------
+ * Algorithm 2 assigns z subgraphs to each of n processors: the processors train one subgraph each at the same time,
+ * take the weighted consensus (Section 3.4.2) and go on to their next subgraph until all have been traversed (last
+ * paragraph of Section 3.3).  One context holds the subgraphs that train at the same time on ONE GPU.  Two uses:
+ *   - several GPUs: every GPU holds a context with its share of the subgraphs; per step each runs
+ *     gad_train_epoch_local and gad_consensus_partial, the buffers are added over the GPUs (one all-reduce of
+ *     gad_consensus_floats floats) and every GPU calls gad_consensus_apply with the sum;
+ *   - rounds (z > 1): one context per round; after a round's gad_train_epoch its model goes to the next round's
+ *     context with gad_export_params + gad_consensus_apply.
+ * All contexts must have the same layer sizes.  The buffers are device memory of gad_consensus_floats floats,
+ * 16-byte aligned, owned by the caller, in the library's padded parameter layout (opaque; the same for every context
+ * with the same layer sizes).  Everything is enqueued on the context's stream and nothing waits. */
+
+/* gad_train_epoch without the update and the consensus: forward, loss, backward, zeta.  Parameters unchanged,
+ * gradients ready for gad_consensus_partial.  loss_out as in gad_train_epoch (the last entry is the mean over THIS
+ * context's training rows). */
+int gad_train_epoch_local(gad_ctx* ctx, float* loss_out);
+
+/* |T_k|: the core training nodes of every subgraph, host [K] (the weights with which the subgraph losses combine
+ * into the loss of an epoch over several contexts). */
+int gad_get_train_counts(const gad_ctx* ctx, int64_t* counts);
+
+/* Floats in a consensus buffer. */
+int gad_consensus_floats(const gad_ctx* ctx, int64_t* count);
+
+/* This context's share of the weighted consensus (Section 3.4.2):
+ *   dev_out = sum over this context's replicas k of  w_k (theta_k - eta grad_k),   w_k = zeta_k / zeta_total,
+ * with zeta_total the sum of zeta over the subgraphs of ALL contexts (from gad_subgraph_weights of each); with
+ * weighted == 0 (Definition 3) w_k = 1 / zeta_total and zeta_total is the number of subgraphs of all contexts.
+ * with_step == 0 leaves out the "- eta grad_k" (a consensus of the parameters as they are; zeta is evaluated
+ * first).  with_step != 0 uses the gradients and zeta of the last gad_train_epoch_local.  The parameters are not
+ * changed. */
+int gad_consensus_partial(gad_ctx* ctx, double zeta_total, int32_t with_step, float* dev_out);
+
+/* theta_k <- dev_in for every replica k of this context (the finished consensus, or another context's model). */
+int gad_consensus_apply(gad_ctx* ctx, const float* dev_in);
+
+/* Replica k's parameters into a consensus buffer (device to device). */
+int gad_export_params(gad_ctx* ctx, int32_t k, float* dev_out);
+
 /* Parameter copy / gradient of replica k, host [P] in the layout above.  Gradients are those of the most recent
  * epoch (d L_k / d theta_k).  These calls wait for the stream. */
 int gad_get_params(gad_ctx* ctx, int32_t k, float* out);

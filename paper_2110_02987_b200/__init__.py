@@ -3,3 +3,4 @@
 from .binding import (  # noqa: F401
     Gad, GadError, gad_workspace_bytes, from_workload, launch_count, load, subgraph_weights_static, LIB_PATH, SYMBOLS,
 )
+from .multi import ShardedEpoch, RoundsEpoch, shard_subgraphs  # noqa: F401

@@ -25,7 +25,8 @@ SYMBOLS = (
     "gad_consensus", "gad_get_params", "gad_set_params", "gad_get_grads", "gad_param_count", "gad_store_sizes",
     "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_read_loss_async", "gad_synchronize", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
     "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_subgraph_weights_static", "gad_launch_count",
-    "gad_last_error", "gad_destroy",
+    "gad_last_error", "gad_destroy", "gad_train_epoch_local", "gad_consensus_floats", "gad_consensus_partial",
+    "gad_consensus_apply", "gad_export_params", "gad_get_train_counts",
 )
 
 
@@ -226,6 +227,55 @@ class Gad:
 
     def consensus(self):
         self._ck(self._L.gad_consensus(self._h))
+
+    # -- the subgraphs spread over several contexts ---------------------------------------------
+    def train_epoch_local(self, wait=True):
+        """gad_train_epoch_local: forward, loss, backward and zeta; no update, no consensus.  Returns the float32 [K+1]
+        losses with wait=True, None otherwise."""
+        if not wait:
+            self._ck(self._L.gad_train_epoch_local(self._h, None))
+            return None
+        out = np.zeros(self.K + 1, dtype=np.float32)
+        self._ck(self._L.gad_train_epoch_local(self._h, _ptr(out, C.c_float)))
+        return out
+
+    def ntrain(self):
+        """gad_get_train_counts: |T_k| of every subgraph, int64 [K]."""
+        out = np.zeros(self.K, dtype=np.int64)
+        self._ck(self._L.gad_get_train_counts(self._h, _ptr(out, C.c_int64)))
+        return out
+
+    def consensus_floats(self) -> int:
+        n = C.c_int64(0)
+        self._ck(self._L.gad_consensus_floats(self._h, C.byref(n)))
+        return int(n.value)
+
+    def new_consensus_buffer(self):
+        """A float32 CUDA tensor of gad_consensus_floats elements on this context's device."""
+        import torch
+        return torch.zeros(self.consensus_floats(), dtype=torch.float32, device=self.device)
+
+    def consensus_partial(self, zeta_total, out, with_step=True):
+        """gad_consensus_partial into the CUDA tensor ``out`` (see new_consensus_buffer)."""
+        self._check_buffer(out)
+        self._ck(self._L.gad_consensus_partial(self._h, C.c_double(float(zeta_total)), C.c_int32(1 if with_step else 0),
+                                               C.c_void_p(out.data_ptr())))
+        return out
+
+    def consensus_apply(self, buf):
+        self._check_buffer(buf)
+        self._ck(self._L.gad_consensus_apply(self._h, C.c_void_p(buf.data_ptr())))
+
+    def export_params(self, k, out):
+        self._check_buffer(out)
+        self._ck(self._L.gad_export_params(self._h, C.c_int32(k), C.c_void_p(out.data_ptr())))
+        return out
+
+    def _check_buffer(self, t):
+        import torch
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+                and t.numel() >= self.consensus_floats()):
+            raise GadError(-1, "a consensus buffer is a contiguous float32 CUDA tensor of consensus_floats() elements")
 
     # -- accessors -----------------------------------------------------------------------------
     def get_params(self, k):

@@ -679,7 +679,12 @@ int gad_get_loss(gad_ctx* ctx, float* loss_out) {
     return GAD_OK;
 }
 
-int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
+static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus);
+
+int gad_train_epoch(gad_ctx* ctx, float* loss_out) { return train_epoch(ctx, loss_out, true); }
+int gad_train_epoch_local(gad_ctx* ctx, float* loss_out) { return train_epoch(ctx, loss_out, false); }
+
+static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus) {
     if (!ctx) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
     cudaStream_t ss = side_of(ctx);
@@ -698,10 +703,11 @@ int gad_train_epoch(gad_ctx* ctx, float* loss_out) {
     if ((rc = backward_pass(ctx, ss)) != GAD_OK) return rc;
     if (ss == ctx->stream && (rc = zeta_pass(ctx, ss)) != GAD_OK) return rc;
     if ((rc = hand_over(ctx, ss, ctx->stream, ctx->ev_join)) != GAD_OK) return rc;
-    GAD_RUN("sgd_consensus", -1, 12.0 * p.K * p.Pint, 4.0 * p.K * p.Pint, [&] {
-        return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
-                                    ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->stream);
-    });
+    if (consensus)
+        GAD_RUN("sgd_consensus", -1, 12.0 * p.K * p.Pint, 4.0 * p.K * p.Pint, [&] {
+            return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
+                                        ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->stream);
+        });
     ctx->epoch += 1;
     if (loss_out) return gad_get_loss(ctx, loss_out);
     return GAD_OK;
@@ -743,6 +749,49 @@ int gad_consensus(gad_ctx* ctx) {
         return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, 0.f,
                                     ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 0, ctx->stream);
     });
+    return GAD_OK;
+}
+
+int gad_get_train_counts(const gad_ctx* ctx, int64_t* counts) {
+    if (!ctx || !counts) return GAD_ERR_ARG;
+    for (int32_t k = 0; k < ctx->p.K; ++k) counts[k] = ctx->ntrain[(size_t)k];
+    return GAD_OK;
+}
+
+int gad_consensus_floats(const gad_ctx* ctx, int64_t* count) {
+    if (!ctx || !count) return GAD_ERR_ARG;
+    *count = ctx->p.pstride;
+    return GAD_OK;
+}
+
+int gad_consensus_partial(gad_ctx* ctx, double total, int32_t with_step, float* dev_out) {
+    if (!ctx || !dev_out || !(total > 0.0) || ((uintptr_t)dev_out & 15) != 0) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    if (!with_step) {   // no epoch has necessarily run: evaluate zeta here
+        int rc = zeta_pass(ctx, ctx->stream);
+        if (rc != GAD_OK) return rc;
+    }
+    GAD_RUN("consensus_partial", -1, (with_step ? 8.0 : 4.0) * p.K * p.Pint + 4.0 * p.Pint, 4.0 * p.K * p.Pint, [&] {
+        return launch_consensus_partial(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
+                                        ctx->at<double>(p.o_zeta), ctx->cfg.weighted, with_step ? 1 : 0, total, dev_out, ctx->stream);
+    });
+    return GAD_OK;
+}
+
+int gad_consensus_apply(gad_ctx* ctx, const float* dev_in) {
+    if (!ctx || !dev_in || ((uintptr_t)dev_in & 15) != 0) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    GAD_RUN("consensus_apply", -1, 4.0 * (p.K + 1) * p.Pint, 0.0, [&] {
+        return launch_consensus_apply(ctx->at<float>(p.o_params), p.pstride, p.pstride, p.K, dev_in, ctx->stream);
+    });
+    return GAD_OK;
+}
+
+int gad_export_params(gad_ctx* ctx, int32_t k, float* dev_out) {
+    if (!ctx || !dev_out || k < 0 || k >= ctx->p.K) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    GAD_CK(cudaMemcpyAsync(dev_out, ctx->at<float>(p.o_params) + (int64_t)k * p.pstride, 4 * (size_t)p.pstride, cudaMemcpyDeviceToDevice,
+                           ctx->stream));
     return GAD_OK;
 }
 

@@ -197,6 +197,11 @@ cudaError_t launch_zeta_pair(const float* X, int ld, int F, const int32_t* deg, 
 
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, cudaStream_t s);
+// One context's share of a consensus over several contexts: out = sum_k w_k (theta_k - lr grad_k) with w_k = zeta_k / total
+// (or 1 / total), the parameters unchanged; and the finished sum written to every replica.
+cudaError_t launch_consensus_partial(const float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
+                                     const double* zeta, int weighted, int with_sgd, double total, float* out, cudaStream_t s);
+cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, int K, const float* in, cudaStream_t s);
 cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s);
 
 cudaError_t launch_gather_rows(const float* Xg, int F, const int32_t* gid, int64_t Np, float* H0, int ld,

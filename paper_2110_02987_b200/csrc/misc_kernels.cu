@@ -507,6 +507,54 @@ cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstr
     return cudaGetLastError();
 }
 
+// The same sum over the replicas of one context when the subgraphs are spread over several contexts:
+//   out = sum_k w_k (theta_k - lr * grad_k),  w_k = zeta_k / total (weighted) or 1 / total,
+// with `total` the sum over ALL contexts, so that the contexts' results add up to the consensus.  The parameters
+// themselves are left alone; consensus_apply_kernel writes the finished sum to every replica.
+__global__ void __launch_bounds__(256) consensus_partial_kernel(const float* __restrict__ params, const float* __restrict__ grads,
+                                                                long long pstride, long long len4, int K, float lr,
+                                                                const double* __restrict__ zeta, int weighted, int with_sgd,
+                                                                double total, float* __restrict__ out) {
+    extern __shared__ float w_sm[];
+    for (int k = threadIdx.x; k < K; k += blockDim.x) w_sm[k] = (float)((weighted ? zeta[k] : 1.0) / total);
+    __syncthreads();
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= len4) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < K; ++k) {
+        float4 p = reinterpret_cast<const float4*>(params + (long long)k * pstride)[i];
+        if (with_sgd) {
+            float4 g = reinterpret_cast<const float4*>(grads + (long long)k * pstride)[i];
+            p.x = fmaf(-lr, g.x, p.x); p.y = fmaf(-lr, g.y, p.y); p.z = fmaf(-lr, g.z, p.z); p.w = fmaf(-lr, g.w, p.w);
+        }
+        const float w = w_sm[k];
+        acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y); acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
+    }
+    reinterpret_cast<float4*>(out)[i] = acc;
+}
+__global__ void __launch_bounds__(256) consensus_apply_kernel(float* __restrict__ params, long long pstride, long long len4, int K,
+                                                              const float* __restrict__ in) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= len4) return;
+    const float4 v = reinterpret_cast<const float4*>(in)[i];
+    for (int k = 0; k < K; ++k) reinterpret_cast<float4*>(params + (long long)k * pstride)[i] = v;
+}
+cudaError_t launch_consensus_partial(const float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
+                                     const double* zeta, int weighted, int with_sgd, double total, float* out, cudaStream_t s) {
+    const long long len4 = len / 4;
+    if (len4 > 0) {
+        consensus_partial_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
+                                                                                                       zeta, weighted, with_sgd, total, out);
+        ++g_kernel_launches;
+    }
+    return cudaGetLastError();
+}
+cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, int K, const float* in, cudaStream_t s) {
+    const long long len4 = len / 4;
+    if (len4 > 0) { consensus_apply_kernel<<<(unsigned)((len4 + 255) / 256), 256, 0, s>>>(params, pstride, len4, K, in); ++g_kernel_launches; }
+    return cudaGetLastError();
+}
+
 __global__ void weights_kernel(const double* __restrict__ zeta, int K, int weighted, float* __restrict__ zeta_f,
                                float* __restrict__ w_f) {
     extern __shared__ float w_sm[];
