@@ -77,7 +77,10 @@ typedef struct {
     int32_t gemm_mode;    /* 0: fp32-accurate transform (SIMT, or tensor cores with every operand split in two);  *
                            * 1: reduced-precision operands (one TF32 pass) with fp32 accumulation on tensor cores */
     int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form, O(n'^2 F_0) per subgraph       *
-                           * (GAD_ERR_UNSUPPORTED when a subgraph has more than 32768 rows)                   */
+                           * (GAD_ERR_UNSUPPORTED when a subgraph has more than 32768 rows); 2: the aggregate  *
+                           * term with the sum over layers of the variance equation (Section 3.4.1) kept: the  *
+                           * squared distances are summed over the inputs H^(0) .. H^(L-1) of all layers, as   *
+                           * the most recent forward pass left them, so zeta changes from epoch to epoch        */
     float beta;           /* beta of the importance weight (Section 3.4.1); the paper uses 1                  */
     int32_t weighted;     /* 1: weighted global consensus (Section 3.4.2); 0: plain average (Definition 3)    */
     int32_t flags;        /* bit 0: force the SIMT transform even where a tensor-core kernel exists;

@@ -25,14 +25,18 @@
  *     subgraph's own (non-replicated) nodes; replicated nodes only feed aggregation.
  *   - p(v_i) = local degree / sum of local degrees, unordered pairs, beta = 1 (fixed by the worked
  *     example); the distance term is the p-weighted RMS pairwise Euclidean distance of the input
- *     features ("aggregate" reading), or the literal pairwise form ("pairwise" reading).
+ *     features ("aggregate" reading), or the literal pairwise form ("pairwise" reading); with
+ *     zeta_mode 2 the aggregate reading keeps the sum over the layers of the variance equation: the
+ *     squared distance is summed over the inputs H^(0) .. H^(L-1) of all layers (the activations of the
+ *     most recent forward pass).
  *   - each processor takes one SGD step on its own copy, then the copies are replaced by their
  *     zeta-weighted mean; from identical copies this equals applying the weighted mean gradient.
  *
  * Pins: see tests/test_oracle_*.py (dense brute force, finite differences, the paper's printed
  * zeta values, Property 2, closed forms, special cases).  Parity unpinned (readings, not facts):
- * the choice between the aggregate and pairwise distance term when distances differ, local versus
- * global degrees in A~, induced halo-halo edges, loss on core nodes only.
+ * the choice between the aggregate and pairwise distance term when distances differ, whether the sum
+ * over layers is kept (zeta_mode 2) or not, local versus global degrees in A~, induced halo-halo edges,
+ * loss on core nodes only.
  */
 #include <math.h>
 #include <stdint.h>
@@ -260,7 +264,7 @@ orc_model* orc_create(int64_t Np, int64_t nnz, const int64_t* s_rowptr, const in
     int ok = m->rowptr && m->col && m->val && m->sub_off && m->deg && m->label && m->train && m->ntrain && m->H &&
              m->Z && m->dPre && m->dZ && m->params && m->grads;
     if (ok) for (int l = 0; l <= L; ++l) {
-        m->H[l] = (double*)malloc(sizeof(double) * rows * (size_t)dims[l]);
+        m->H[l] = (double*)calloc(rows * (size_t)dims[l], sizeof(double));
         if (!m->H[l]) ok = 0;
     }
     if (!ok) { orc_destroy(m); return NULL; }
@@ -494,8 +498,26 @@ void orc_subgraph_weights(orc_model* m, double* zeta, double* w) {
     double tot = 0.0;
     for (int32_t k = 0; k < m->K; ++k) {
         int64_t r0 = m->sub_off[k], n = m->sub_off[k + 1] - r0;
-        zeta[k] = m->zeta_mode == 1 ? orc_zeta_pairwise(m->deg + r0, m->H[0] + r0 * F, n, F, m->beta)
-                                    : orc_zeta_aggregate(m->deg + r0, m->H[0] + r0 * F, n, F, m->beta);
+        if (m->zeta_mode == 2) {
+            /* The sum over the layers l of the variance equation (Section 3.4.1) kept: the squared distance of two
+             * nodes is summed over the inputs H^(0) .. H^(L-1) of all layers, i.e. it is the squared distance of the
+             * rows of [H^(0) | H^(1) | ... | H^(L-1)], as they stand after the most recent forward pass. */
+            int Ft = 0;
+            for (int l = 0; l < m->L; ++l) Ft += m->dims[l];
+            double* cat = (double*)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1) * (size_t)Ft);
+            for (int64_t i = 0; i < n; ++i) {
+                int o = 0;
+                for (int l = 0; l < m->L; ++l) {
+                    for (int f = 0; f < m->dims[l]; ++f) cat[i * Ft + o + f] = m->H[l][(r0 + i) * m->dims[l] + f];
+                    o += m->dims[l];
+                }
+            }
+            zeta[k] = orc_zeta_aggregate(m->deg + r0, cat, n, Ft, m->beta);
+            free(cat);
+        } else {
+            zeta[k] = m->zeta_mode == 1 ? orc_zeta_pairwise(m->deg + r0, m->H[0] + r0 * F, n, F, m->beta)
+                                        : orc_zeta_aggregate(m->deg + r0, m->H[0] + r0 * F, n, F, m->beta);
+        }
         tot += zeta[k];
     }
     for (int32_t k = 0; k < m->K; ++k)

@@ -44,6 +44,7 @@ struct Plan {
     std::vector<RowSpan> nchunks;     // their row chunks: about three CTAs per SM, never across subgraphs
     std::vector<int32_t> nchunk_ptr;  // [K+1]
     size_t o_nchunks = 0, o_nchunk_ptr = 0, o_nw_partial = 0;
+    size_t o_zeta_q = 0;              // [K] doubles: distance sums carried from layer to layer (zeta_mode 2)
     size_t bytes = 0;
     // offsets into the workspace
     size_t o_rowptr, o_ecv, o_fin, o_items, o_trowptr, o_tecv, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
@@ -66,7 +67,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         if (cfg->dims[l] < 1) { err = "layer size must be positive"; return GAD_ERR_ARG; }
     if (!(cfg->dropout >= 0.f && cfg->dropout < 1.f)) { err = "dropout must be in [0,1)"; return GAD_ERR_ARG; }
     if (cfg->gemm_mode != 0 && cfg->gemm_mode != 1) { err = "gemm_mode must be 0 or 1"; return GAD_ERR_ARG; }
-    if (cfg->zeta_mode != 0 && cfg->zeta_mode != 1) { err = "zeta_mode must be 0 or 1"; return GAD_ERR_ARG; }
+    if (cfg->zeta_mode < 0 || cfg->zeta_mode > 2) { err = "zeta_mode must be 0, 1 or 2"; return GAD_ERR_ARG; }
     if (cfg->zeta_mode == 1)   // O(n'^2 F_0) pairs per subgraph
         for (int32_t k = 0; k < K; ++k)
             if (sub_off[k + 1] - sub_off[k] > kZetaPairMaxRows) {
@@ -148,7 +149,11 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
     p.o_params = take(cur, 4 * (size_t)K * (size_t)p.pstride); p.o_grads = take(cur, 4 * (size_t)K * (size_t)p.pstride);
     p.o_dw_partial = take(cur, 4 * p.dw_chunks.size() * (size_t)p.dw_partial); p.o_cs_partial = take(cur, 4 * nc * (size_t)p.maxld);
-    p.o_loss_partial = take(cur, 4 * nc); p.o_zeta_partial = take(cur, 8 * nc * 2 * (size_t)p.ld[0]);
+    int32_t zeta_ld = p.ld[0];   // widest matrix the importance statistics run over: H^(0), or every layer's input (zeta_mode 2)
+    if (cfg->zeta_mode == 2)
+        for (int l = 0; l < p.L; ++l) zeta_ld = std::max(zeta_ld, p.ld[l]);
+    p.o_loss_partial = take(cur, 4 * nc); p.o_zeta_partial = take(cur, 8 * nc * 2 * (size_t)zeta_ld);
+    p.o_zeta_q = take(cur, 8 * (size_t)K);
     p.o_zeta = take(cur, 8 * (size_t)K); p.o_loss = take(cur, 4 * (size_t)(K + 1)); p.o_flags = take(cur, 16);
     p.o_zeta_f = take(cur, 4 * (size_t)K); p.o_w_f = take(cur, 4 * (size_t)K);
     p.o_stage = take(cur, 4 * (size_t)n * (size_t)std::max(p.dims[0], p.dims[p.L])); p.o_stage_lab = take(cur, 4 * (size_t)n);
@@ -168,7 +173,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         const Layer& y = p.layers[l];
         const bool agg_first = l == 0 && p.agg_first0;
         p.narrow[l] = (cfg->flags & 5) == 0 && l > 0 && !agg_first && narrow_supported(y.ldi, y.ldo);
-        if (p.narrow[l]) narrow_partial = std::max(narrow_partial, (int64_t)y.fi * y.ldw);
+        if (p.narrow[l]) narrow_partial = std::max(narrow_partial, (int64_t)y.fi * y.ldw + y.ldi);
     }
     if (narrow_partial > 0) {
         const int64_t Rn = std::max<int64_t>(64, round_up((p.Np + 443) / 444, 32));
@@ -216,6 +221,7 @@ struct gad_ctx {
     int stage_idx = 0;              // staging pair the next gad_set_inputs uses
     bool hoist = false;             // keep A~ H^(0) across epochs (config flag bit 1)
     bool P_valid = false;           // A~ H^(0) matches the current features
+    bool acts_valid = false;        // a forward pass has filled H^(1) .. H^(L)
     bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
     int num_sms = 1;
     struct alignas(64) TMap { unsigned char bytes[128]; };
@@ -341,11 +347,16 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
         GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                 [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, ctx->stream); });
     }
+    ctx->acts_valid = true;
     return GAD_OK;
 }
 
 int zeta_pass(gad_ctx* ctx, cudaStream_t s) {
     const Plan& p = ctx->p;
+    if (ctx->cfg.zeta_mode == 2 && !ctx->acts_valid) {   // asked for before any pass has run: an inference pass provides the activations
+        int rc = forward_pass(ctx, false, ctx->stream);
+        if (rc != GAD_OK) return rc;
+    }
     if (ctx->cfg.zeta_mode == 1) {
         const double pairs = 64.0 * 64.0 * (double)p.pair_ptr[p.K];
         GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 1), 3.0 * pairs * p.dims[0], [&] {
@@ -356,12 +367,22 @@ int zeta_pass(gad_ctx* ctx, cudaStream_t s) {
         });
         return GAD_OK;
     }
-    GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 1), 4.0 * p.Np * p.dims[0], [&] {
-        return launch_zeta(ctx->H(0), p.ld[0], p.dims[0], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
-                           (int)p.chunks.size(), ctx->at<int32_t>(p.o_chunk_ptr), ctx->at<int32_t>(p.o_sub_off),
-                           ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_deg_sq), ctx->cfg.beta,
-                           ctx->at<double>(p.o_zeta_partial), ctx->at<unsigned>(p.o_counters) + 1 + p.K, ctx->at<double>(p.o_zeta),
-                           s);
+    // zeta_mode 2 keeps the sum over the layers of the variance equation (Section 3.4.1): the statistics run over the
+    // input H^(l) of every layer (activations of the most recent forward pass), their distance sums added up
+    const int nl = ctx->cfg.zeta_mode == 2 ? p.L : 1;
+    double cols = 0.0;
+    for (int l = 0; l < nl; ++l) cols += p.dims[l];
+    GAD_RUN("zeta", -1, 4.0 * p.Np * (cols + nl), 4.0 * p.Np * cols, [&] {
+        for (int l = 0; l < nl; ++l) {
+            const int phase = nl == 1 ? 0 : (l == 0 ? 1 : (l == nl - 1 ? 3 : 2));
+            cudaError_t e = launch_zeta(ctx->H(l), p.ld[l], p.dims[l], ctx->at<int32_t>(p.o_deg), ctx->at<RowSpan>(p.o_chunks),
+                                        (int)p.chunks.size(), ctx->at<int32_t>(p.o_chunk_ptr), ctx->at<int32_t>(p.o_sub_off),
+                                        ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_deg_sq), ctx->cfg.beta,
+                                        ctx->at<double>(p.o_zeta_partial), ctx->at<unsigned>(p.o_counters) + 1 + p.K,
+                                        ctx->at<double>(p.o_zeta), ctx->at<double>(p.o_zeta_q), phase, s);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
     });
     return GAD_OK;
 }
@@ -379,16 +400,20 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
     const int ndw = (int)p.dw_chunks.size();
     const int32_t* dw_chunk_ptr = ctx->at<int32_t>(p.o_dw_chunk_ptr);
     const float scale = ctx->cfg.dropout > 0.f ? 1.f / (1.f - ctx->cfg.dropout) : 1.f;
+    bool bias_done = false;   // the layer above was narrow: its fused kernel has already summed this layer's dPre columns
     for (int l = p.L - 1; l >= 0; --l) {
         const Layer& y = p.layers[l];
-        // db reads dPre (G1) beside the kernels that follow; the next writer of G1 waits for it
-        int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_g1);
-        if (rc != GAD_OK) return rc;
-        GAD_RUN("bias_grad", l, 4.0 * p.Np * y.fo, 1.0 * p.Np * y.fo, [&] {
-            return launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr,
-                                        ctx->at<unsigned>(p.o_counters) + 1, grads, p.pstride, y.b_int, ss);
-        });
-        if (ss != ctx->stream) GAD_CK(cudaEventRecord(ctx->ev_bias, ss));
+        if (!bias_done) {
+            // db reads dPre (G1) beside the kernels that follow; the next writer of G1 waits for it
+            int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_g1);
+            if (rc != GAD_OK) return rc;
+            GAD_RUN("bias_grad", l, 4.0 * p.Np * y.fo, 1.0 * p.Np * y.fo, [&] {
+                return launch_colsum_chunks(G1, y.ldo, chunks, nc, ctx->at<float>(p.o_cs_partial), p.maxld, chunk_ptr,
+                                            ctx->at<unsigned>(p.o_counters) + 1, grads, p.pstride, y.b_int, ss);
+            });
+            if (ss != ctx->stream) GAD_CK(cudaEventRecord(ctx->ev_bias, ss));
+        }
+        bias_done = false;
         const bool agg_first = l == 0 && p.agg_first0;   // then dW = (A~ X)^T dPre and nothing flows further back
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
@@ -396,15 +421,17 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
         if (ctx->use_tc && p.narrow[l]) {
             // one pass over H^(l) and dZ gives both dW and dPre of the layer below (it writes G1: the column sums come first)
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
+            // the chunk results hold db of layer l-1 and then dW of layer l, which is also their order in the parameter block
+            const int64_t plen = (int64_t)y.ldi + (int64_t)y.fi * y.ldw;
             GAD_RUN("gemm_dwdh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 8.0 * p.K * y.fi * y.fo, 4.0 * p.Np * y.fi * y.fo, [&] {
                 cudaError_t e = launch_narrow_bwd(ctx->H(l), y.ldi, y.fi, G2, y.ldo, params, p.pstride, y.w_int, y.ldw,
                                                   ctx->at<RowSpan>(p.o_nchunks), (int)p.nchunks.size(), scale, G1,
-                                                  ctx->at<float>(p.o_nw_partial), (int64_t)y.fi * y.ldw,
-                                                  ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
+                                                  ctx->at<float>(p.o_nw_partial), plen, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
                 if (e != cudaSuccess) return e;
-                return launch_reduce_chunks(ctx->at<float>(p.o_nw_partial), (int64_t)y.fi * y.ldw, ctx->at<int32_t>(p.o_nchunk_ptr), p.K,
-                                            grads, p.pstride, y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
+                return launch_reduce_chunks(ctx->at<float>(p.o_nw_partial), plen, ctx->at<int32_t>(p.o_nchunk_ptr), p.K, grads, p.pstride,
+                                            p.layers[l - 1].b_int, plen, ctx->stream);
             });
+            bias_done = true;
             continue;
         }
         GAD_RUN("gemm_dw", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
@@ -691,7 +718,9 @@ static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus) {
     int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_fork);   // this epoch's side work follows everything enqueued so far
     if (rc != GAD_OK) return rc;
     if ((rc = forward_pass(ctx, true, ss)) != GAD_OK) return rc;
-    if (ss != ctx->stream && (rc = zeta_pass(ctx, ss)) != GAD_OK) return rc;   // beside the forward pass
+    // zeta beside the forward pass; with zeta_mode 2 it reads this pass's activations, so it follows it (beside the backward pass)
+    if (ctx->cfg.zeta_mode == 2 && (rc = hand_over(ctx, ctx->stream, ss, ctx->ev_fork)) != GAD_OK) return rc;
+    if (ss != ctx->stream && (rc = zeta_pass(ctx, ss)) != GAD_OK) return rc;
     const int C = p.dims[p.L];
     GAD_RUN("softmax_xent", -1, 8.0 * p.Np * C, 0.0, [&] {
         return launch_softmax_xent(ctx->H(p.L), p.ld[p.L], C, ctx->at<int32_t>(p.o_label), ctx->at<uint8_t>(p.o_train),

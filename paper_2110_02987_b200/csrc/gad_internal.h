@@ -152,9 +152,9 @@ cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, in
                               int nchunks, float* partial, int32_t* err, cudaStream_t s);
 
 // Backward transforms of a layer with at most 16 output columns as one stream on the FP32 ALUs (narrow.cu).  `chunks`
-// are runs of rows of one subgraph, one CTA each.  In one pass over H and dZ: partial[chunk] = H[chunk rows]^T dZ[chunk
-// rows] ([fi x ldw], to be added per subgraph by launch_reduce_chunks) and dPre = (dZ W_k^T) masked by H > 0, times
-// `scale`.  H and dZ must be contiguous (leading dimension = row length).  err receives 90 if a bounded wait runs out.
+// are runs of rows of one subgraph, one CTA each.  In one pass over H and dZ: dPre = (dZ W_k^T) masked by H > 0, times
+// `scale`, and partial[chunk] = [column sums of those dPre rows (ldh floats)] [H[chunk rows]^T dZ[chunk rows] (fi x ldw)],
+// to be added per subgraph by launch_reduce_chunks (the bias of a layer lies right before the weights of the next).  H and dZ must be contiguous (leading dimension = row length).  err receives 90 if a bounded wait runs out.
 bool narrow_supported(int ldi, int ldo);
 cudaError_t launch_narrow_bwd(const float* H, int ldh, int fi, const float* dZ, int ldz, const float* params, int64_t pstride,
                               int64_t w_int, int ldw, const RowSpan* chunks, int nchunks, float scale, float* dPre, float* partial,
@@ -182,10 +182,11 @@ cudaError_t launch_softmax_xent(const float* logits, int ld, int C, const int32_
                                 float* loss_partial, const int32_t* chunk_ptr, int K, float inv_total, float* loss,
                                 int32_t* nonfinite, unsigned* counter, cudaStream_t s);
 
-// zeta[k] of every subgraph that has rows  (counters: one per subgraph).
+// zeta[k] of every subgraph that has rows  (counters: one per subgraph).  phase 0: from the matrix X alone; phases 1, 2, 3:
+// X is the first, a further, the last of several matrices whose squared distances add up (q_acc: one double per subgraph).
 cudaError_t launch_zeta(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
                         const int32_t* chunk_ptr, const int32_t* sub_off, const int64_t* deg_sum, const int64_t* deg_sq,
-                        float beta, double* partial, unsigned* counters, double* zeta, cudaStream_t s);
+                        float beta, double* partial, unsigned* counters, double* zeta, double* q_acc, int phase, cudaStream_t s);
 
 // zeta_k in the literal pairwise form, sum_{i<j} p_i p_j / (|x_i - x_j| + beta), 64 x 64 tiles of pairs (one CTA each,
 // pair_ptr[k] = first tile of subgraph k); counters: one per subgraph; partial: one double per tile.

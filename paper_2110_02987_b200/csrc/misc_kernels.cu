@@ -340,9 +340,12 @@ cudaError_t launch_reduce_chunks(const float* partial, int64_t pstride_chunk, co
 // two weighted sums per chunk and per feature in double precision.
 // ---------------------------------------------------------------------------------------------
 // zeta_k = S_k / (D_k + beta) from the chunk sums of subgraph k, chunks added in order; run by one whole CTA.
+// `phase` spreads one zeta over several matrices (the layers' inputs, zeta_mode 2): 0 = this matrix alone; 1 = the first
+// of several (its distance sum goes to q_acc[k]); 2 = a further one (added to q_acc[k]); 3 = the last one (added, then zeta).
 __device__ __forceinline__ void zeta_finalize(int k, const double* partial, int F, int ld, const int32_t* __restrict__ chunk_ptr,
                                               const int32_t* __restrict__ sub_off, const int64_t* __restrict__ deg_sum,
-                                              const int64_t* __restrict__ deg_sq, float beta, double* __restrict__ zeta) {
+                                              const int64_t* __restrict__ deg_sq, float beta, double* __restrict__ zeta,
+                                              double* __restrict__ q_acc, int phase) {
     __shared__ double red[256];
     __shared__ double seg_a[256], seg_b[256];
     const long long n = sub_off[k + 1] - sub_off[k];
@@ -375,14 +378,19 @@ __device__ __forceinline__ void zeta_finalize(int k, const double* partial, int 
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        double z = 0.0;
-        if (n > 0) {
-            const double sq = uniform ? 1.0 / (double)n : (double)deg_sq[k] / (D * D);
-            const double S = 0.5 * (1.0 - sq);
-            const double Q = red[0] > 0.0 ? red[0] : 0.0;
-            if (S > 0.0) z = S / (sqrt(Q / S) + (double)beta);
+        double Q = red[0] > 0.0 ? red[0] : 0.0;
+        if (phase == 2 || phase == 3) Q += q_acc[k];
+        if (phase == 1 || phase == 2) {
+            q_acc[k] = Q;
+        } else {
+            double z = 0.0;
+            if (n > 0) {
+                const double sq = uniform ? 1.0 / (double)n : (double)deg_sq[k] / (D * D);
+                const double S = 0.5 * (1.0 - sq);
+                if (S > 0.0) z = S / (sqrt(Q / S) + (double)beta);
+            }
+            zeta[k] = z;
         }
-        zeta[k] = z;
     }
 }
 
@@ -393,7 +401,8 @@ __global__ void __launch_bounds__(256) zeta_partial_kernel(const float* __restri
                                                            const int64_t* __restrict__ deg_sum, double* partial,
                                                            const int32_t* __restrict__ chunk_ptr,
                                                            const int64_t* __restrict__ deg_sq, float beta,
-                                                           unsigned* counters, double* __restrict__ zeta) {
+                                                           unsigned* counters, double* __restrict__ zeta,
+                                                           double* __restrict__ q_acc, int phase) {
     // threads = 8 row lanes x 32 column lanes of one float4 each (as in the column sums above)
     __shared__ double sm[8][32][8];
     const RowSpan c = chunks[blockIdx.x];
@@ -445,16 +454,16 @@ __global__ void __launch_bounds__(256) zeta_partial_kernel(const float* __restri
     }
     // the last CTA of this subgraph turns the chunk sums into zeta_k
     if (cta_arrive_last(counters + c.k, (unsigned)(chunk_ptr[c.k + 1] - chunk_ptr[c.k])))
-        zeta_finalize(c.k, partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta);
+        zeta_finalize(c.k, partial, F, ld, chunk_ptr, sub_off, deg_sum, deg_sq, beta, zeta, q_acc, phase);
 }
 
 // zeta[k] for every subgraph that has rows (the entry of an empty subgraph is left as it is: zero since creation).
 cudaError_t launch_zeta(const float* X, int ld, int F, const int32_t* deg, const RowSpan* chunks, int nchunks,
                         const int32_t* chunk_ptr, const int32_t* sub_off, const int64_t* deg_sum, const int64_t* deg_sq,
-                        float beta, double* partial, unsigned* counters, double* zeta, cudaStream_t s) {
+                        float beta, double* partial, unsigned* counters, double* zeta, double* q_acc, int phase, cudaStream_t s) {
     if (nchunks > 0) {
         zeta_partial_kernel<<<(unsigned)nchunks, 256, 0, s>>>(X, ld, F, deg, chunks, sub_off, deg_sum, partial, chunk_ptr, deg_sq, beta,
-                                                              counters, zeta);
+                                                              counters, zeta, q_acc, phase);
         ++g_kernel_launches;
     }
     return cudaGetLastError();

@@ -2,6 +2,7 @@
 // 3 .. 41 classes), on the FP32 ALUs:
 //
 //   dW_k^(l) = H^(l)^T dZ_l   and   dPre_(l-1) = (dZ_l W_k^(l)^T) masked by H^(l) > 0
+//   (and db_k^(l-1), the column sums of the dPre_(l-1) rows it writes)
 //
 // in ONE pass over H^(l) and dZ_l (chain rule through the forward equation, Section 3.3).  With so few columns
 // both products cost 2 * 16 flops per loaded value of H^(l), and the tensor-core kernels, whose M = 128 tile costs
@@ -130,6 +131,7 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
 #pragma unroll
             for (int m = 0; m < NP / 2; ++m) accp[j][m] = make_float2(0.f, 0.f);
     }
+    float bsum[4] = {0.f, 0.f, 0.f, 0.f};   // column sums of the dPre rows this lane writes (the bias gradient of the layer below)
     const float4* As = reinterpret_cast<const float4*>(narrow_smem);
     const float4* Bs = reinterpret_cast<const float4*>(narrow_smem + kStages * ring.stage_a_bytes);
     const int a_stage4 = (int)(ring.stage_a_bytes >> 4), b_stage4 = (int)(ring.stage_b_bytes >> 4);
@@ -169,6 +171,7 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
                 o.x = h[0] > 0.f ? v[0] * scale : 0.f; o.y = h[1] > 0.f ? v[1] * scale : 0.f;
                 o.z = h[2] > 0.f ? v[2] * scale : 0.f; o.w = h[3] > 0.f ? v[3] * scale : 0.f;
                 reinterpret_cast<float4*>(dPre + (long long)(ch.row0 + b * BR + r) * ldh)[col4] = o;
+                bsum[0] += o.x; bsum[1] += o.y; bsum[2] += o.z; bsum[3] += o.w;
             }
         }
         __syncthreads();   // the stage has been read by every warp
@@ -180,8 +183,13 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
     for (int j = 0; j < 4; ++j)
 #pragma unroll
         for (int n = 0; n < NP; ++n) red[(warp * 4 * NP + j * NP + n) * 32 + lane] = (n & 1) ? accp[j][n / 2].y : accp[j][n / 2].x;
+    float* redb = red + kWarps * 4 * NP * 32;             // [warp][4][32 lanes]
+#pragma unroll
+    for (int j = 0; j < 4; ++j) redb[(warp * 4 + j) * 32 + lane] = bsum[j];
     __syncthreads();
-    float* out = partial + (long long)blockIdx.x * partial_stride;
+    // the chunk's result: [column sums of dPre (ldh)] [dW (fi x ldw)]
+    float* outb = partial + (long long)blockIdx.x * partial_stride;
+    float* out = outb + ldh;
     for (int e = threadIdx.x; e < nslab * 4 * NP * 32; e += 32 * kWarps) {
         const int sl = e / (4 * NP * 32), jn = (e / 32) % (4 * NP), ln = e & 31;
         float sum = 0.f;
@@ -189,11 +197,19 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
         const int c = 128 * sl + 4 * ln + jn / NP, n = jn % NP;
         if (c < fi) out[(long long)c * ldw + n] = sum;
     }
+    for (int e = threadIdx.x; e < nslab * 4 * 32; e += 32 * kWarps) {
+        const int sl = e / 128, j = (e / 32) & 3, ln = e & 31;
+        float sum = 0.f;
+        for (int g = 0; g < nrg; ++g) sum += redb[((g * nslab + sl) * 4 + j) * 32 + ln];
+        const int c = 128 * sl + 4 * ln + j;
+        if (c < ldh) outb[c] = sum;
+    }
 }
 
 }  // namespace
 
-bool narrow_supported(int ldi, int ldo) { return ldo >= 4 && ldo <= 16 && ldi >= 4 && ldi <= 128 * kWarps; }
+// At least three quarters of a warp's lanes must own columns (a lane owns four): narrower inputs stay on the tensor cores.
+bool narrow_supported(int ldi, int ldo) { return ldo >= 4 && ldo <= 16 && ldi >= 96 && ldi <= 128 * kWarps; }
 
 // Room for the ring beyond the default 48 KB, and the shared-memory share of the SM set for three resident CTAs; once
 // per kernel (the instantiations share one function-pointer type, so they are told apart by address).
@@ -219,7 +235,7 @@ cudaError_t launch_narrow_bwd(const float* H, int ldh, int fi, const float* dZ, 
     if (nchunks <= 0) return cudaSuccess;
     const int nslab = slabs_for(ldh), BR = block_rows(nslab), nq = ldz / 4;
     size_t smem = (size_t)kStages * BR * (ldh + ldz) * 4;
-    smem = std::max(smem, (size_t)kWarps * 4 * ldz * 32 * 4);   // the exchange of the dW blocks at the end
+    smem = std::max(smem, (size_t)kWarps * 4 * (ldz + 1) * 32 * 4);   // the exchange of the dW blocks and column sums at the end
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = prepare(kernel);
         if (e != cudaSuccess) return e;

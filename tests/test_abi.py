@@ -63,7 +63,7 @@ def test_malformed_inputs_are_rejected_on_the_host():
     with pytest.raises(GadError) as e:
         _ws((n, rowptr, col, w, core, h3))
     assert e.value.code == -2
-    for kw, code in ((dict(dropout=1.0), -1), (dict(zeta_mode=2), -1), (dict(gemm_mode=7), -1), (dict(beta=0.0), -1)):
+    for kw, code in ((dict(dropout=1.0), -1), (dict(zeta_mode=3), -1), (dict(gemm_mode=7), -1), (dict(beta=0.0), -1)):
         with pytest.raises(GadError) as e:
             _ws((n, rowptr, col, w, core, halo), **kw)
         assert e.value.code == code

@@ -472,12 +472,13 @@ def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
 
 @pytest.mark.parametrize("flags", [0, 4])
 @pytest.mark.parametrize("dims,dropout", [((40, 128, 16), 0.0), ((30, 200, 12), 0.0), ((24, 500, 7), 0.3), ((100, 8, 3), 0.0),
-                                          ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0)])
+                                          ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0), ((20, 100, 10), 0.0)])
 def test_layers_of_at_most_sixteen_output_columns(flags, dims, dropout):
     """The backward pass of a layer l >= 1 with at most 16 output columns runs as one stream on the FP32 ALUs (dW and
     the masked input gradient in one pass over H and dZ), or with flags bit 2 through the tensor-core transforms like
     any other layer.  Input widths of one, two and four 128-column slabs, ragged ones, one beyond the kernel's limit
-    (516: tensor cores again), a narrow layer in the middle of the network and one that is layer 0 (tensor cores)."""
+    (516) and some below it (under 96 columns: tensor cores again), a narrow layer in the middle of the network (its
+    kernel also sums the bias gradient of the layer below) and one that is layer 0 (tensor cores)."""
     case = small_random_case(31, n=1500, K=3, p=0.006)
     g, ref, st = make_pair(case, dims, 31, lr=0.05, dropout=dropout, flags=flags)
     with g:
@@ -492,3 +493,26 @@ def test_layers_of_at_most_sixteen_output_columns(flags, dims, dropout):
             assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
         assert rel_err(g.forward(), ref.forward_global(case[0])) <= TOL
+
+
+@pytest.mark.parametrize("dims,dropout", [((12, 40, 9, 4), 0.0), ((130, 24, 6), 0.3), ((10, 5), 0.0)])
+def test_importance_weights_summed_over_the_layers(dims, dropout):
+    """zeta_mode 2: the aggregate distance term with the sum over layers kept (inputs H^(0) .. H^(L-1) of the epoch's own
+    forward pass).  Weights, losses and parameters against the oracle over three epochs, and the standalone call."""
+    case = small_random_case(51, n=400, K=4, p=0.02)
+    g, ref, st = make_pair(case, dims, 51, lr=0.2, dropout=dropout, zeta_mode=2, beta=0.5)
+    with g:
+        zg, wg = g.subgraph_weights()          # before any epoch: an inference pass provides the activations
+        ref.forward()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(wg - wr)) <= 1e-5 and rel_err(zg, zr) <= 1e-5
+        for _ in range(3):
+            lg, lr = g.train_epoch(), ref.train_epoch()
+            assert np.max(np.abs(lg - lr)) <= 1e-4
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(wg - wr)) <= 1e-5 and rel_err(zg, zr) <= 1e-5
+        gt = grad_tol(g, ref, TOL)
+        for k in range(g.K):
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL

@@ -181,3 +181,55 @@ def test_parameter_consensus_equals_weighted_gradient_step():
     m2.train_epoch()
     for k in range(m2.K):
         assert rel_err(m2.get_params(k), want) < 1e-12
+
+
+def test_layer_sum_reading_against_pair_loops_over_every_layer():
+    """zeta_mode 2 keeps the sum over the layers of the variance equation.  Pinned against O(n^2) pair loops written
+    here: S from the degrees, and the p-weighted squared distances added up layer by layer over the activations the
+    forward pass left (one loop nest per layer, not the concatenation the oracle forms)."""
+    dims = (6, 5, 4, 3)
+    n, rowptr, col, w, core, halo, X, y, split, theta, st = make_case(8, dims, n=36, K=2)
+    m = orc.Model(st, X, y, split, dims, theta, zeta_mode=2, beta=0.7)
+    m.forward()
+    zeta, wts = m.subgraph_weights()
+    acts = [m.activation(l) for l in range(len(dims) - 1)]
+    for k in range(st.K):
+        r0, r1 = int(st.sub_off[k]), int(st.sub_off[k + 1])
+        deg = st.deg[r0:r1].astype(np.float64)
+        p = deg / deg.sum() if deg.sum() > 0 else np.full(r1 - r0, 1.0 / (r1 - r0))
+        S = Q = 0.0
+        for i in range(r1 - r0):
+            for j in range(i + 1, r1 - r0):
+                S += p[i] * p[j]
+                for H in acts:
+                    d = H[r0 + i] - H[r0 + j]
+                    Q += p[i] * p[j] * float(d @ d)
+        want = S / (np.sqrt(Q / S) + 0.7)
+        assert abs(zeta[k] - want) <= 1e-12 * want
+    assert abs(wts.sum() - 1.0) < 1e-15
+
+
+def test_layer_sum_reading_with_one_layer_is_the_aggregate_reading():
+    dims = (6, 3)
+    n, rowptr, col, w, core, halo, X, y, split, theta, st = make_case(9, dims)
+    a = orc.Model(st, X, y, split, dims, theta, zeta_mode=0)
+    b = orc.Model(st, X, y, split, dims, theta, zeta_mode=2)
+    for _ in range(2):
+        assert np.array_equal(a.train_epoch(), b.train_epoch())
+    assert np.array_equal(a.get_params(0), b.get_params(0))
+    assert np.array_equal(a.subgraph_weights()[0], b.subgraph_weights()[0])
+
+
+def test_layer_sum_reading_changes_with_the_model():
+    """With hidden layers the weights follow the activations: they differ from the input-only reading and move as
+    the parameters move (the input-only weights never do)."""
+    dims = (6, 5, 3)
+    n, rowptr, col, w, core, halo, X, y, split, theta, st = make_case(10, dims)
+    a = orc.Model(st, X, y, split, dims, theta, zeta_mode=0, lr=0.5)
+    b = orc.Model(st, X, y, split, dims, theta, zeta_mode=2, lr=0.5)
+    b.train_epoch(); a.train_epoch()
+    z0, zb0 = a.subgraph_weights()[0].copy(), b.subgraph_weights()[0].copy()
+    assert np.all(zb0 < z0)            # more squared distance in the denominator
+    b.train_epoch(); a.train_epoch()
+    assert np.array_equal(a.subgraph_weights()[0], z0)
+    assert not np.array_equal(b.subgraph_weights()[0], zb0)
