@@ -88,7 +88,8 @@ typedef struct {
                              changes only with the features, i.e. with gad_set_inputs);
                              bit 2: the backward pass of a layer of at most 16 output columns also goes through the
                              tensor-core transforms instead of the streaming FP32 kernel written for it (for
-                             comparison)                                                                      */
+                             comparison);
+                             bit 3: never replay an epoch as a CUDA graph (see gad_train_epoch)                */
 } gad_config;
 
 /* Bytes of device workspace gad_create needs for these inputs.  Host-only; touches no GPU. */
@@ -120,7 +121,12 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
  * loss_out: host [K+1] = the K subgraph losses, then sum_k |T_k| L_k / sum_k |T_k|, all evaluated before the
  * update; the call then waits for the stream.  loss_out == NULL: the epoch is only enqueued (no wait, no
  * copy); read the losses later with gad_get_loss.  Returns GAD_ERR_NONFINITE if a loss is NaN or infinite
- * (detected when the losses are read). */
+ * (detected when the losses are read).
+ * From the second call on the launches of an epoch are replayed as one CUDA graph (captured on the context's
+ * stream, thread-local mode) when nothing in them changes from epoch to epoch: dropout == 0, flag bits 1 and 3 clear,
+ * per-kernel timing off, and a stream that can be captured (any stream but the legacy default one).  Otherwise, while
+ * the caller is capturing that stream itself, or if the capture fails, they are enqueued one by one; the results are
+ * the same either way. */
 int gad_train_epoch(gad_ctx* ctx, float* loss_out);
 
 /* Losses of the most recent epoch, host [K+1]; waits for the stream. */

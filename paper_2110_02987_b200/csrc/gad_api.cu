@@ -222,6 +222,9 @@ struct gad_ctx {
     bool hoist = false;             // keep A~ H^(0) across epochs (config flag bit 1)
     bool P_valid = false;           // A~ H^(0) matches the current features
     bool acts_valid = false;        // a forward pass has filled H^(1) .. H^(L)
+    // The launches of an epoch captured once and replayed (index 0: gad_train_epoch_local, 1: gad_train_epoch).
+    struct EpochGraph { cudaGraphExec_t exec = nullptr; int64_t kernels = 0; bool failed = false; } graphs[2];
+    int64_t direct_epochs = 0;      // epochs enqueued launch by launch so far (the first one also sets up the kernels)
     bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
     int num_sms = 1;
     struct alignas(64) TMap { unsigned char bytes[128]; };
@@ -711,8 +714,8 @@ static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus);
 int gad_train_epoch(gad_ctx* ctx, float* loss_out) { return train_epoch(ctx, loss_out, true); }
 int gad_train_epoch_local(gad_ctx* ctx, float* loss_out) { return train_epoch(ctx, loss_out, false); }
 
-static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus) {
-    if (!ctx) return GAD_ERR_ARG;
+// Every launch of one epoch, on the context's two streams.
+static int enqueue_epoch(gad_ctx* ctx, bool consensus) {
     const Plan& p = ctx->p;
     cudaStream_t ss = side_of(ctx);
     int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_fork);   // this epoch's side work follows everything enqueued so far
@@ -737,6 +740,59 @@ static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus) {
             return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
                                         ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->stream);
         });
+    return GAD_OK;
+}
+
+// An epoch's launch sequence depends on nothing that changes from epoch to epoch unless dropout is on (the mask is
+// indexed by the epoch) or A~ H^(0) is being kept (its first epoch differs), so it can be captured into a CUDA graph
+// once and replayed: one submission instead of about twenty, and no gaps between dependent kernels.  Needs a stream
+// that can be captured (not the legacy default stream).
+static bool graph_allowed(const gad_ctx* ctx) {
+    return (ctx->cfg.flags & 8) == 0 && ctx->stream != nullptr && ctx->stream != cudaStreamLegacy && ctx->stream != cudaStreamPerThread &&
+           !ctx->profiling && !ctx->hoist && !(ctx->cfg.dropout > 0.f) && ctx->direct_epochs >= 1;
+}
+
+static void capture_epoch(gad_ctx* ctx, bool consensus, gad_ctx::EpochGraph& eg) {
+    if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        eg.failed = true;   // e.g. the caller is capturing this stream already: the launches then go into that capture
+        return;
+    }
+    const int64_t before = g_kernel_launches;
+    const int rc = enqueue_epoch(ctx, consensus);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+    const int64_t kernels = g_kernel_launches - before;
+    g_kernel_launches = before;   // nothing has run yet
+    if (rc == GAD_OK && e == cudaSuccess && graph && cudaGraphInstantiate(&eg.exec, graph, 0) == cudaSuccess) {
+        eg.kernels = kernels;
+    } else {
+        eg.exec = nullptr;
+        eg.failed = true;
+    }
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+}
+
+static int train_epoch(gad_ctx* ctx, float* loss_out, bool consensus) {
+    if (!ctx) return GAD_ERR_ARG;
+    gad_ctx::EpochGraph& eg = ctx->graphs[consensus ? 1 : 0];
+    bool done = false;
+    cudaStreamCaptureStatus outer = cudaStreamCaptureStatusNone;   // a caller capturing the stream gets plain launches into its capture
+    if (graph_allowed(ctx) && !eg.failed && cudaStreamIsCapturing(ctx->stream, &outer) == cudaSuccess &&
+        outer == cudaStreamCaptureStatusNone) {
+        if (!eg.exec) capture_epoch(ctx, consensus, eg);
+        if (eg.exec) {
+            GAD_CK(cudaGraphLaunch(eg.exec, ctx->stream));
+            g_kernel_launches += eg.kernels;
+            done = true;
+        }
+    }
+    if (!done) {
+        int rc = enqueue_epoch(ctx, consensus);
+        if (rc != GAD_OK) return rc;
+        ctx->direct_epochs += 1;
+    }
     ctx->epoch += 1;
     if (loss_out) return gad_get_loss(ctx, loss_out);
     return GAD_OK;
@@ -1002,6 +1058,8 @@ const char* gad_last_error(const gad_ctx* ctx) { return ctx ? ctx->err.c_str() :
 
 void gad_destroy(gad_ctx* ctx) {
     if (!ctx) return;
+    for (auto& eg : ctx->graphs)
+        if (eg.exec) cudaGraphExecDestroy(eg.exec);
     for (auto& e : ctx->prof)
         for (auto& pr : e.pending) { cudaEventDestroy(pr.first); cudaEventDestroy(pr.second); }
     if (ctx->copy_stream) { cudaStreamSynchronize(ctx->copy_stream); cudaStreamDestroy(ctx->copy_stream); }

@@ -516,3 +516,39 @@ def test_importance_weights_summed_over_the_layers(dims, dropout):
         for k in range(g.K):
             assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+
+
+@pytest.mark.parametrize("dims,zeta_mode", [((24, 40, 5), 0), ((130, 128, 16), 0), ((12, 20, 9, 4), 2)])
+def test_epochs_replayed_as_a_graph_equal_epochs_enqueued_one_by_one(dims, zeta_mode):
+    """On a stream of its own the library captures the epoch's launches after the first epoch and replays them as one
+    CUDA graph; flags bit 3 keeps the launches one by one.  Same kernels in the same order: the results must agree
+    bit for bit, the launch counter must advance alike, and both must match the oracle."""
+    import torch
+    case = small_random_case(61, n=500, K=4, p=0.02)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        g, ref, st = make_pair(case, dims, 61, lr=0.1, zeta_mode=zeta_mode, stream=stream)
+        h, _, _ = make_pair(case, dims, 61, lr=0.1, zeta_mode=zeta_mode, stream=stream, flags=8)
+        with g, h:
+            for epoch in range(4):
+                n0 = pkg().launch_count()
+                lg = g.train_epoch()
+                n1 = pkg().launch_count()
+                lh = h.train_epoch()
+                n2 = pkg().launch_count()
+                lr = ref.train_epoch()
+                assert np.array_equal(lg, lh) and n1 - n0 == n2 - n1 > 0
+                assert np.max(np.abs(lg - lr)) <= 1e-4
+            for k in range(g.K):
+                assert np.array_equal(g.get_params(k), h.get_params(k))
+                assert np.array_equal(g.get_grads(k), h.get_grads(k))
+                assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+            # the epoch without update and consensus has a graph of its own
+            for _ in range(3):
+                assert np.array_equal(g.train_epoch_local(), h.train_epoch_local())
+            assert np.array_equal(g.get_grads(1), h.get_grads(1))
+            # new inputs between replays
+            X2 = np.random.default_rng(9).standard_normal((case[0], dims[0])).astype(np.float32)
+            g.set_inputs(X2); h.set_inputs(X2)
+            assert np.array_equal(g.train_epoch(), h.train_epoch())
+            assert np.array_equal(g.get_params(0), h.get_params(0))
