@@ -18,6 +18,7 @@
 #include <algorithm>
 #include <mutex>
 #include <set>
+#include <utility>
 
 #include "gad_internal.h"
 
@@ -216,14 +217,18 @@ bool narrow_supported(int ldi, int ldo) { return ldo >= 4 && ldo <= 16 && ldi >=
 template <class Kernel>
 static cudaError_t prepare(Kernel kernel) {
     static std::mutex lock;
-    static std::set<const void*> done;
+    static std::set<std::pair<int, const void*>> done;   // (device, kernel): function attributes are per device
     std::lock_guard<std::mutex> guard(lock);
-    if (done.count(reinterpret_cast<const void*>(kernel))) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const std::pair<int, const void*> key(dev, reinterpret_cast<const void*>(kernel));
+    if (done.count(key)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    done.insert(reinterpret_cast<const void*>(kernel));
+    done.insert(key);
     return cudaSuccess;
 }
 
