@@ -427,13 +427,18 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
             // the chunk results hold db of layer l-1 and then dW of layer l, which is also their order in the parameter block
             const int64_t plen = (int64_t)y.ldi + (int64_t)y.fi * y.ldw;
             GAD_RUN("gemm_dwdh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 8.0 * p.K * y.fi * y.fo, 4.0 * p.Np * y.fi * y.fo, [&] {
-                cudaError_t e = launch_narrow_bwd(ctx->H(l), y.ldi, y.fi, G2, y.ldo, params, p.pstride, y.w_int, y.ldw,
-                                                  ctx->at<RowSpan>(p.o_nchunks), (int)p.nchunks.size(), scale, G1,
-                                                  ctx->at<float>(p.o_nw_partial), plen, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
-                if (e != cudaSuccess) return e;
-                return launch_reduce_chunks(ctx->at<float>(p.o_nw_partial), plen, ctx->at<int32_t>(p.o_nchunk_ptr), p.K, grads, p.pstride,
-                                            p.layers[l - 1].b_int, plen, ctx->stream);
+                return launch_narrow_bwd(ctx->H(l), y.ldi, y.fi, G2, y.ldo, params, p.pstride, y.w_int, y.ldw,
+                                         ctx->at<RowSpan>(p.o_nchunks), (int)p.nchunks.size(), scale, G1,
+                                         ctx->at<float>(p.o_nw_partial), plen, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
             });
+            // the sum over the chunks is needed only by the update at the end of the epoch: beside the kernels that follow
+            int rc2 = hand_over(ctx, ctx->stream, ss, ctx->ev_g1);
+            if (rc2 != GAD_OK) return rc2;
+            GAD_RUN("reduce_dwdh", l, 4.0 * (double)p.nchunks.size() * (double)plen, 1.0 * (double)p.nchunks.size() * (double)plen, [&] {
+                return launch_reduce_chunks(ctx->at<float>(p.o_nw_partial), plen, ctx->at<int32_t>(p.o_nchunk_ptr), p.K, grads, p.pstride,
+                                            p.layers[l - 1].b_int, plen, ss);
+            });
+            if (ss != ctx->stream) GAD_CK(cudaEventRecord(ctx->ev_bias, ss));   // a later narrow layer reuses the chunk results' buffer
             bias_done = true;
             continue;
         }

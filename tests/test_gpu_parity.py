@@ -472,7 +472,7 @@ def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
 
 @pytest.mark.parametrize("flags", [0, 4])
 @pytest.mark.parametrize("dims,dropout", [((40, 128, 16), 0.0), ((30, 200, 12), 0.0), ((24, 500, 7), 0.3), ((100, 8, 3), 0.0),
-                                          ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0), ((20, 100, 10), 0.0)])
+                                          ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0), ((20, 100, 10), 0.0), ((12, 128, 16, 100, 8), 0.0)])
 def test_layers_of_at_most_sixteen_output_columns(flags, dims, dropout):
     """The backward pass of a layer l >= 1 with at most 16 output columns runs as one stream on the FP32 ALUs (dW and
     the masked input gradient in one pass over H and dZ), or with flags bit 2 through the tensor-core transforms like
