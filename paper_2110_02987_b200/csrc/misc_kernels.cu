@@ -161,16 +161,33 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(const float* __
     const int ld4 = ld >> 2;
     const float inv = inv_ntrain[c.k];
     float acc = 0.f;
-    for (int r = warp * RPW + g; r < c.nrows; r += 8 * RPW) {
+    // the loads of a row (loss mask, label, logits) do not wait for one another, and the next row's are requested
+    // before this row's are used
+    struct RowIn { bool train; int y; float4 v; };
+    auto fetch = [&](int r) {
+        RowIn in{false, 0, make_float4(0.f, 0.f, 0.f, 0.f)};
+        if (r < c.nrows) {
+            const long long row = c.row0 + r;
+            in.train = train[row] != 0;
+            in.y = label[row];
+            if (gl < ld4) in.v = reinterpret_cast<const float4*>(logits + row * ld)[gl];
+        }
+        return in;
+    };
+    int r = warp * RPW + g;
+    RowIn cur = fetch(r);
+    for (; r < c.nrows; r += 8 * RPW) {
+        const RowIn nxt = fetch(r + 8 * RPW);
         const long long row = c.row0 + r;
         float4* gout = reinterpret_cast<float4*>(dlogits + row * ld);
-        if (!train[row]) {
+        if (!cur.train) {
             if (gl < ld4) gout[gl] = make_float4(0.f, 0.f, 0.f, 0.f);
+            cur = nxt;
             continue;
         }
         float z[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         if (gl < ld4) {
-            const float4 v = reinterpret_cast<const float4*>(logits + row * ld)[gl];
+            const float4 v = cur.v;
             if (4 * gl + 0 < C) z[0] = v.x;
             if (4 * gl + 1 < C) z[1] = v.y;
             if (4 * gl + 2 < C) z[2] = v.z;
@@ -185,7 +202,7 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(const float* __
 #pragma unroll
         for (int o = L / 2; o > 0; o >>= 1) se += __shfl_xor_sync(gmask, se, o, L);
         const float lse = mx + logf(se);
-        const int y = label[row];
+        const int y = cur.y;
         const int yt = y & 3;
         const float mine = yt == 0 ? z[0] : (yt == 1 ? z[1] : (yt == 2 ? z[2] : z[3]));
         const float zy = __shfl_sync(gmask, mine, y >> 2, L);
@@ -199,6 +216,7 @@ __global__ void __launch_bounds__(256) softmax_xent_small_kernel(const float* __
             }
             gout[gl] = make_float4(o4[0], o4[1], o4[2], o4[3]);
         }
+        cur = nxt;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
