@@ -447,6 +447,28 @@ def test_c2_two_epochs_full_size():
         assert np.max(np.abs(wg - wr)) <= 1e-6
 
 
+def test_c2_ten_epoch_loss_curve_full_size_in_the_benchmark_configuration():
+    """The launch configuration bench.py times: full-size c2 on a stream of its own, so epochs 2 .. 10 are graph
+    replays.  Loss curve within 1e-3 of the oracle's over ten epochs (lr 0.5 so that it moves), parameters and
+    logits within 1e-4 at the end."""
+    import torch
+    w = make_workload("c2")
+    theta = glorot_params(w.dims, np.random.default_rng(0))
+    ref = orc().from_workload(w, theta, lr=0.5)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        with pkg().from_workload(w, theta, lr=0.5, stream=stream) as g:
+            n0 = pkg().launch_count()
+            lg = np.array([g.train_epoch() for _ in range(10)])
+            assert pkg().launch_count() - n0 == 10 * 18
+            lr = np.array([ref.train_epoch() for _ in range(10)])
+            assert np.max(np.abs(lg - lr)) <= LOSS_TOL
+            assert lr[0, -1] - lr[-1, -1] > 5e-3          # the curve moves by several times the tolerance
+            for k in (0, g.K - 1):
+                assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+            assert rel_err(g.forward(), ref.forward_global(w.n)) <= TOL
+
+
 @pytest.mark.parametrize("gemm_mode,flags,tol", [(0, 0, TOL), (0, 1, TOL), (1, 0, 5e-2), (0, 2, TOL), (0, 3, TOL)])
 @pytest.mark.parametrize("dims", [(96, 160, 40, 8), (602, 256, 41), (20, 300, 130, 3)])
 def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
