@@ -75,7 +75,8 @@ typedef struct {
     float dropout;        /* probability of dropping a hidden unit after the ReLU, in [0,1); 0 = none         */
     uint64_t seed;        /* seed of the dropout mask and of the default initialisation                       */
     int32_t gemm_mode;    /* 0: fp32-accurate transform (SIMT, or tensor cores with every operand split in two);  *
-                           * 1: reduced-precision operands (one TF32 pass) with fp32 accumulation on tensor cores */
+                           * 1: reduced-precision operands with fp32 accumulation: one TF32 pass on the tensor      *
+                           *    cores, and the aggregation gathers a bfloat16 copy of its operand (tolerance 5e-2)  */
     int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form, O(n'^2 F_0) per subgraph       *
                            * (GAD_ERR_UNSUPPORTED when a subgraph has more than 32768 rows); 2: the aggregate  *
                            * term with the sum over layers of the variance equation (Section 3.4.1) kept: the  *

@@ -45,6 +45,7 @@ struct Plan {
     std::vector<int32_t> nchunk_ptr;  // [K+1]
     size_t o_nchunks = 0, o_nchunk_ptr = 0, o_nw_partial = 0;
     size_t o_zeta_q = 0;              // [K] doubles: distance sums carried from layer to layer (zeta_mode 2)
+    size_t o_bf16 = 0;                // [Np x widest SpMM operand] bfloat16 copy of the operand (gemm_mode 1), else unused
     size_t bytes = 0;
     // offsets into the workspace
     size_t o_rowptr, o_ecv, o_fin, o_items, o_trowptr, o_tecv, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
@@ -146,6 +147,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     int32_t max_spmm_ld = 4;   // the SpMM runs at the widths F_1 .. F_L, and at F_0 when layer 0 aggregates first
     for (int l = p.agg_first0 ? 0 : 1; l <= p.L; ++l) max_spmm_ld = std::max(max_spmm_ld, p.ld[l]);
     p.o_spmm_scratch = take(cur, 4 * (size_t)slots * (size_t)max_spmm_ld);
+    if (cfg->gemm_mode == 1) p.o_bf16 = take(cur, 2 * Np * (size_t)max_spmm_ld);
     p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
     p.o_params = take(cur, 4 * (size_t)K * (size_t)p.pstride); p.o_grads = take(cur, 4 * (size_t)K * (size_t)p.pstride);
     p.o_dw_partial = take(cur, 4 * p.dw_chunks.size() * (size_t)p.dw_partial); p.o_cs_partial = take(cur, 4 * nc * (size_t)p.maxld);
@@ -284,6 +286,9 @@ int run(gad_ctx* ctx, const char* name, int layer, double bytes, double flops, F
         if (rc_ != GAD_OK) return rc_;          \
     } while (0)
 
+// Room for the bfloat16 copy of an aggregation's operand: the reduced-precision mode gathers from that copy.
+void* bf16_of(gad_ctx* ctx) { return ctx->cfg.gemm_mode == 1 ? (void*)(ctx->ws + ctx->p.o_bf16) : nullptr; }
+
 double spmm_bytes(const Plan& p, int F) { return 8.0 * p.nnz + 8.0 * p.Np + 8.0 * (double)p.Np * F; }
 
 // Inside a training epoch the kernels that depend on little (operand split of the weights, zeta, bias gradients) go
@@ -323,7 +328,7 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
             // A~ (X W) = (A~ X) W: aggregate at the input width, finish the layer in the transform's epilogue
             if (!(ctx->hoist && ctx->P_valid)) {
                 GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
-                        [&] { return launch_spmm(ctx->A, ctx->H(0), y.ldi, ctx->at<float>(p.o_P), y.ldi, y.fi, nullptr, ctx->stream); });
+                        [&] { return launch_spmm(ctx->A, ctx->H(0), y.ldi, ctx->at<float>(p.o_P), y.ldi, y.fi, nullptr, bf16_of(ctx), ctx->stream); });
                 ctx->P_valid = true;
             }
             const ActEpi act = make_act(ep, 0);
@@ -348,7 +353,7 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
                                          ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr, ctx->stream);
         });
         GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
-                [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, ctx->stream); });
+                [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, bf16_of(ctx), ctx->stream); });
     }
     ctx->acts_valid = true;
     return GAD_OK;
@@ -420,7 +425,7 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
         const bool agg_first = l == 0 && p.agg_first0;   // then dW = (A~ X)^T dPre and nothing flows further back
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
-                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, ctx->stream); });
+                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, bf16_of(ctx), ctx->stream); });
         if (ctx->use_tc && p.narrow[l]) {
             // one pass over H^(l) and dZ gives both dW and dPre of the layer below (it writes G1: the column sums come first)
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));

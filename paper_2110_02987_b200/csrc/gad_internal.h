@@ -126,8 +126,10 @@ inline ActEpi make_act(const Epilogue& e, int col0) {
 // ---------------------------------------------------------------------------------------------
 // Kernel launchers (each enqueues on `s` and returns the cudaGetLastError of its launches)
 // ---------------------------------------------------------------------------------------------
+// bf16_scratch: null, or device room for nrows x ldz bfloat16 values: the operand is then copied there in bfloat16 and
+// gathered from the copy (reduced-precision mode).
 cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F,
-                        const Epilogue* epi, cudaStream_t s);
+                        const Epilogue* epi, void* bf16_scratch, cudaStream_t s);
 
 // mode 0: C = A * W_k (W row-major [Kd x N], ld ldw); mode 1: C = (A * W_k^T) masked by Hmask > 0, scaled
 // (W row-major [N x Kd]); mode 2: C = sigma(A * W_k + b_k) with dropout as `act` says.  Tiles never cross a subgraph.

@@ -21,6 +21,20 @@ __device__ __forceinline__ int find_sub(const int32_t* __restrict__ sub_off, int
     return lo;
 }
 
+// Four consecutive operand values at p: fp32 (16 bytes), or with BF bfloat16 (8 bytes, value i in bits 16 i .. 16 i + 15),
+// widened to fp32.  The bfloat16 copy of the operand is what the reduced-precision mode gathers: half the bytes per entry.
+template <bool BF>
+__device__ __forceinline__ float4 load_row4(const char* p) {
+    if constexpr (BF) {
+        const uint2 u = __ldg(reinterpret_cast<const uint2*>(p));
+        return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                           __uint_as_float(u.y & 0xffff0000u));
+    } else {
+        return __ldg(reinterpret_cast<const float4*>(p));
+    }
+}
+template <bool BF> struct OpBytes { static constexpr uint32_t elem = BF ? 2u : 4u, quad = BF ? 8u : 16u; };
+
 struct EpiDev {
     ActEpi act;
     const int32_t* sub_off;
@@ -72,7 +86,7 @@ __device__ __forceinline__ Item load_item(const int4* __restrict__ items, int id
 constexpr int kNarrowBatch = GAD_SPMM_NBATCH;
 template <int GROUP> struct NarrowCfg { static constexpr int EPL = kNarrowBatch / GROUP > 0 ? kNarrowBatch / GROUP : 1; };
 
-template <int GROUP, int NB>
+template <int GROUP, int NB, bool BF>
 __device__ __forceinline__ void narrow_batch(float4& acc, const uint2 (&mine)[NarrowCfg<GROUP>::EPL], unsigned gmask,
                                              const char* zl, uint32_t ldzb) {
     float4 z[NB];
@@ -81,7 +95,7 @@ __device__ __forceinline__ void narrow_batch(float4& acc, const uint2 (&mine)[Na
     for (int t = 0; t < NB; ++t) {
         const uint32_t c = __shfl_sync(gmask, mine[t / GROUP].x, t % GROUP, GROUP);
         a[t] = __uint_as_float(__shfl_sync(gmask, mine[t / GROUP].y, t % GROUP, GROUP));
-        z[t] = __ldg(reinterpret_cast<const float4*>(zl + (unsigned long long)c * ldzb));
+        z[t] = load_row4<BF>(zl + (unsigned long long)c * ldzb);
     }
 #pragma unroll
     for (int t = 0; t < NB; ++t) {
@@ -92,7 +106,7 @@ __device__ __forceinline__ void narrow_batch(float4& acc, const uint2 (&mine)[Na
     }
 }
 
-template <int GROUP, bool EPI>
+template <int GROUP, bool EPI, bool BF>
 __global__ void __launch_bounds__(256, GAD_SPMM_NMINB)
 spmm_items_narrow_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z, int ldz,
                          float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
@@ -103,8 +117,8 @@ spmm_items_narrow_kernel(const uint2* __restrict__ ecv, const int4* __restrict__
     if (idx >= nitems) return;   // the whole group leaves together
     const Item it = load_item(items, (int)idx, ecv);
     const uint2 pad = make_uint2((uint32_t)it.row, 0u);
-    const char* zl = reinterpret_cast<const char*>(Z) + 16ll * min(gl, F4 - 1);   // lanes past the last column read it again
-    const uint32_t ldzb = 4u * (uint32_t)ldz;
+    const char* zl = reinterpret_cast<const char*>(Z) + (long long)OpBytes<BF>::quad * min(gl, F4 - 1);   // lanes past the last column read it again
+    const uint32_t ldzb = OpBytes<BF>::elem * (uint32_t)ldz;
     float4 acc[1] = {make_float4(0.f, 0.f, 0.f, 0.f)};
     uint2 next[EPL];
 #pragma unroll
@@ -120,8 +134,8 @@ spmm_items_narrow_kernel(const uint2* __restrict__ ecv, const int4* __restrict__
             const int e = gl + GROUP * i;
             next[i] = (e < NB && b + NB + e < it.len) ? __ldg(it.ent + b + NB + e) : pad;
         }
-        if (it.len - b > NB / 2) narrow_batch<GROUP, NB>(acc[0], mine, gmask, zl, ldzb);
-        else narrow_batch<GROUP, NB / 2>(acc[0], mine, gmask, zl, ldzb);
+        if (it.len - b > NB / 2) narrow_batch<GROUP, NB, BF>(acc[0], mine, gmask, zl, ldzb);
+        else narrow_batch<GROUP, NB / 2, BF>(acc[0], mine, gmask, zl, ldzb);
     }
     if (it.slot >= 0) {
         if (gl < F4) reinterpret_cast<float4*>(scratch + (long long)it.slot * ldo)[gl] = acc[0];
@@ -173,20 +187,20 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
 // next smaller power of two, so a batch costs at most one round trip more than its full groups.
 // Where a lane finds its 16 bytes of operand row c: operand start + c * (row stride in bytes) + the lane's column
 // offset.  With OFF32 the whole operand is smaller than 4 GiB and the offset is formed in 32 bits by one multiply-add.
-template <int NV, bool OFF32>
+template <int NV, bool OFF32, bool BF>
 struct ZLane {
     const char* base;      // OFF32: start of the operand (the same for the whole warp)
     const char* ptr[NV];   // otherwise: start of the operand plus the lane's column offset
     uint32_t off[NV];
     uint32_t ldzb;
     __device__ __forceinline__ float4 load(uint32_t c, int j) const {
-        if constexpr (OFF32) return __ldg(reinterpret_cast<const float4*>(base + (c * ldzb + off[j])));
-        else return __ldg(reinterpret_cast<const float4*>(ptr[j] + (unsigned long long)c * ldzb));
+        if constexpr (OFF32) return load_row4<BF>(base + (c * ldzb + off[j]));
+        else return load_row4<BF>(ptr[j] + (unsigned long long)c * ldzb);
     }
 };
 
-template <int NV, int UU, bool OFF32>
-__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const ZLane<NV, OFF32>& zl) {
+template <int NV, int UU, bool OFF32, bool BF>
+__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const ZLane<NV, OFF32, BF>& zl) {
     uint32_t c[UU];
     float a[UU];
     if constexpr (UU == 1) {
@@ -216,11 +230,11 @@ __device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, c
         }
 }
 
-template <int NV, int V, bool OFF32>
-__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const ZLane<NV, OFF32>& zl) {
+template <int NV, int V, bool OFF32, bool BF>
+__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const ZLane<NV, OFF32, BF>& zl) {
     if constexpr (V >= 1) {
-        if (r > V / 2) gather_fma<NV, V, OFF32>(acc, st, zl);
-        else gather_tail<NV, V / 2, OFF32>(acc, st, r, zl);
+        if (r > V / 2) gather_fma<NV, V, OFF32, BF>(acc, st, zl);
+        else gather_tail<NV, V / 2, OFF32, BF>(acc, st, r, zl);
     }
 }
 
@@ -244,7 +258,7 @@ template <int NV> struct ItemCfg {
     static constexpr int MINB = NV == 1 ? GAD_SPMM_MINB1 : (NV == 2 ? GAD_SPMM_MINB2 : (NV <= 4 ? 6 : 4));   // CTAs of 4 warps per SM
 };
 
-template <int NV, bool EPI, bool OFF32>
+template <int NV, bool EPI, bool OFF32, bool BF>
 __global__ void __launch_bounds__(32 * kItemWarps, ItemCfg<NV>::MINB)
 spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z,
                   int ldz, float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
@@ -259,12 +273,12 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
     const uint2* ent = item.ent;
     const uint2 pad = make_uint2((uint32_t)row, 0u);
     // lanes past the last column read the last one (their sums are never stored)
-    ZLane<NV, OFF32> zl;
+    ZLane<NV, OFF32, BF> zl;
     zl.base = reinterpret_cast<const char*>(Z);
-    zl.ldzb = 4u * (uint32_t)ldz;
+    zl.ldzb = OpBytes<BF>::elem * (uint32_t)ldz;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-        zl.off[j] = 16u * (uint32_t)min(lane + 32 * j, F4 - 1);
+        zl.off[j] = OpBytes<BF>::quad * (uint32_t)min(lane + 32 * j, F4 - 1);
         zl.ptr[j] = zl.base + zl.off[j];
     }
     float4 acc[NV];
@@ -280,8 +294,8 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
         stage[lane] = mine;
         __syncwarp();
         int t = 0;
-        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU, OFF32>(acc, stage + t, zl);
-        gather_tail<NV, UU / 2, OFF32>(acc, stage + t, cnt - t, zl);
+        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU, OFF32, BF>(acc, stage + t, zl);
+        gather_tail<NV, UU / 2, OFF32, BF>(acc, stage + t, cnt - t, zl);
     }
     if (item.slot >= 0) {
 #pragma unroll
@@ -294,17 +308,17 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
     }
 }
 
-template <int NV, int GROUP, bool EPI>
+template <int NV, int GROUP, bool EPI, bool BF>
 static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F4, const EpiDev& ep,
                                cudaStream_t s) {
     if constexpr (GROUP == 32) {
         if (A.nitems > 0) {
             const unsigned grid = (unsigned)((A.nitems + kItemWarps - 1) / kItemWarps);
             // every byte of the operand within 4 GiB of its start: 32-bit offsets
-            if ((unsigned long long)A.nrows * 4ull * (unsigned long long)ldz < (1ull << 32))
-                spmm_items_kernel<NV, EPI, true><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+            if ((unsigned long long)A.nrows * (unsigned long long)OpBytes<BF>::elem * (unsigned long long)ldz < (1ull << 32))
+                spmm_items_kernel<NV, EPI, true, BF><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
             else
-                spmm_items_kernel<NV, EPI, false><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+                spmm_items_kernel<NV, EPI, false, BF><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
             ++g_kernel_launches;
         }
         if (A.nfin > 0) {
@@ -315,7 +329,7 @@ static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, floa
     }
     if (A.nitems > 0) {
         const unsigned grid = (unsigned)(((long long)A.nitems * GROUP + 255) / 256);
-        spmm_items_narrow_kernel<GROUP, EPI><<<grid, 256, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+        spmm_items_narrow_kernel<GROUP, EPI, BF><<<grid, 256, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
         ++g_kernel_launches;
     }
     if (A.nfin > 0) {
@@ -325,11 +339,11 @@ static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, floa
     return cudaGetLastError();
 }
 
-template <bool EPI>
+template <bool EPI, bool BF>
 static cudaError_t dispatch(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F4, const EpiDev& ep,
                             cudaStream_t s) {
     cudaError_t e;
-#define GAD_ROWS(NV, G) { e = launch_rows<NV, G, EPI>(A, Z, ldz, out, ldo, F4, ep, s); if (e != cudaSuccess) return e; }
+#define GAD_ROWS(NV, G) { e = launch_rows<NV, G, EPI, BF>(A, Z, ldz, out, ldo, F4, ep, s); if (e != cudaSuccess) return e; }
     if (F4 <= 4) GAD_ROWS(1, 4) else if (F4 <= 8) GAD_ROWS(1, 8) else if (F4 <= 16) GAD_ROWS(1, 16)
     else if (F4 <= 32) GAD_ROWS(1, 32) else if (F4 <= 64) GAD_ROWS(2, 32) else if (F4 <= 96) GAD_ROWS(3, 32)
     else if (F4 <= 128) GAD_ROWS(4, 32) else if (F4 <= 160) GAD_ROWS(5, 32) else if (F4 <= 192) GAD_ROWS(6, 32)
@@ -338,10 +352,32 @@ static cudaError_t dispatch(const SparseDev& A, const float* Z, int ldz, float* 
     return cudaSuccess;
 }
 
+// fp32 -> bfloat16 (round to nearest even; NaN stays NaN), four values per thread.
+__global__ void __launch_bounds__(256) to_bf16_kernel(const float4* __restrict__ in, uint2* __restrict__ out, long long n4) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    const float4 v = in[i];
+    auto cvt = [](float x) -> uint32_t {
+        const uint32_t b = __float_as_uint(x);
+        if ((b & 0x7fffffffu) > 0x7f800000u) return (b >> 16) | 0x40u;   // NaN: keep it quiet
+        return (b + 0x7fffu + ((b >> 16) & 1u)) >> 16;
+    };
+    out[i] = make_uint2(cvt(v.x) | (cvt(v.y) << 16), cvt(v.z) | (cvt(v.w) << 16));
+}
+
 // F up to 1024 columns per pass (8 float4 per lane); wider operands are processed in column slabs.
+// With `bf16_scratch` (room for nrows x ldz bfloat16) the operand is first copied there in bfloat16 and gathered from
+// that copy: the reduced-precision mode, in which the gather moves half the bytes.
 cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F, const Epilogue* epi,
-                        cudaStream_t s) {
+                        void* bf16_scratch, cudaStream_t s) {
     const int F4_all = (int)(round_up(F, 4) / 4);
+    if (bf16_scratch && A.nrows > 0) {
+        const long long n4 = (long long)A.nrows * (ldz / 4);
+        to_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float4*>(Z), reinterpret_cast<uint2*>(bf16_scratch), n4);
+        ++g_kernel_launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     for (int c0 = 0; c0 < F4_all; c0 += 256) {
         const int F4 = min(256, F4_all - c0);
         EpiDev ep{};
@@ -349,8 +385,15 @@ cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out,
             ep.act = make_act(*epi, 4 * c0);
             ep.sub_off = epi->sub_off; ep.K = epi->K;
         }
-        cudaError_t e = epi ? dispatch<true>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s)
-                            : dispatch<false>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s);
+        cudaError_t e;
+        if (bf16_scratch) {
+            // the kernels take the operand as a float pointer and read it through byte offsets: 4 c0 bfloat16 = 2 c0 floats
+            const float* Zb = reinterpret_cast<const float*>(bf16_scratch) + 2 * c0;
+            e = epi ? dispatch<true, true>(A, Zb, ldz, out + 4 * c0, ldo, F4, ep, s) : dispatch<false, true>(A, Zb, ldz, out + 4 * c0, ldo, F4, ep, s);
+        } else {
+            e = epi ? dispatch<true, false>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s)
+                    : dispatch<false, false>(A, Z + 4 * c0, ldz, out + 4 * c0, ldo, F4, ep, s);
+        }
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

@@ -574,3 +574,25 @@ def test_epochs_replayed_as_a_graph_equal_epochs_enqueued_one_by_one(dims, zeta_
             g.set_inputs(X2); h.set_inputs(X2)
             assert np.array_equal(g.train_epoch(), h.train_epoch())
             assert np.array_equal(g.get_params(0), h.get_params(0))
+
+
+def test_reduced_precision_mode_on_a_power_law_graph():
+    """gemm_mode 1 (one TF32 pass per transform, the aggregation gathering a bfloat16 copy of its operand) on a scaled
+    c2: hub rows cut into parts, wide and narrow aggregations, graph replay.  Bar of this mode: 5e-2."""
+    import torch
+    w = make_workload("c2", scale=0.2)
+    theta = glorot_params(w.dims, np.random.default_rng(0), bias_scale=0.1)
+    ref = orc().from_workload(w, theta, lr=0.5)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        with pkg().from_workload(w, theta, lr=0.5, gemm_mode=1, stream=stream) as g:
+            for _ in range(3):
+                lg, lr = g.train_epoch(), ref.train_epoch()
+                assert np.max(np.abs(lg - lr)) <= 5e-2
+            L = len(w.dims) - 1
+            assert rel_err(g.get_activation(L), ref.activation(L)) <= 5e-2
+            for k in range(g.K):
+                assert rel_err(g.get_grads(k), ref.get_grads(k)) <= 5e-2
+                assert rel_err(g.get_params(k), ref.get_params(k)) <= 5e-2
+            # and it is not the fp32 path in disguise: the rounding of the operands shows
+            assert rel_err(g.get_activation(L), ref.activation(L)) > 1e-5
