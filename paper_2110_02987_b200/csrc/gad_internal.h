@@ -43,7 +43,7 @@ int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_
 
 // Work lists of the SpMM launch (host side).  A row of at most `part_entries` entries is one item; a longer row is
 // cut into parts of `part_entries` entries, each an item with a scratch slot of its own, and gets an entry
-// fin = {row, first scratch slot, slots, 0}.  The part length starts at kMinPart and doubles (up to kMaxPart)
+// fin = {row, first scratch slot, slots, subgraph of the row}.  The part length starts at kMinPart and doubles (up to kMaxPart)
 // until the cut rows need at most one scratch slot per two store rows; a row that would still need more than
 // kMaxSlotsPerRow parts gets longer parts of its own.
 // items = {row, low 32 bits of the first entry's position in the store, (high bits << 16) | entries, scratch slot

@@ -43,9 +43,9 @@ struct EpiDev {
 
 template <int NV, bool EPI>
 __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, int group, int F4, float* __restrict__ out,
-                                           int ldo, const EpiDev& ep) {
+                                           int ldo, const EpiDev& ep, int known_k = -1) {
     if (EPI) {
-        const int k = find_sub(ep.sub_off, ep.K, row);
+        const int k = known_k >= 0 ? known_k : find_sub(ep.sub_off, ep.K, row);   // the list of cut rows carries the subgraph
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
             const int v = gl + group * j;
@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
     const int lane = threadIdx.x & 31;
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (i >= nfin || lane >= GROUP) return;
-    const int4 f = fin[i];  // {row, first slot, slots, unused}
+    const int4 f = fin[i];  // {row, first slot, slots, subgraph of the row}
     float4 acc[NV];
 #pragma unroll
     for (int j = 0; j < NV; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
                 acc[j].x += t[q][j].x; acc[j].y += t[q][j].y; acc[j].z += t[q][j].z; acc[j].w += t[q][j].w;
             }
     }
-    finish_row<NV, EPI>(acc, f.x, lane, GROUP, F4, out, ldo, ep);
+    finish_row<NV, EPI>(acc, f.x, lane, GROUP, F4, out, ldo, ep, f.w);
 }
 
 // ---- operands wider than 64 columns: one warp per item of the unified list (a whole row or a part of a cut row) ----

@@ -277,7 +277,7 @@ void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& su
         if (len <= part) { out.perm[(size_t)start[bin_of(len)]++] = (int32_t)r; continue; }
         const int64_t pl = row_part_entries(len, part);
         const int64_t np = (len + pl - 1) / pl;
-        out.fin.push_back(make_int4((int)r, (int)out.slots, (int)np, 0));
+        out.fin.push_back(make_int4((int)r, (int)out.slots, (int)np, 0));   // the subgraph is filled in below
         for (int64_t q = 0; q < np; ++q)
             out.parts.push_back(make_int4((int)r, (int)(q * pl), (int)std::min(pl, len - q * pl), (int)(out.slots + q)));
         out.slots += np;
@@ -291,6 +291,7 @@ void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& su
     std::vector<int32_t> sub_of((size_t)Np);
     for (int64_t k = 0; k < K; ++k)
         for (int64_t r = sub_off[k]; r < sub_off[k + 1]; ++r) sub_of[(size_t)r] = (int32_t)k;
+    for (int4& f : out.fin) f.w = sub_of[(size_t)f.x];
     auto key = [&](int64_t row, int64_t len) { return (size_t)(sub_of[(size_t)row] * 64 + (63 - bin_of(len))); };
     std::vector<int64_t> istart((size_t)K * 64 + 1, 0);
     for (const int4& pt : out.parts) istart[key(pt.x, pt.z) + 1]++;
