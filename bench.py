@@ -258,6 +258,47 @@ def run_micro_consensus(args):
     print(json.dumps(line))
 
 
+def run_micro_augment(args):
+    """Importance-based augmentation (Algorithm 1) of the benchmark graph's partition: gad_augment end to end (graph
+    upload, boundary test, walks, counts, scores on the GPU; ranking and selection on the host), and the oracle on a
+    small sample of the same recipe.  One JSON line."""
+    import torch
+    import __graft_entry__ as entry
+    from gad_synth import make_workload
+    from gad_synth.partition import bfs_partition
+    import paper_2110_02987_b200 as pkg
+    if not os.path.exists(pkg.LIB_PATH):
+        entry.build()
+    torch.cuda.set_device(0)
+    w = make_workload(args.workload, **args.wl_kw)
+    steps = len(w.dims) - 1
+    kw = dict(alpha=0.01, E=0.05, zc=1.96, seed=0, cap=4)
+    for _ in range(2):
+        halos, walks = pkg.augment(w.n, w.rowptr, w.col, w.core, steps, **kw)
+    torch.cuda.synchronize()
+    reps = max(1, min(args.steps or 5, 20))
+    l0 = pkg.launch_count()
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        halos, walks = pkg.augment(w.n, w.rowptr, w.col, w.core, steps, **kw)
+    dt = (time.perf_counter() - t0) / reps
+    launches = (pkg.launch_count() - l0) // reps
+    line = {"micro": "augment", "workload": describe(w), "steps": steps, "walks": int(walks.sum()), "replication_nodes": int(sum(len(h) for h in halos)),
+            "ms": 1e3 * dt, "walks_per_s": float(walks.sum()) / dt, "gpu_launches": int(launches),
+            "note": "whole call: host-to-device copy of the graph, GPU kernels, host ranking and selection; bound by the latency "
+                    "of dependent random reads (a walk is steps + 1 dependent row look-ups)"}
+    if not args.no_cpu_baseline:
+        from oracle import augment_oracle as aug
+        small = make_workload(args.workload, scale=0.02) if args.workload != "tiny" else w
+        cores = bfs_partition(small.rowptr, small.col, 4)
+        t0 = time.perf_counter()
+        _, info = aug.augment(small.n, small.rowptr, small.col, cores, steps, **kw)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sum(it["n"] for it in info) / dt, "unit": "walks/s", "cores": 1, "kind": "oracle",
+                                "sample": "the same recipe at scale 0.02 with 4 breadth-first blocks (%d walks)" % sum(it["n"] for it in info)}
+    print(json.dumps(line))
+
+
 def run_sharded(args, w, theta, rank, world, local_rank):
     """Algorithm 2's deployment shape: the K subgraphs spread over the ranks, every rank a context with its share,
     one all-reduce (NCCL) of the consensus buffer per epoch.  Strong scaling: the whole job is K subgraphs however
@@ -346,8 +387,9 @@ def main():
     ap.add_argument("--kernels", action="store_true", help="also print the per-kernel table to stderr")
     ap.add_argument("--shard", action="store_true",
                     help="spread the K subgraphs over the ranks (one all-reduce per epoch) instead of running N replicas of the job")
-    ap.add_argument("--micro", default=None, choices=["consensus"],
-                    help="a single-kernel point instead of the epoch benchmark (consensus: K = 8 copies of a 4096 x 4096 layer)")
+    ap.add_argument("--micro", default=None, choices=["consensus", "augment"],
+                    help="a single point instead of the epoch benchmark (consensus: K = 8 copies of a 4096 x 4096 layer; "
+                         "augment: Algorithm 1 on the workload's partition)")
     args = ap.parse_args()
     if args.micro == "consensus":
         run_micro_consensus(args)
@@ -358,6 +400,9 @@ def main():
     args.wl_kw = {"scale": args.scale}
     if args.workload == "sweep":
         args.wl_kw.update(mean_deg=args.mean_deg, F=args.F, K=args.K)
+    if args.micro == "augment":
+        run_micro_augment(args)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

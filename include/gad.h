@@ -261,6 +261,39 @@ int gad_subgraph_weights_static(const float* X, int64_t rows, int32_t F, int32_t
                                 const int32_t* sub_off, int32_t K, float beta, int32_t weighted, float* zeta_out,
                                 float* w_out, void* stream);
 
+/* ---- Importance-based subgraph augmentation (Algorithm 1, Section 3.2.2) -----------------------------------------
+ * Produces the replication-node lists that gad_create takes as halo_nodes, from a partition of G into K core sets:
+ * for every subgraph, random walks of `steps` steps (the number of GCN layers, Property 1) start at uniformly drawn
+ * boundary nodes; count[v] = walks that contain the outside node v (importance equation, I(v) = count[v] / n); after the
+ * first d |B| walks (d = average degree of the boundary nodes) the number of walks n follows the Monte-Carlo error
+ * equation, n = (zc sigma / (mean E))^2, at most cap times the first batch; walks are ranked by the sum of I over
+ * their outside nodes and their nodes are taken in walk order until alpha (1 + density) |v_i| nodes are selected.
+ * The boundary test, the walks, the counts, their statistics and the walk scores run on the GPU; the ranking and
+ * the selection loop on the host.  Every random number is mix(seed, subgraph, walk, step) (splitmix64 output
+ * function), so the result is a pure function of the arguments. */
+typedef struct {
+    int32_t steps;   /* walk length l = number of GCN layers, 1 .. 8                                      */
+    int32_t cap;     /* at most cap times the first batch of walks (>= 1)                                  */
+    double alpha;    /* replication constant of n(g_i) = alpha (1 + d(g_i)) |v_i|; the paper uses 0.01     */
+    double E;        /* Monte-Carlo error bound; the paper uses 0.05                                       */
+    double zc;       /* confidence statistic; 1.96 for the paper's 95 % level                              */
+    uint64_t seed;
+} gad_augment_config;
+
+/* Bytes of device workspace gad_augment needs.  Host-only. */
+int gad_augment_workspace_bytes(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int32_t* core_nodes,
+                                const gad_augment_config* cfg, size_t* bytes);
+
+/* g (its weights are ignored), core_ptr [K+1], core_nodes: host.  workspace: device, 256-byte aligned, owned by the
+ * caller.  Outputs, host: halo_ptr [K+1]; halo_nodes [halo_capacity], subgraph k's replication nodes in selection order
+ * at halo_ptr[k] .. halo_ptr[k+1]-1 (GAD_ERR_OOM if the capacity is too small: sum_k alpha (1 + d_k) |v_k| always
+ * suffices); walks_out [K] = walks drawn per subgraph, or NULL.  Waits for the stream.  After an error
+ * gad_augment_last_error gives the message of the calling thread. */
+int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int32_t* core_nodes, const gad_augment_config* cfg,
+                void* workspace, size_t workspace_bytes, void* stream, int64_t* halo_ptr, int32_t* halo_nodes,
+                int64_t halo_capacity, int64_t* walks_out);
+const char* gad_augment_last_error(void);
+
 /* Number of CUDA kernels this library has launched in this process so far (all contexts). */
 int gad_launch_count(int64_t* launches);
 

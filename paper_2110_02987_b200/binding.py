@@ -26,7 +26,8 @@ SYMBOLS = (
     "gad_get_store", "gad_get_activation", "gad_set_inputs", "gad_read_loss_async", "gad_synchronize", "gad_get_epoch", "gad_set_epoch", "gad_profile_enable",
     "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_subgraph_weights_static", "gad_launch_count",
     "gad_last_error", "gad_destroy", "gad_train_epoch_local", "gad_consensus_floats", "gad_consensus_partial",
-    "gad_consensus_apply", "gad_export_params", "gad_get_train_counts",
+    "gad_consensus_apply", "gad_export_params", "gad_get_train_counts", "gad_augment_workspace_bytes", "gad_augment",
+    "gad_augment_last_error",
 )
 
 
@@ -389,6 +390,46 @@ def launch_count() -> int:
     if rc != GAD_OK:
         raise GadError(rc)
     return int(n.value)
+
+
+class _AugmentConfig(C.Structure):
+    _fields_ = [("steps", C.c_int32), ("cap", C.c_int32), ("alpha", C.c_double), ("E", C.c_double), ("zc", C.c_double),
+                ("seed", C.c_uint64)]
+
+
+def augment(n, rowptr, col, cores, steps, *, alpha=0.01, E=0.05, zc=1.96, seed=0, cap=4, stream=None):
+    """gad_augment: the replication-node list of every core set (Algorithm 1 of the paper) on the current CUDA device.
+    Returns (list of int32 arrays in selection order, int64 array of the walks drawn per subgraph)."""
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("the GAD library needs a CUDA device (there is no CPU fallback)")
+    L = load()
+    L.gad_augment_last_error.restype = C.c_char_p
+    rowptr = _arr(rowptr, np.int64)
+    col = _arr(col, np.int32)
+    K = len(cores)
+    cp = np.zeros(K + 1, dtype=np.int64)
+    np.cumsum([len(c) for c in cores], out=cp[1:])
+    cn = _arr(np.concatenate(cores) if cp[-1] > 0 else np.empty(0, np.int32), np.int32)
+    csr = gad_csr(int(n), int(rowptr[-1]), _ptr(rowptr, C.c_int64), _ptr(col, C.c_int32), None)
+    cfg = _AugmentConfig(int(steps), int(cap), float(alpha), float(E), float(zc), int(seed))
+    nbytes = C.c_size_t(0)
+    rc = L.gad_augment_workspace_bytes(C.byref(csr), C.c_int32(K), _ptr(cp, C.c_int64), _ptr(cn, C.c_int32), C.byref(cfg), C.byref(nbytes))
+    if rc != GAD_OK:
+        raise GadError(rc, (L.gad_augment_last_error() or b"").decode())
+    ws = torch.empty(int(nbytes.value) + 256, dtype=torch.uint8, device="cuda")
+    aligned = (ws.data_ptr() + 255) // 256 * 256
+    st = stream if stream is not None else torch.cuda.current_stream()
+    capacity = int(sum(int(np.floor(alpha * 2.0 * len(c))) for c in cores)) + 1
+    halo_ptr = np.zeros(K + 1, dtype=np.int64)
+    halo = np.zeros(capacity, dtype=np.int32)
+    walks = np.zeros(K, dtype=np.int64)
+    rc = L.gad_augment(C.byref(csr), C.c_int32(K), _ptr(cp, C.c_int64), _ptr(cn, C.c_int32), C.byref(cfg), C.c_void_p(aligned),
+                       C.c_size_t(int(nbytes.value)), C.c_void_p(st.cuda_stream), _ptr(halo_ptr, C.c_int64), _ptr(halo, C.c_int32),
+                       C.c_int64(capacity), _ptr(walks, C.c_int64))
+    if rc != GAD_OK:
+        raise GadError(rc, (L.gad_augment_last_error() or b"").decode())
+    return [halo[halo_ptr[k]:halo_ptr[k + 1]].copy() for k in range(K)], walks
 
 
 def from_workload(w, init_params, **kw):

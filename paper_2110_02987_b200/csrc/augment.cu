@@ -1,0 +1,303 @@
+// Importance-based subgraph augmentation (Algorithm 1 of the paper, Section 3.2.2): for every subgraph of a
+// partition, Monte-Carlo random walks from its boundary nodes estimate how often each outside node is reached
+// (importance equation), the number of walks follows the Monte-Carlo error equation, and the replication nodes are
+// taken walk by walk in descending order of the walks' summed importance until the density-sized number n(g_i) is
+// reached.  Its output (the replication-node lists) is what gad_create takes as `halo_nodes`.
+//
+// On the GPU: the boundary test, the walks with their visit counts, the count statistics and the walk scores, all in
+// integers (the same draws, counts and scores as a CPU evaluation: every random number is a pure function
+// mix(seed, subgraph, walk, step) of the splitmix64 output function).  Walks are never stored: the scoring kernel and
+// the host's selection loop regenerate them from the generator.  On the host: the boundary list, the number of walks
+// from the integer sums, the ranking of the walks and the selection loop, which is sequential by definition.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <numeric>
+#include <string>
+#include <vector>
+
+#include "gad_internal.h"
+
+namespace gad {
+
+namespace {
+
+constexpr int kMaxSteps = 8;
+
+__host__ __device__ inline uint64_t aug_mix64(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ULL;
+    z = (z ^ (z >> 27)) * 0x94d049bb133111ebULL;
+    return z ^ (z >> 31);
+}
+// key of (seed, subgraph, walk); the step is mixed in per draw
+__host__ __device__ inline uint64_t walk_key(uint64_t seed, int sub, int64_t walk) {
+    const uint64_t G = 0x9e3779b97f4a7c15ULL;
+    const uint64_t h = aug_mix64(seed + G * (uint64_t)(1 + sub));
+    return aug_mix64(h + G * (uint64_t)(1 + walk));
+}
+__host__ __device__ inline uint64_t walk_draw(uint64_t key, int step) {
+    const uint64_t G = 0x9e3779b97f4a7c15ULL;
+    return aug_mix64(key + G * (uint64_t)(1 + step));
+}
+// The node sequence of one walk: start at a uniformly drawn boundary node, every step to a uniformly drawn neighbour.
+__host__ __device__ inline void make_walk(const int64_t* rowptr, const int32_t* col, const int32_t* B, int64_t nB, uint64_t seed, int sub,
+                                          int64_t walk, int steps, int32_t* seq) {
+    const uint64_t key = walk_key(seed, sub, walk);
+    int32_t cur = B[walk_draw(key, 0) % (uint64_t)nB];
+    seq[0] = cur;
+    for (int s = 1; s <= steps; ++s) {
+        const int64_t r0 = rowptr[cur], d = rowptr[cur + 1] - r0;
+        if (d > 0) cur = col[r0 + (int64_t)(walk_draw(key, s) % (uint64_t)d)];
+        seq[s] = cur;
+    }
+}
+// v is outside the subgraph and does not occur earlier in the walk
+__host__ __device__ inline bool first_outside(const uint8_t* inside, const int32_t* seq, int s) {
+    const int32_t v = seq[s];
+    if (inside[v]) return false;
+    for (int t = 0; t < s; ++t)
+        if (seq[t] == v) return false;
+    return true;
+}
+
+__global__ void boundary_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ core,
+                                int64_t ncore, const uint8_t* __restrict__ inside, uint8_t* __restrict__ flag) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= ncore) return;
+    const int32_t v = core[t];
+    uint8_t f = 0;
+    for (int64_t e = rowptr[v]; e < rowptr[v + 1] && !f; ++e) f = inside[col[e]] ? 0 : 1;
+    flag[t] = f;
+}
+__global__ void mark_kernel(const int32_t* __restrict__ core, int64_t ncore, uint8_t* __restrict__ inside, uint8_t value) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < ncore) inside[core[t]] = value;
+}
+__global__ void walk_count_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ B,
+                                  int64_t nB, const uint8_t* __restrict__ inside, uint64_t seed, int sub, int64_t j0, int64_t j1,
+                                  int steps, int32_t* __restrict__ count) {
+    const int64_t j = j0 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= j1) return;
+    int32_t seq[kMaxSteps + 1];
+    make_walk(rowptr, col, B, nB, seed, sub, j, steps, seq);
+    for (int s = 0; s <= steps; ++s)
+        if (first_outside(inside, seq, s)) atomicAdd(count + seq[s], 1);   // integer: the result does not depend on the order
+}
+__global__ void walk_score_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ B,
+                                  int64_t nB, const uint8_t* __restrict__ inside, uint64_t seed, int sub, int64_t nwalks, int steps,
+                                  const int32_t* __restrict__ count, int64_t* __restrict__ score) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= nwalks) return;
+    int32_t seq[kMaxSteps + 1];
+    make_walk(rowptr, col, B, nB, seed, sub, j, steps, seq);
+    int64_t sc = 0;
+    for (int s = 0; s <= steps; ++s)
+        if (first_outside(inside, seq, s)) sc += count[seq[s]];
+    score[j] = sc;
+}
+// m = visited candidates, S1 = sum of counts, S2 = sum of squared counts
+__global__ void count_stats_kernel(const int32_t* __restrict__ count, int64_t n, unsigned long long* __restrict__ stats) {
+    __shared__ unsigned long long sm[3][256];
+    unsigned long long m = 0, s1 = 0, s2 = 0;
+    for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < n; v += (int64_t)gridDim.x * blockDim.x) {
+        const unsigned long long c = (unsigned long long)count[v];
+        if (c) { ++m; s1 += c; s2 += c * c; }
+    }
+    sm[0][threadIdx.x] = m; sm[1][threadIdx.x] = s1; sm[2][threadIdx.x] = s2;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o)
+            for (int q = 0; q < 3; ++q) sm[q][threadIdx.x] += sm[q][threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0)
+        for (int q = 0; q < 3; ++q) atomicAdd(stats + q, sm[q][0]);
+}
+
+struct AugPlan { size_t o_rowptr, o_col, o_inside, o_core, o_flag, o_B, o_count, o_stats, o_score, bytes; int64_t max_core, max_walks; };
+
+size_t take(size_t& cur, size_t bytes) { size_t o = cur; cur += (size_t)round_up((int64_t)std::max<size_t>(bytes, 4), 256); return o; }
+
+int plan_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int32_t* core_nodes, const gad_augment_config* cfg, AugPlan& p,
+                 std::string& err) {
+    if (!g || !g->rowptr || (g->nnz > 0 && !g->col) || g->n < 0 || K < 1 || !core_ptr || !cfg) { err = "bad arguments"; return GAD_ERR_ARG; }
+    if (cfg->steps < 1 || cfg->steps > kMaxSteps) { err = "steps must be 1 .. 8"; return GAD_ERR_ARG; }
+    if (!(cfg->alpha >= 0.0) || !(cfg->E > 0.0) || !(cfg->zc > 0.0) || cfg->cap < 1) { err = "alpha >= 0, E > 0, zc > 0, cap >= 1"; return GAD_ERR_ARG; }
+    p.max_core = 0; p.max_walks = 1;
+    for (int32_t k = 0; k < K; ++k) {
+        if (core_ptr[k + 1] < core_ptr[k]) { err = "core_ptr decreases"; return GAD_ERR_UNSORTED; }
+        int64_t deg = 0;
+        for (int64_t t = core_ptr[k]; t < core_ptr[k + 1]; ++t) {
+            const int32_t v = core_nodes[t];
+            if (v < 0 || v >= g->n) { err = "core node out of range"; return GAD_ERR_RANGE; }
+            deg += g->rowptr[v + 1] - g->rowptr[v];
+        }
+        p.max_core = std::max(p.max_core, core_ptr[k + 1] - core_ptr[k]);
+        p.max_walks = std::max(p.max_walks, deg * (int64_t)cfg->cap);   // n0 is at most the subgraph's degree sum
+    }
+    size_t cur = 0;
+    p.o_rowptr = take(cur, 8 * (size_t)(g->n + 1)); p.o_col = take(cur, 4 * (size_t)g->nnz);
+    p.o_inside = take(cur, (size_t)g->n); p.o_core = take(cur, 4 * (size_t)p.max_core); p.o_flag = take(cur, (size_t)p.max_core);
+    p.o_B = take(cur, 4 * (size_t)p.max_core); p.o_count = take(cur, 4 * (size_t)g->n); p.o_stats = take(cur, 24);
+    p.o_score = take(cur, 8 * (size_t)p.max_walks);
+    p.bytes = cur;
+    return GAD_OK;
+}
+
+thread_local std::string g_aug_error;
+int aug_fail(int code, const std::string& msg) { g_aug_error = msg; return code; }
+
+#define AUG_CK(call)                                                                      \
+    do {                                                                                  \
+        cudaError_t e_ = (call);                                                          \
+        if (e_ != cudaSuccess) return aug_fail(GAD_ERR_CUDA, cudaGetErrorString(e_));     \
+    } while (0)
+
+}  // namespace
+
+const char* augment_last_error() { return g_aug_error.c_str(); }
+
+}  // namespace gad
+
+using namespace gad;
+
+extern "C" {
+
+int gad_augment_workspace_bytes(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int32_t* core_nodes,
+                                const gad_augment_config* cfg, size_t* bytes) {
+    if (!bytes) return GAD_ERR_ARG;
+    AugPlan p;
+    std::string err;
+    int rc = plan_augment(g, K, core_ptr, core_nodes, cfg, p, err);
+    if (rc != GAD_OK) return aug_fail(rc, err);
+    *bytes = p.bytes;
+    return GAD_OK;
+}
+
+int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int32_t* core_nodes, const gad_augment_config* cfg,
+                void* workspace, size_t workspace_bytes, void* stream_, int64_t* halo_ptr, int32_t* halo_nodes, int64_t halo_capacity,
+                int64_t* walks_out) {
+    if (!workspace || !halo_ptr || (halo_capacity > 0 && !halo_nodes) || ((uintptr_t)workspace & 255) != 0) return aug_fail(GAD_ERR_ARG, "bad arguments");
+    AugPlan p;
+    std::string err;
+    int rc = plan_augment(g, K, core_ptr, core_nodes, cfg, p, err);
+    if (rc != GAD_OK) return aug_fail(rc, err);
+    if (workspace_bytes < p.bytes) return aug_fail(GAD_ERR_OOM, "workspace smaller than gad_augment_workspace_bytes");
+    cudaStream_t s = (cudaStream_t)stream_;
+    char* ws = (char*)workspace;
+    int64_t* d_rowptr = (int64_t*)(ws + p.o_rowptr);
+    int32_t* d_col = (int32_t*)(ws + p.o_col);
+    uint8_t* d_inside = (uint8_t*)(ws + p.o_inside);
+    int32_t* d_core = (int32_t*)(ws + p.o_core);
+    uint8_t* d_flag = (uint8_t*)(ws + p.o_flag);
+    int32_t* d_B = (int32_t*)(ws + p.o_B);
+    int32_t* d_count = (int32_t*)(ws + p.o_count);
+    unsigned long long* d_stats = (unsigned long long*)(ws + p.o_stats);
+    int64_t* d_score = (int64_t*)(ws + p.o_score);
+    const int64_t n = g->n;
+    const int steps = cfg->steps;
+    AUG_CK(cudaMemcpyAsync(d_rowptr, g->rowptr, 8 * (size_t)(n + 1), cudaMemcpyHostToDevice, s));
+    if (g->nnz > 0) AUG_CK(cudaMemcpyAsync(d_col, g->col, 4 * (size_t)g->nnz, cudaMemcpyHostToDevice, s));
+    AUG_CK(cudaMemsetAsync(d_inside, 0, (size_t)n, s));
+    std::vector<uint8_t> inside((size_t)n, 0), flag;
+    std::vector<int32_t> B, seq((size_t)steps + 1);
+    std::vector<int64_t> score, order;
+    std::vector<uint8_t> taken((size_t)n, 0);
+    auto grid = [](int64_t work) { return (unsigned)((work + 255) / 256); };
+    int64_t out = 0;
+    halo_ptr[0] = 0;
+    for (int32_t k = 0; k < K; ++k) {
+        const int32_t* core = core_nodes + core_ptr[k];
+        const int64_t ncore = core_ptr[k + 1] - core_ptr[k];
+        int64_t nwalks = 0;
+        if (ncore > 0) {
+            AUG_CK(cudaMemcpyAsync(d_core, core, 4 * (size_t)ncore, cudaMemcpyHostToDevice, s));
+            mark_kernel<<<grid(ncore), 256, 0, s>>>(d_core, ncore, d_inside, 1); ++g_kernel_launches;
+            boundary_kernel<<<grid(ncore), 256, 0, s>>>(d_rowptr, d_col, d_core, ncore, d_inside, d_flag); ++g_kernel_launches;
+            flag.resize((size_t)ncore);
+            AUG_CK(cudaMemcpyAsync(flag.data(), d_flag, (size_t)ncore, cudaMemcpyDeviceToHost, s));
+            AUG_CK(cudaStreamSynchronize(s));
+            B.clear();
+            int64_t inner_directed = 0;
+            for (int64_t t = 0; t < ncore; ++t) inside[(size_t)core[t]] = 1;
+            for (int64_t t = 0; t < ncore; ++t) {
+                if (flag[(size_t)t]) B.push_back(core[t]);
+                for (int64_t e = g->rowptr[core[t]]; e < g->rowptr[core[t] + 1]; ++e)
+                    inner_directed += (inside[(size_t)g->col[e]] && g->col[e] != core[t]) ? 1 : 0;
+            }
+            std::sort(B.begin(), B.end());
+            const int64_t nB = (int64_t)B.size();
+            if (nB > 0) {
+                int64_t n0 = 0;
+                for (int32_t b : B) n0 += g->rowptr[b + 1] - g->rowptr[b];
+                AUG_CK(cudaMemcpyAsync(d_B, B.data(), 4 * (size_t)nB, cudaMemcpyHostToDevice, s));
+                AUG_CK(cudaMemsetAsync(d_count, 0, 4 * (size_t)n, s));
+                AUG_CK(cudaMemsetAsync(d_stats, 0, 24, s));
+                if (n0 > 0) {
+                    walk_count_kernel<<<grid(n0), 256, 0, s>>>(d_rowptr, d_col, d_B, nB, d_inside, cfg->seed, k, 0, n0, steps, d_count);
+                    ++g_kernel_launches;
+                }
+                count_stats_kernel<<<148 * 4, 256, 0, s>>>(d_count, n, d_stats); ++g_kernel_launches;
+                unsigned long long st[3];
+                AUG_CK(cudaMemcpyAsync(st, d_stats, 24, cudaMemcpyDeviceToHost, s));
+                AUG_CK(cudaStreamSynchronize(s));
+                // Monte-Carlo error equation with sigma / mean of the visit frequencies from the integer sums
+                nwalks = n0;
+                if (st[0] > 0) {
+                    const double ratio = ((double)st[0] * (double)st[2]) / ((double)st[1] * (double)st[1]) - 1.0;
+                    const int64_t want = ratio > 0.0 ? (int64_t)std::ceil((cfg->zc / cfg->E) * (cfg->zc / cfg->E) * ratio) : 0;
+                    nwalks = std::max(n0, std::min(want, (int64_t)cfg->cap * n0));
+                }
+                if (nwalks > p.max_walks) return aug_fail(GAD_ERR_OOM, "more walks than planned");
+                if (nwalks > n0) {
+                    walk_count_kernel<<<grid(nwalks - n0), 256, 0, s>>>(d_rowptr, d_col, d_B, nB, d_inside, cfg->seed, k, n0, nwalks, steps, d_count);
+                    ++g_kernel_launches;
+                    AUG_CK(cudaMemsetAsync(d_stats, 0, 24, s));
+                    count_stats_kernel<<<148 * 4, 256, 0, s>>>(d_count, n, d_stats); ++g_kernel_launches;
+                    AUG_CK(cudaMemcpyAsync(st, d_stats, 24, cudaMemcpyDeviceToHost, s));
+                }
+                if (nwalks > 0) {
+                    walk_score_kernel<<<grid(nwalks), 256, 0, s>>>(d_rowptr, d_col, d_B, nB, d_inside, cfg->seed, k, nwalks, steps, d_count, d_score);
+                    ++g_kernel_launches;
+                }
+                score.resize((size_t)nwalks);
+                if (nwalks > 0) AUG_CK(cudaMemcpyAsync(score.data(), d_score, 8 * (size_t)nwalks, cudaMemcpyDeviceToHost, s));
+                AUG_CK(cudaStreamSynchronize(s));
+                // n(g_i) = alpha (1 + d(g_i)) |v_i|, at most the visited candidates
+                int64_t n_rep = 0;
+                if (ncore >= 2) {
+                    const double dens = (double)inner_directed / ((double)ncore * (double)(ncore - 1));
+                    n_rep = (int64_t)std::floor(cfg->alpha * (1.0 + dens) * (double)ncore);
+                }
+                n_rep = std::min<int64_t>(n_rep, (int64_t)st[0]);
+                // walks in descending order of their summed importance (equal scores: ascending index)
+                order.resize((size_t)nwalks);
+                std::iota(order.begin(), order.end(), (int64_t)0);
+                std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return score[(size_t)a] > score[(size_t)b]; });
+                const int64_t first = out;
+                for (int64_t a = 0; a < nwalks && out - first < n_rep; ++a) {
+                    make_walk(g->rowptr, g->col, B.data(), nB, cfg->seed, k, order[(size_t)a], steps, seq.data());
+                    for (int t = 0; t <= steps && out - first < n_rep; ++t) {
+                        const int32_t v = seq[(size_t)t];
+                        if (inside[(size_t)v] || taken[(size_t)v]) continue;
+                        if (out >= halo_capacity) return aug_fail(GAD_ERR_OOM, "halo_nodes too small");
+                        taken[(size_t)v] = 1;
+                        halo_nodes[out++] = v;
+                    }
+                }
+                for (int64_t t = first; t < out; ++t) taken[(size_t)halo_nodes[t]] = 0;
+            }
+            for (int64_t t = 0; t < ncore; ++t) inside[(size_t)core[t]] = 0;
+            mark_kernel<<<grid(ncore), 256, 0, s>>>(d_core, ncore, d_inside, 0); ++g_kernel_launches;
+        }
+        if (walks_out) walks_out[k] = nwalks;
+        halo_ptr[k + 1] = out;
+    }
+    AUG_CK(cudaStreamSynchronize(s));
+    AUG_CK(cudaGetLastError());
+    return GAD_OK;
+}
+
+const char* gad_augment_last_error(void) { return augment_last_error(); }
+
+}  // extern "C"
