@@ -270,12 +270,22 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
                     n_rep = (int64_t)std::floor(cfg->alpha * (1.0 + dens) * (double)ncore);
                 }
                 n_rep = std::min<int64_t>(n_rep, (int64_t)st[0]);
-                // walks in descending order of their summed importance (equal scores: ascending index)
+                // walks in descending order of their summed importance (equal scores: ascending index).  Only the best
+                // walks are ever looked at, so the order is established for a leading stretch first and for all
+                // walks only if that stretch does not yield n(g_i) nodes.
                 order.resize((size_t)nwalks);
                 std::iota(order.begin(), order.end(), (int64_t)0);
-                std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return score[(size_t)a] > score[(size_t)b]; });
+                auto better = [&](int64_t a, int64_t b) {
+                    return score[(size_t)a] != score[(size_t)b] ? score[(size_t)a] > score[(size_t)b] : a < b;
+                };
+                int64_t sorted = std::min<int64_t>(nwalks, std::max<int64_t>(1024, 8 * n_rep));
+                if (n_rep > 0) std::partial_sort(order.begin(), order.begin() + sorted, order.end(), better);
                 const int64_t first = out;
                 for (int64_t a = 0; a < nwalks && out - first < n_rep; ++a) {
+                    if (a == sorted) {   // the leading stretch is used up: order the rest as well
+                        std::sort(order.begin() + sorted, order.end(), better);
+                        sorted = nwalks;
+                    }
                     make_walk(g->rowptr, g->col, B.data(), nB, cfg->seed, k, order[(size_t)a], steps, seq.data());
                     for (int t = 0; t <= steps && out - first < n_rep; ++t) {
                         const int32_t v = seq[(size_t)t];
