@@ -79,3 +79,27 @@ def test_compute_calls_fail_loudly_without_a_gpu():
     with pytest.raises(RuntimeError):
         pkg.Gad(n, rowptr, col, *flat(core), *flat(halo), np.zeros((n, 6), np.float32), np.zeros(n, np.int32),
                 np.zeros(n, np.uint8), (6, 5, 3))
+
+
+def test_augment_arguments_are_checked_on_the_host():
+    import ctypes as C
+    from paper_2110_02987_b200 import binding as b
+    L = pkg.load()
+    n, rowptr, col, w, core, halo = small_random_case(4)
+    cp, cn = flat(core)
+    rowptr = np.ascontiguousarray(rowptr, np.int64); col = np.ascontiguousarray(col, np.int32)
+    csr = b.gad_csr(int(n), int(rowptr[-1]), b._ptr(rowptr, C.c_int64), b._ptr(col, C.c_int32), None)
+
+    def ws(steps=2, cap=4, alpha=0.01, E=0.05, zc=1.96, nodes=cn):
+        cfg = b._AugmentConfig(steps, cap, alpha, E, zc, 0)
+        out = C.c_size_t(0)
+        rc = L.gad_augment_workspace_bytes(C.byref(csr), C.c_int32(len(core)), b._ptr(cp, C.c_int64), b._ptr(nodes, C.c_int32),
+                                           C.byref(cfg), C.byref(out))
+        return rc, out.value
+
+    rc, nbytes = ws()
+    assert rc == 0 and nbytes > 0 and nbytes % 256 == 0
+    assert ws(steps=0)[0] == -1 and ws(steps=9)[0] == -1 and ws(cap=0)[0] == -1 and ws(E=0.0)[0] == -1 and ws(alpha=-1.0)[0] == -1
+    bad = cn.copy(); bad[0] = n
+    assert ws(nodes=bad)[0] == -2
+    assert ws(cap=8)[1] > nbytes                      # room for more walks
