@@ -146,6 +146,7 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
         const int nb = min(BR, ch.nrows - b * BR);
         const float4* Ab = As + s * a_stage4;
         const float4* Bb = Bs + s * b_stage4;
+#pragma unroll 2
         for (int r = rg; r < nb; r += nrg) {
             const float4 h4 = live ? Ab[r * ldh4 + col4] : make_float4(0.f, 0.f, 0.f, 0.f);
             float2 dzp[NP / 2];
