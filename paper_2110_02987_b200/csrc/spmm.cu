@@ -41,20 +41,28 @@ struct EpiDev {
     int K;
 };
 
-template <int NV, bool EPI>
+// Which four columns (in units of four) accumulator j of lane gl holds: gl + group * j, or with PAIR (a lane owns eight
+// consecutive columns per 16-byte bfloat16 load) the halves of the eight columns 2 (gl + group * (j / 2)).
+template <bool PAIR>
+__device__ __forceinline__ int col4_of(int gl, int group, int j) {
+    if constexpr (PAIR) return 2 * (gl + group * (j >> 1)) + (j & 1);
+    else return gl + group * j;
+}
+
+template <int NV, bool EPI, bool PAIR = false>
 __device__ __forceinline__ void finish_row(float4 (&acc)[NV], int row, int gl, int group, int F4, float* __restrict__ out,
                                            int ldo, const EpiDev& ep, int known_k = -1) {
     if (EPI) {
         const int k = known_k >= 0 ? known_k : find_sub(ep.sub_off, ep.K, row);   // the list of cut rows carries the subgraph
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
-            const int v = gl + group * j;
+            const int v = col4_of<PAIR>(gl, group, j);
             if (v < F4) acc[j] = apply_act(acc[j], ep.act, k, row, 4 * v);
         }
     }
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-        int v = gl + group * j;
+        int v = col4_of<PAIR>(gl, group, j);
         if (v < F4) reinterpret_cast<float4*>(out + (long long)row * ldo)[v] = acc[j];
     }
 }
@@ -187,7 +195,7 @@ __global__ void __launch_bounds__(256) spmm_finish_kernel(const int4* __restrict
 // next smaller power of two, so a batch costs at most one round trip more than its full groups.
 // Where a lane finds its 16 bytes of operand row c: operand start + c * (row stride in bytes) + the lane's column
 // offset.  With OFF32 the whole operand is smaller than 4 GiB and the offset is formed in 32 bits by one multiply-add.
-template <int NV, bool OFF32, bool BF>
+template <int NV, bool OFF32, bool BF, bool PAIR = false>
 struct ZLane {
     const char* base;      // OFF32: start of the operand (the same for the whole warp)
     const char* ptr[NV];   // otherwise: start of the operand plus the lane's column offset
@@ -197,10 +205,21 @@ struct ZLane {
         if constexpr (OFF32) return load_row4<BF>(base + (c * ldzb + off[j]));
         else return load_row4<BF>(ptr[j] + (unsigned long long)c * ldzb);
     }
+    // PAIR: eight bfloat16 values (16 bytes) of operand row c at this lane's j-th position, widened to two float4
+    __device__ __forceinline__ void load_pair(uint32_t c, int j, float4& lo, float4& hi) const {
+        const char* p;
+        if constexpr (OFF32) p = base + (c * ldzb + off[j]);
+        else p = ptr[j] + (unsigned long long)c * ldzb;
+        const uint4 u = __ldg(reinterpret_cast<const uint4*>(p));
+        lo = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                         __uint_as_float(u.y & 0xffff0000u));
+        hi = make_float4(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u), __uint_as_float(u.w << 16),
+                         __uint_as_float(u.w & 0xffff0000u));
+    }
 };
 
-template <int NV, int UU, bool OFF32, bool BF>
-__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const ZLane<NV, OFF32, BF>& zl) {
+template <int NV, int UU, bool OFF32, bool BF, bool PAIR>
+__device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, const ZLane<NV, OFF32, BF, PAIR>& zl) {
     uint32_t c[UU];
     float a[UU];
     if constexpr (UU == 1) {
@@ -215,10 +234,17 @@ __device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, c
         }
     }
     float4 z[UU][NV];
+    if constexpr (PAIR) {
 #pragma unroll
-    for (int u = 0; u < UU; ++u)
+        for (int u = 0; u < UU; ++u)
 #pragma unroll
-        for (int j = 0; j < NV; ++j) z[u][j] = zl.load(c[u], j);
+            for (int j = 0; j < NV / 2; ++j) zl.load_pair(c[u], j, z[u][2 * j], z[u][2 * j + 1]);
+    } else {
+#pragma unroll
+        for (int u = 0; u < UU; ++u)
+#pragma unroll
+            for (int j = 0; j < NV; ++j) z[u][j] = zl.load(c[u], j);
+    }
 #pragma unroll
     for (int u = 0; u < UU; ++u)
 #pragma unroll
@@ -230,11 +256,11 @@ __device__ __forceinline__ void gather_fma(float4 (&acc)[NV], const uint2* st, c
         }
 }
 
-template <int NV, int V, bool OFF32, bool BF>
-__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const ZLane<NV, OFF32, BF>& zl) {
+template <int NV, int V, bool OFF32, bool BF, bool PAIR>
+__device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, int r, const ZLane<NV, OFF32, BF, PAIR>& zl) {
     if constexpr (V >= 1) {
-        if (r > V / 2) gather_fma<NV, V, OFF32, BF>(acc, st, zl);
-        else gather_tail<NV, V / 2, OFF32, BF>(acc, st, r, zl);
+        if (r > V / 2) gather_fma<NV, V, OFF32, BF, PAIR>(acc, st, zl);
+        else gather_tail<NV, V / 2, OFF32, BF, PAIR>(acc, st, r, zl);
     }
 }
 
@@ -258,11 +284,11 @@ template <int NV> struct ItemCfg {
     static constexpr int MINB = NV == 1 ? GAD_SPMM_MINB1 : (NV == 2 ? GAD_SPMM_MINB2 : (NV <= 4 ? 6 : 4));   // CTAs of 4 warps per SM
 };
 
-template <int NV, bool EPI, bool OFF32, bool BF>
+template <int NV, bool EPI, bool OFF32, bool BF, bool PAIR>
 __global__ void __launch_bounds__(32 * kItemWarps, ItemCfg<NV>::MINB)
 spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z,
                   int ldz, float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
-    constexpr int UU = ItemCfg<NV>::UU;
+    constexpr int UU = PAIR ? 2 * ItemCfg<NV>::UU : ItemCfg<NV>::UU;   // half the bytes per operand row: twice the rows in flight
     __shared__ __align__(16) uint2 stage_all[kItemWarps][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int idx = blockIdx.x * kItemWarps + warp;
@@ -273,12 +299,13 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
     const uint2* ent = item.ent;
     const uint2 pad = make_uint2((uint32_t)row, 0u);
     // lanes past the last column read the last one (their sums are never stored)
-    ZLane<NV, OFF32, BF> zl;
+    ZLane<NV, OFF32, BF, PAIR> zl;
     zl.base = reinterpret_cast<const char*>(Z);
     zl.ldzb = OpBytes<BF>::elem * (uint32_t)ldz;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-        zl.off[j] = OpBytes<BF>::quad * (uint32_t)min(lane + 32 * j, F4 - 1);
+        // PAIR (F4 even): position j < NV / 2 is the lane's j-th run of eight bfloat16 columns (16 bytes)
+        zl.off[j] = PAIR ? 16u * (uint32_t)min(lane + 32 * j, F4 / 2 - 1) : OpBytes<BF>::quad * (uint32_t)min(lane + 32 * j, F4 - 1);
         zl.ptr[j] = zl.base + zl.off[j];
     }
     float4 acc[NV];
@@ -294,17 +321,17 @@ spmm_items_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items,
         stage[lane] = mine;
         __syncwarp();
         int t = 0;
-        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU, OFF32, BF>(acc, stage + t, zl);
-        gather_tail<NV, UU / 2, OFF32, BF>(acc, stage + t, cnt - t, zl);
+        for (; t + UU / 2 < cnt; t += UU) gather_fma<NV, UU, OFF32, BF, PAIR>(acc, stage + t, zl);
+        gather_tail<NV, UU / 2, OFF32, BF, PAIR>(acc, stage + t, cnt - t, zl);
     }
     if (item.slot >= 0) {
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
-            const int v = lane + 32 * j;
+            const int v = col4_of<PAIR>(lane, 32, j);
             if (v < F4) reinterpret_cast<float4*>(scratch + (long long)item.slot * ldo)[v] = acc[j];
         }
     } else {
-        finish_row<NV, EPI>(acc, row, lane, 32, F4, out, ldo, ep);
+        finish_row<NV, EPI, PAIR>(acc, row, lane, 32, F4, out, ldo, ep);
     }
 }
 
@@ -315,10 +342,20 @@ static cudaError_t launch_rows(const SparseDev& A, const float* Z, int ldz, floa
         if (A.nitems > 0) {
             const unsigned grid = (unsigned)((A.nitems + kItemWarps - 1) / kItemWarps);
             // every byte of the operand within 4 GiB of its start: 32-bit offsets
-            if ((unsigned long long)A.nrows * (unsigned long long)OpBytes<BF>::elem * (unsigned long long)ldz < (1ull << 32))
-                spmm_items_kernel<NV, EPI, true, BF><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
-            else
-                spmm_items_kernel<NV, EPI, false, BF><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+            const bool off32 = (unsigned long long)A.nrows * (unsigned long long)OpBytes<BF>::elem * (unsigned long long)ldz < (1ull << 32);
+            bool paired = false;
+            if constexpr (BF && NV % 2 == 0) {
+                // a bfloat16 operand of a whole number of 8-column runs: 16-byte loads, eight columns per lane and load
+                if (F4 % 2 == 0 && ldz % 8 == 0) {
+                    paired = true;
+                    if (off32) spmm_items_kernel<NV, EPI, true, true, true><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+                    else spmm_items_kernel<NV, EPI, false, true, true><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+                }
+            }
+            if (!paired) {
+                if (off32) spmm_items_kernel<NV, EPI, true, BF, false><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+                else spmm_items_kernel<NV, EPI, false, BF, false><<<grid, 32 * kItemWarps, 0, s>>>(A.ecv, A.items, A.nitems, Z, ldz, out, ldo, A.scratch, F4, ep);
+            }
             ++g_kernel_launches;
         }
         if (A.nfin > 0) {
