@@ -31,6 +31,10 @@
  *     most recent forward pass).
  *   - each processor takes one SGD step on its own copy, then the copies are replaced by their
  *     zeta-weighted mean; from identical copies this equals applying the weighted mean gradient.
+ *   - the ReLU of the forward equation has a kink at 0: a hidden unit whose pre-activation is zero
+ *     within rounding may be "on" in one arithmetic and "off" in another, and both are valid results.
+ *     A caller comparing another implementation with this one may prescribe the branch of such units
+ *     (orc_set_relu_branch), so that both sides take that decision alike; nothing else is affected.
  *
  * Pins: see tests/test_oracle_*.py (dense brute force, finite differences, the paper's printed
  * zeta values, Property 2, closed forms, special cases).  Parity unpinned (readings, not facts):
@@ -212,6 +216,7 @@ typedef struct {
     uint64_t seed;
     int32_t weighted, zeta_mode;
     int64_t epoch;
+    int8_t** branch;          /* L+1 maps [Np x dims[l]] or NULL: 0 = ReLU decides, 1 = unit taken as on, 2 = as off */
 } orc_model;
 
 static int64_t w_off(const orc_model* m, int l) {
@@ -224,6 +229,7 @@ static int64_t b_off(const orc_model* m, int l) { return w_off(m, l) + (int64_t)
 void orc_destroy(orc_model* m) {
     if (!m) return;
     if (m->H) { for (int l = 0; l <= m->L; ++l) free(m->H[l]); free(m->H); }
+    if (m->branch) { for (int l = 0; l <= m->L; ++l) free(m->branch[l]); free(m->branch); }
     free(m->dims); free(m->rowptr); free(m->col); free(m->val); free(m->sub_off); free(m->deg); free(m->label);
     free(m->train); free(m->ntrain); free(m->Z); free(m->dPre); free(m->dZ); free(m->params); free(m->grads);
     free(m);
@@ -333,7 +339,8 @@ static void forward(orc_model* m, int train) {
                         s += m->val[e] * m->Z[(int64_t)m->col[e] * fo + j];
                     s += b[j];
                     if (l < m->L - 1) {
-                        s = s > 0.0 ? s : 0.0;
+                        int br = (m->branch && m->branch[l + 1]) ? m->branch[l + 1][r * fo + j] : 0;
+                        s = br == 1 ? s : (br == 2 ? 0.0 : (s > 0.0 ? s : 0.0));
                         if (train && m->dropout > 0.0)
                             s = keep_unit(m->seed, m->epoch, l, r, j, m->dropout) ? s / (1.0 - m->dropout) : 0.0;
                     }
@@ -415,7 +422,11 @@ static void backward(orc_model* m) {
                     for (int j = 0; j < fo; ++j) s += m->dZ[r * fo + j] * W[(int64_t)f * fo + j];
                     double h = m->H[l][r * fi + f];
                     double scale = m->dropout > 0.0 ? 1.0 / (1.0 - m->dropout) : 1.0;
-                    next[r * fi + f] = h > 0.0 ? s * scale : 0.0;
+                    int br = (m->branch && m->branch[l]) ? m->branch[l][r * fi + f] : 0;
+                    int on = h > 0.0;
+                    if (br == 1) on = !(m->dropout > 0.0) || keep_unit(m->seed, m->epoch, l - 1, r, f, m->dropout);
+                    if (br == 2) on = 0;
+                    next[r * fi + f] = on ? s * scale : 0.0;
                 }
         }
         memcpy(m->dPre, next, sizeof(double) * (size_t)m->Np * (size_t)fi);
@@ -564,6 +575,27 @@ void orc_train_epoch(orc_model* m, double* loss_out) {
     for (int64_t i = 0; i < (int64_t)m->K * m->P; ++i) m->params[i] -= m->lr * m->grads[i];
     orc_consensus(m);
     m->epoch += 1;
+}
+
+/* Prescribes the ReLU branch of n hidden units of H^(layer), 1 <= layer <= L-1 (side 1: on, 2: off, 0: let the ReLU
+ * decide again); n < 0 forgets every prescription of that layer.  For units at the kink, see the header comment. */
+int orc_set_relu_branch(orc_model* m, int32_t layer, int64_t n, const int64_t* rows, const int32_t* cols, int32_t side) {
+    if (!m || layer < 1 || layer > m->L - 1 || side < 0 || side > 2) return ORC_ERR_ARG;
+    if (!m->branch) {
+        m->branch = (int8_t**)calloc((size_t)(m->L + 1), sizeof(int8_t*));
+        if (!m->branch) return ORC_ERR_OOM;
+    }
+    size_t cells = (size_t)(m->Np > 0 ? m->Np : 1) * (size_t)m->dims[layer];
+    if (n < 0) { free(m->branch[layer]); m->branch[layer] = NULL; return ORC_OK; }
+    if (!m->branch[layer]) {
+        m->branch[layer] = (int8_t*)calloc(cells, 1);
+        if (!m->branch[layer]) return ORC_ERR_OOM;
+    }
+    for (int64_t i = 0; i < n; ++i) {
+        if (rows[i] < 0 || rows[i] >= m->Np || cols[i] < 0 || cols[i] >= m->dims[layer]) return ORC_ERR_RANGE;
+        m->branch[layer][rows[i] * m->dims[layer] + cols[i]] = (int8_t)side;
+    }
+    return ORC_OK;
 }
 
 /* accessors */

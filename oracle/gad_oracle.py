@@ -195,6 +195,19 @@ class Model:
         lib().orc_get_grads(self._h, C.c_int32(k), _p(out, C.c_double))
         return out
 
+    def set_relu_branch(self, layer: int, rows, cols, side: int):
+        """Prescribes the ReLU branch (1 on, 2 off, 0 undecided again) of hidden units of H^(layer) at the kink."""
+        rows = np.ascontiguousarray(rows, dtype=np.int64)
+        cols = np.ascontiguousarray(cols, dtype=np.int32)
+        rc = lib().orc_set_relu_branch(self._h, C.c_int32(layer), C.c_int64(rows.shape[0]), _p(rows, C.c_int64),
+                                       _p(cols, C.c_int32), C.c_int32(side))
+        if rc != 0:
+            raise ValueError("orc_set_relu_branch: error %d" % rc)
+
+    def clear_relu_branches(self):
+        for l in range(1, len(self.dims) - 1):
+            lib().orc_set_relu_branch(self._h, C.c_int32(l), C.c_int64(-1), None, None, C.c_int32(0))
+
     def ntrain(self) -> np.ndarray:
         out = np.zeros(self.K, dtype=np.int64)
         lib().orc_get_ntrain(self._h, _p(out, C.c_int64))

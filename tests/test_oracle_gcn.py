@@ -265,3 +265,58 @@ def test_dropout_mask_is_a_pure_counter_function():
     other = np.array([[orc.keep_unit(3, 3, 1, r, c, 0.3) for c in range(64)] for r in range(256)])
     assert (keep != other).mean() > 0.2
     assert all(orc.keep_unit(9, 0, 0, r, 0, 0.0) for r in range(100))
+
+
+def test_prescribed_relu_branches_equal_a_network_with_that_mask():
+    """orc_set_relu_branch (for hidden units at the kink of the ReLU): with the branch of some units prescribed, forward
+    and gradients are those of the network whose layer-1 activation is `mask * pre-activation` with that mask held
+    fixed - checked against a dense forward and central finite differences of that masked network; prescribing the
+    branch the ReLU takes anyway changes nothing, and clearing restores the plain ReLU bit for bit."""
+    dims = (6, 5, 3)
+    n, rowptr, col, w, core, halo, X, y, split, theta, st = make_case(3, dims, K=1, halo=False)
+    idx = core[0]
+    hat, _ = dense_hat(dense_graph(n, rowptr, col, w), idx)
+    Xd, yd = X[idx].astype(np.float64), y[idx]
+    train = np.nonzero(split[idx] == 0)[0]
+    m = orc.Model(st, X, y, split, dims, theta)
+    m.forward_backward()
+    g_plain, h1_plain = m.get_grads(0), m.activation(1)
+    natural = h1_plain > 0
+    on = np.argwhere(natural)[:3]            # three active units to switch off
+    off = np.argwhere(~natural)[:3]          # three inactive units to switch on
+    mask = natural.copy()
+    mask[on[:, 0], on[:, 1]] = False
+    mask[off[:, 0], off[:, 1]] = True
+
+    def loss_of(t):
+        (W0, b0), (W1, b1) = unpack(t, dims)
+        z = hat @ ((mask * (hat @ (Xd @ W0) + b0)) @ W1) + b1
+        zt = z[train]
+        lse = zt.max(axis=1) + np.log(np.exp(zt - zt.max(axis=1, keepdims=True)).sum(axis=1))
+        return np.mean(lse - zt[np.arange(len(train)), yd[train]]), z
+
+    # the branch the ReLU takes anyway: nothing changes
+    m.set_relu_branch(1, on[:, 0], on[:, 1], 1)
+    m.set_relu_branch(1, off[:, 0], off[:, 1], 2)
+    m.forward_backward()
+    assert np.array_equal(m.get_grads(0), g_plain) and np.array_equal(m.activation(1), h1_plain)
+    # the other branch: the masked network
+    m.set_relu_branch(1, on[:, 0], on[:, 1], 2)
+    m.set_relu_branch(1, off[:, 0], off[:, 1], 1)
+    loss = m.forward_backward()
+    t0 = theta.astype(np.float64)
+    want_loss, want_logits = loss_of(t0)
+    assert abs(loss[0] - want_loss) < 1e-13
+    assert rel_err(m.activation(2), want_logits) < 1e-13
+    fd = np.zeros_like(t0)
+    for i in range(t0.size):
+        tp, tm = t0.copy(), t0.copy()
+        tp[i] += 1e-6; tm[i] -= 1e-6
+        fd[i] = (loss_of(tp)[0] - loss_of(tm)[0]) / 2e-6
+    assert rel_err(m.get_grads(0), fd) < 1e-7
+    assert rel_err(m.get_grads(0), g_plain) > 1e-4          # and it is a different network
+    m.clear_relu_branches()
+    m.forward_backward()
+    assert np.array_equal(m.get_grads(0), g_plain)
+    with pytest.raises(ValueError):
+        m.set_relu_branch(2, [0], [0], 1)                    # the last layer has no ReLU
