@@ -1,7 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the GAD training epoch (all hot-path kernels) on seeded synthetic graphs.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3k4|c3k8|c4|tiny|sweep] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c3k4|c3k8|c2|tiny|sweep] [--impl reference]
+
+The default workload is c4, the largest configuration that runs on one GPU (2.45 M nodes, K = 16, 100-256-256-47).
 
 A step is one call of gad_train_epoch: forward, loss, backward, importance weights and weighted consensus for
 all K replicas.  Prints ONE JSON line (rank 0).  ``value`` is epochs/s with every input resident in HBM;
@@ -117,8 +119,40 @@ def describe(w):
     return "%s: n=%d, nnz=%d, K=%d, dims=%s; %s" % (w.name, w.n, w.nnz, w.K, "-".join(str(d) for d in w.dims), w.recipe)
 
 
+def oracle_sample(w, theta, seconds_per_step):
+    """The oracle's share of the workload for one timed step: whole epochs when one fits `seconds_per_step`, otherwise
+    the leading store rows of subgraph 0 (its core nodes in the partition's own breadth-first / contiguous order, as a
+    block of their own), sized from a short pilot run so that a step takes about that long.  Nothing is timed on the
+    whole workload first: on the largest configuration one oracle epoch takes minutes.
+    Returns (model, fraction of an epoch one step stands for, description)."""
+    from oracle import gad_oracle as orc
+    rows_all = int(sum(len(c) + len(h) for c, h in zip(w.core, w.halo)))
+    core0 = w.core[0]
+
+    def prefix_model(m):
+        sub = type(w)(**{**w.__dict__})
+        sub.core, sub.halo = [core0[:m]], [np.empty(0, dtype=np.int32)]
+        return orc.from_workload(sub, theta)
+
+    m0 = int(min(len(core0), 2000))
+    pilot = prefix_model(m0)
+    pilot.train_epoch()                      # page everything in
+    t0 = time.perf_counter()
+    pilot.train_epoch()
+    per_row = (time.perf_counter() - t0) / max(m0, 1)
+    pilot.close()
+    if per_row * rows_all <= seconds_per_step:
+        return orc.from_workload(w, theta), 1.0, "whole epochs of the workload"
+    m = int(min(len(core0), max(m0, seconds_per_step / per_row)))
+    frac = m / float(rows_all)
+    return prefix_model(m), frac, ("the first %d core rows of subgraph 0 of %d as a block of their own (%.4f of the %d store rows) "
+                                   "per step, sized from a %d-row pilot; epochs/s = that fraction / time per step"
+                                   % (m, w.K, frac, rows_all, m0))
+
+
 def run_reference(args, rank):
-    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only): every step a bounded sample of the workload,
+    sized so that warm-up and timed steps together take about two minutes."""
     if rank != 0:
         return
     from gad_synth import make_workload, glorot_params
@@ -127,40 +161,16 @@ def run_reference(args, rank):
     w = make_workload(args.workload, **args.wl_kw)
     theta = glorot_params(w.dims, np.random.default_rng(0))
     cores = orc.threads()
-    # bound the run: whole epochs if K*... fits, else the first subgraph alone (1/K of an epoch's work)
-    m = orc.from_workload(w, theta)
-    t0 = time.perf_counter()
-    m.train_epoch()
-    one = time.perf_counter() - t0
     total_steps = args.steps + args.warmup
-    if one * total_steps <= 150.0 or w.K == 1:
-        sample = "whole epochs of the workload (%d timed)" % args.steps
-        scale = 1.0
-        for _ in range(max(args.warmup - 1, 0)):
-            m.train_epoch()
-        t0 = time.perf_counter()
-        for _ in range(args.steps):
-            m.train_epoch()
-        dt = time.perf_counter() - t0
-    else:
-        m.close()
-        sub = type(w)(**{**w.__dict__})
-        sub.core, sub.halo = [w.core[0]], [w.halo[0]]
-        m = orc.from_workload(sub, theta)
+    m, frac, sample = oracle_sample(w, theta, 120.0 / max(total_steps, 1))
+    for _ in range(args.warmup):
         m.train_epoch()
-        frac = (len(w.core[0]) + len(w.halo[0])) / float(sum(len(c) + len(h) for c, h in zip(w.core, w.halo)))
-        scale = frac
-        sample = "subgraph 0 of %d only (%.3f of the store rows) per step; epochs/s = steps * that fraction / time" % (w.K, frac)
-        steps = args.steps
-        t0 = time.perf_counter()
-        for _ in range(steps):
-            m.train_epoch()
-            if time.perf_counter() - t0 > 150.0:
-                steps = _ + 1
-                break
-        dt = time.perf_counter() - t0
-        args.steps = steps
-    value = args.steps * scale / dt
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        m.train_epoch()
+    dt = time.perf_counter() - t0
+    m.close()
+    value = args.steps * frac / dt
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -173,33 +183,28 @@ def run_reference(args, rank):
 
 
 def cpu_baseline(w, theta, budget_s=20.0):
+    """The oracle timed beside the library: about `budget_s` seconds of CPU work on a bounded sample of the workload."""
     from oracle import gad_oracle as orc
     orc.build()
-    m = orc.from_workload(w, theta)
     cores = orc.threads()
+    m, frac, sample = oracle_sample(w, theta, budget_s)
+    if frac >= 1.0:
+        m.train_epoch()
+        n, t0 = 0, time.perf_counter()
+        while True:
+            m.train_epoch()
+            n += 1
+            dt = time.perf_counter() - t0
+            if dt > budget_s or n >= 20:
+                break
+        m.close()
+        return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": "%d whole epochs of the same workload after one warm-up epoch" % n}
     t0 = time.perf_counter()
     m.train_epoch()
-    first = time.perf_counter() - t0
-    if first > budget_s and w.K > 1:
-        m.close()
-        sub = type(w)(**{**w.__dict__})
-        sub.core, sub.halo = [w.core[0]], [w.halo[0]]
-        m = orc.from_workload(sub, theta)
-        t0 = time.perf_counter()
-        m.train_epoch()
-        dt = time.perf_counter() - t0
-        frac = (len(w.core[0]) + len(w.halo[0])) / float(sum(len(c) + len(h) for c, h in zip(w.core, w.halo)))
-        return {"value": frac / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": "one epoch of subgraph 0 of %d (%.3f of the store rows), scaled to a whole epoch" % (w.K, frac)}
-    n, t0 = 0, time.perf_counter()
-    while True:
-        m.train_epoch()
-        n += 1
-        dt = time.perf_counter() - t0
-        if dt + first > budget_s or n >= 20:
-            break
-    return {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "%d whole epochs of the same workload after one warm-up epoch" % n}
+    dt = time.perf_counter() - t0
+    m.close()
+    return {"value": frac / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": "one step: " + sample}
 
 
 def run_micro_consensus(args):
@@ -375,7 +380,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None, help="timed epochs (default: 1000 for c2 and smaller, 20 otherwise)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="gad", choices=["gad", "reference"])
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c4", help="c4 (default: the largest single-GPU configuration), c3k4, c3k8, c2, tiny, sweep")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--mean-deg", type=float, default=32)
     ap.add_argument("--F", type=int, default=128)

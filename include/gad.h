@@ -15,8 +15,10 @@
  *   - "host" pointers are ordinary CPU memory owned by the caller; they are only read (or written) during the
  *     call.  "device" pointers are CUDA device memory of the current device.
  *   - The library allocates no device memory: the caller passes one device workspace (size from
- *     gad_workspace_bytes) and a CUDA stream; both must outlive the context.  All kernels of a context run on
- *     that stream.  A context is not thread-safe.
+ *     gad_workspace_bytes) and a CUDA stream; both must outlive the context.  Work is ordered as if it all ran on
+ *     that stream; the context also owns two streams of its own (one for the host-to-device copies of
+ *     gad_set_inputs, one for small kernels of an epoch that run beside the main sequence), tied to the caller's
+ *     stream by events.  A context is not thread-safe.
  *   - Matrices are row-major.  One replica's parameters are the P floats
  *       [ W_0 (F_0 x F_1), b_0 (F_1), W_1 (F_1 x F_2), b_1 (F_2), ... ],  P = sum_l (F_l F_{l+1} + F_{l+1}).
  *   - "store row": the K augmented subgraphs are kept as one block-diagonal matrix.  Subgraph k owns the rows
@@ -217,9 +219,19 @@ int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels);
 
 /* For a loop that never waits inside a step: enqueues the copy of the K+1 losses of the most recent epoch
  * (layout of gad_get_loss) into loss_out, host memory that must be pinned and stay valid until gad_synchronize has
- * returned.  No check for non-finite values is made.  gad_synchronize waits for both of the context's streams. */
+ * returned.  No check for non-finite values is made.  gad_synchronize waits for all of the context's streams and
+ * returns GAD_ERR_DEVICE_TIMEOUT if a bounded device-side wait ran out since the last check (the epoch in which that
+ * happened has left the parameters as they were: the update and consensus kernels skip their work once the error
+ * word is set); the error is cleared by reporting it. */
 int gad_read_loss_async(gad_ctx* ctx, float* loss_out);
 int gad_synchronize(gad_ctx* ctx);
+
+/* For testing the time-out path without hanging anything (no counterpart in the paper): enqueues a one-thread kernel
+ * that waits, with the same bounded wait the tensor-core transforms use and a limit of `polls` polls (1 .. 65536), on
+ * a barrier that nothing ever arrives at.  The wait runs out, the kernel raises the context's error word and returns;
+ * the next gad_get_loss / gad_train_epoch with loss_out / gad_synchronize reports GAD_ERR_DEVICE_TIMEOUT, and an epoch
+ * enqueued in between leaves the parameters untouched. */
+int gad_debug_expire_wait(gad_ctx* ctx, uint32_t polls);
 
 /* Epoch counter (it indexes the dropout mask); set it to resume a run. */
 int gad_get_epoch(const gad_ctx* ctx, int64_t* epoch);

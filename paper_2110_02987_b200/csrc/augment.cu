@@ -123,6 +123,13 @@ int plan_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int
     if (!g || !g->rowptr || (g->nnz > 0 && !g->col) || g->n < 0 || K < 1 || !core_ptr || !cfg) { err = "bad arguments"; return GAD_ERR_ARG; }
     if (cfg->steps < 1 || cfg->steps > kMaxSteps) { err = "steps must be 1 .. 8"; return GAD_ERR_ARG; }
     if (!(cfg->alpha >= 0.0) || !(cfg->E > 0.0) || !(cfg->zc > 0.0) || cfg->cap < 1) { err = "alpha >= 0, E > 0, zc > 0, cap >= 1"; return GAD_ERR_ARG; }
+    // the kernels index rowptr, col and the per-node arrays with the caller's values: check the whole CSR here, on the host
+    if (g->nnz < 0 || g->rowptr[0] != 0) { err = "rowptr must start at 0 and nnz must not be negative"; return GAD_ERR_ARG; }
+    for (int32_t v = 0; v < g->n; ++v)
+        if (g->rowptr[v + 1] < g->rowptr[v]) { err = "rowptr decreases"; return GAD_ERR_UNSORTED; }
+    if (g->rowptr[g->n] != g->nnz) { err = "rowptr[n] differs from nnz"; return GAD_ERR_ARG; }
+    for (int64_t e = 0; e < g->nnz; ++e)
+        if (g->col[e] < 0 || g->col[e] >= g->n) { err = "column out of range"; return GAD_ERR_RANGE; }
     p.max_core = 0; p.max_walks = 1;
     for (int32_t k = 0; k < K; ++k) {
         if (core_ptr[k + 1] < core_ptr[k]) { err = "core_ptr decreases"; return GAD_ERR_UNSORTED; }

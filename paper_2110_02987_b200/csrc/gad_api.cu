@@ -8,7 +8,33 @@
 
 using namespace gad;
 
-namespace gad { int64_t g_kernel_launches = 0; }
+#include <mutex>
+#include <set>
+
+namespace gad {
+
+std::atomic<int64_t> g_kernel_launches{0};
+
+cudaError_t configure_kernel_once(const void* kernel, int smem_bytes, bool max_carveout) {
+    static std::mutex lock;
+    static std::set<std::pair<int, const void*>> done;   // (device, kernel)
+    std::lock_guard<std::mutex> guard(lock);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const std::pair<int, const void*> key(dev, kernel);
+    if (done.count(key)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    if (max_carveout) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+    }
+    done.insert(key);
+    return cudaSuccess;
+}
+
+}  // namespace gad
 
 // TMA descriptors kept per layer: forward A, B_hi, B_lo; input-gradient A, B_hi, B_lo; weight-gradient H, dZ.
 constexpr int kMapsPerLayer = 8;
@@ -710,7 +736,7 @@ int gad_get_loss(gad_ctx* ctx, float* loss_out) {
     const int32_t flag = flags[0];
     if (flags[1]) {
         GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 8, ctx->stream));
-        return fail(ctx, GAD_ERR_DEVICE_TIMEOUT, "a bounded wait in the tensor-core transform ran out (role " + std::to_string(flags[1]) + ")");
+        return fail(ctx, GAD_ERR_DEVICE_TIMEOUT, "a bounded device-side wait ran out (role " + std::to_string(flags[1]) + ")");
     }
     if (flag) {
         GAD_CK(cudaMemsetAsync(ctx->ws + p.o_flags, 0, 4, ctx->stream));
@@ -748,7 +774,7 @@ static int enqueue_epoch(gad_ctx* ctx, bool consensus) {
     if (consensus)
         GAD_RUN("sgd_consensus", -1, 12.0 * p.K * p.Pint, 4.0 * p.K * p.Pint, [&] {
             return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
-                                        ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->stream);
+                                        ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 1, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
         });
     return GAD_OK;
 }
@@ -768,12 +794,14 @@ static void capture_epoch(gad_ctx* ctx, bool consensus, gad_ctx::EpochGraph& eg)
         eg.failed = true;   // e.g. the caller is capturing this stream already: the launches then go into that capture
         return;
     }
-    const int64_t before = g_kernel_launches;
+    const int64_t before = g_kernel_launches.load();
     const int rc = enqueue_epoch(ctx, consensus);
     cudaGraph_t graph = nullptr;
     const cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
-    const int64_t kernels = g_kernel_launches - before;
-    g_kernel_launches = before;   // nothing has run yet
+    // (a context belongs to one host thread, so the difference is this capture's own launches unless other threads
+    // launched meanwhile; only this capture's share is taken back: nothing of it has run yet)
+    const int64_t kernels = g_kernel_launches.load() - before;
+    g_kernel_launches -= kernels;
     if (rc == GAD_OK && e == cudaSuccess && graph && cudaGraphInstantiate(&eg.exec, graph, 0) == cudaSuccess) {
         eg.kernels = kernels;
     } else {
@@ -842,7 +870,7 @@ int gad_consensus(gad_ctx* ctx) {
     if (rc != GAD_OK) return rc;
     GAD_RUN("consensus", -1, 8.0 * p.K * p.Pint, 2.0 * p.K * p.Pint, [&] {
         return launch_sgd_consensus(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, 0.f,
-                                    ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 0, ctx->stream);
+                                    ctx->at<double>(p.o_zeta), ctx->cfg.weighted, 0, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
     });
     return GAD_OK;
 }
@@ -868,7 +896,8 @@ int gad_consensus_partial(gad_ctx* ctx, double total, int32_t with_step, float* 
     }
     GAD_RUN("consensus_partial", -1, (with_step ? 8.0 : 4.0) * p.K * p.Pint + 4.0 * p.Pint, 4.0 * p.K * p.Pint, [&] {
         return launch_consensus_partial(ctx->at<float>(p.o_params), ctx->at<float>(p.o_grads), p.pstride, p.pstride, p.K, ctx->cfg.lr,
-                                        ctx->at<double>(p.o_zeta), ctx->cfg.weighted, with_step ? 1 : 0, total, dev_out, ctx->stream);
+                                        ctx->at<double>(p.o_zeta), ctx->cfg.weighted, with_step ? 1 : 0, total, dev_out, ctx->at<int32_t>(p.o_flags) + 1,
+                                        ctx->stream);
     });
     return GAD_OK;
 }
@@ -877,7 +906,7 @@ int gad_consensus_apply(gad_ctx* ctx, const float* dev_in) {
     if (!ctx || !dev_in || ((uintptr_t)dev_in & 15) != 0) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
     GAD_RUN("consensus_apply", -1, 4.0 * (p.K + 1) * p.Pint, 0.0, [&] {
-        return launch_consensus_apply(ctx->at<float>(p.o_params), p.pstride, p.pstride, p.K, dev_in, ctx->stream);
+        return launch_consensus_apply(ctx->at<float>(p.o_params), p.pstride, p.pstride, p.K, dev_in, ctx->at<int32_t>(p.o_flags) + 1, ctx->stream);
     });
     return GAD_OK;
 }
@@ -960,6 +989,11 @@ int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels) {
     if (!ctx) return GAD_ERR_ARG;
     const Plan& p = ctx->p;
     if (!X && !labels) return GAD_OK;
+    if (labels) {   // the loss kernel indexes a row of logits with the label: same range check as gad_create, before anything is enqueued
+        const int C = p.dims[p.L];
+        for (int32_t u = 0; u < p.n; ++u)
+            if (labels[u] < 0 || labels[u] >= C) return fail(ctx, GAD_ERR_RANGE, "label out of range at node " + std::to_string(u));
+    }
     // The copy goes out on its own stream into one of two staging pairs, so it can overlap the epoch that is still
     // running on the context's stream; the gathers then run on the context's stream, after the copy.
     const int b = ctx->stage_idx;
@@ -997,7 +1031,19 @@ int gad_synchronize(gad_ctx* ctx) {
     if (!ctx) return GAD_ERR_ARG;
     GAD_CK(cudaStreamSynchronize(ctx->copy_stream));
     GAD_CK(cudaStreamSynchronize(ctx->side_stream));
+    int32_t timed_out = 0;
+    GAD_CK(cudaMemcpyAsync(&timed_out, ctx->ws + ctx->p.o_flags + 4, 4, cudaMemcpyDeviceToHost, ctx->stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));
+    if (timed_out) {
+        GAD_CK(cudaMemsetAsync(ctx->ws + ctx->p.o_flags + 4, 0, 4, ctx->stream));
+        return fail(ctx, GAD_ERR_DEVICE_TIMEOUT, "a bounded device-side wait ran out (role " + std::to_string(timed_out) + ")");
+    }
+    return GAD_OK;
+}
+
+int gad_debug_expire_wait(gad_ctx* ctx, uint32_t polls) {
+    if (!ctx || polls < 1 || polls > 65536) return GAD_ERR_ARG;
+    GAD_CK(launch_expire_wait(ctx->at<int32_t>(ctx->p.o_flags) + 1, polls, ctx->stream));
     return GAD_OK;
 }
 
@@ -1060,7 +1106,7 @@ int gad_profile_read(gad_ctx* ctx, int32_t i, char* name64, int64_t* launches, d
 
 int gad_launch_count(int64_t* launches) {
     if (!launches) return GAD_ERR_ARG;
-    *launches = gad::g_kernel_launches;
+    *launches = gad::g_kernel_launches.load();
     return GAD_OK;
 }
 

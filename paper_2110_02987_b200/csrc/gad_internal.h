@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <cmath>
 #include <string>
 #include <vector>
@@ -14,8 +15,12 @@ namespace gad {
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 
-// Kernels launched by this library in this process (every <<<>>> adds one).
-extern int64_t g_kernel_launches;
+// Kernels launched by this library in this process (every <<<>>> adds one; contexts on several host threads share it).
+extern std::atomic<int64_t> g_kernel_launches;
+
+// Function attributes belong to a device: asks once per (current device, kernel) for `smem_bytes` of dynamic shared
+// memory and, with `max_carveout`, for the largest shared-memory share of the SM.  Safe from several host threads.
+cudaError_t configure_kernel_once(const void* kernel, int smem_bytes, bool max_carveout);
 
 // ---------------------------------------------------------------------------------------------
 // Host-side result of building the block-diagonal store (create-time, not on the timed path).
@@ -198,13 +203,19 @@ cudaError_t launch_zeta_pair(const float* X, int ld, int F, const int32_t* deg, 
                              const int64_t* pair_ptr, int64_t npairs, int K, float beta, double* partial, unsigned* counters,
                              double* zeta, cudaStream_t s);
 
+// `err_word` (may be null): when a kernel of the epoch has reported a bounded wait that ran out, the gradients are not to
+// be trusted and the three consensus kernels leave the parameters (and `out`) untouched.
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
-                                 const double* zeta, int weighted, int with_sgd, cudaStream_t s);
+                                 const double* zeta, int weighted, int with_sgd, const int32_t* err_word, cudaStream_t s);
 // One context's share of a consensus over several contexts: out = sum_k w_k (theta_k - lr grad_k) with w_k = zeta_k / total
 // (or 1 / total), the parameters unchanged; and the finished sum written to every replica.
 cudaError_t launch_consensus_partial(const float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
-                                     const double* zeta, int weighted, int with_sgd, double total, float* out, cudaStream_t s);
-cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, int K, const float* in, cudaStream_t s);
+                                     const double* zeta, int weighted, int with_sgd, double total, float* out, const int32_t* err_word, cudaStream_t s);
+cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, int K, const float* in, const int32_t* err_word, cudaStream_t s);
+
+// One CTA waits, with the transforms' bounded wait and a limit of `polls` polls, on a barrier that nothing arrives at, and
+// reports it in `err` like a transform would (role 99).  For testing the time-out path; returns at once.
+cudaError_t launch_expire_wait(int32_t* err, uint32_t polls, cudaStream_t s);
 cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s);
 
 cudaError_t launch_gather_rows(const float* Xg, int F, const int32_t* gid, int64_t Np, float* H0, int ld,

@@ -67,8 +67,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the wait ran out or another role of this CTA has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* err, int code) {
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* err, int code,
+                                          uint32_t limit = WAIT_LIMIT) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -574,6 +575,18 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     }
 }
 
+// The bounded wait of the kernels above, made to run out: one thread polls a barrier that nothing ever arrives at.
+__global__ void expire_wait_kernel(int32_t* err, uint32_t polls) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0u, &abort_flag, err, 99, polls);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -614,6 +627,12 @@ bool tc_make_map(void* out_map, const void* base, uint64_t inner, uint64_t rows,
     return r == CUDA_SUCCESS;
 }
 
+cudaError_t launch_expire_wait(int32_t* err, uint32_t polls, cudaStream_t s) {
+    expire_wait_kernel<<<1, 32, 0, s>>>(err, polls);
+    ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w_int, int fi, int fo, int ldw, int ldkt, int K,
                                  float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, cudaStream_t s) {
     const long long n = (long long)fi * ldw;
@@ -628,11 +647,9 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
                                 const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s) {
     if (ntiles <= 0) return cudaSuccess;
     if (mode == 2 && !act) return cudaErrorInvalidValue;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_ROWS);
+    {
+        cudaError_t e = configure_kernel_once(reinterpret_cast<const void*>(gemm_tc_kernel), SMEM_BYTES_ROWS, false);
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     TcArgs a;
     a.tiles = tiles; a.ntiles_rows = ntiles; a.BN = tc_bn_for(n_cols); a.ntn = (ldc + a.BN - 1) / a.BN; a.Kd = Kd;
@@ -649,11 +666,9 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
 cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,
                               int nchunks, float* partial, int32_t* err, cudaStream_t s) {
     if (nchunks <= 0) return cudaSuccess;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    {
+        cudaError_t e = configure_kernel_once(reinterpret_cast<const void*>(gemm_tn_tc_kernel), SMEM_BYTES, false);
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     TnArgs a;
     a.chunks = chunks; a.BN = tc_bn_for(n_cols); a.ntm = (M + BM - 1) / BM; a.ntn = (ldw + a.BN - 1) / a.BN; a.M = M; a.ldw = ldw;

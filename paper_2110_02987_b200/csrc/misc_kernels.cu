@@ -508,8 +508,10 @@ __device__ __forceinline__ void consensus_weights(const double* __restrict__ zet
 // theta_k <- sum_j w_j theta_j for every k (weighted global consensus, Section 3.4.2).  One float4 per thread.
 __global__ void __launch_bounds__(256) sgd_consensus_kernel(float* __restrict__ params, const float* __restrict__ grads,
                                                             long long pstride, long long len4, int K, float lr,
-                                                            const double* __restrict__ zeta, int weighted, int with_sgd) {
+                                                            const double* __restrict__ zeta, int weighted, int with_sgd,
+                                                            const int32_t* __restrict__ err_word) {
     extern __shared__ float w_sm[];
+    if (err_word && *err_word) return;   // a bounded wait ran out earlier in this epoch: keep the parameters as they are
     consensus_weights(zeta, K, weighted, w_sm);
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= len4) return;
@@ -526,11 +528,11 @@ __global__ void __launch_bounds__(256) sgd_consensus_kernel(float* __restrict__ 
     for (int k = 0; k < K; ++k) reinterpret_cast<float4*>(params + (long long)k * pstride)[i] = acc;
 }
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
-                                 const double* zeta, int weighted, int with_sgd, cudaStream_t s) {
+                                 const double* zeta, int weighted, int with_sgd, const int32_t* err_word, cudaStream_t s) {
     const long long len4 = len / 4;
     if (len4 > 0) {
         sgd_consensus_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
-                                                                                                   zeta, weighted, with_sgd); ++g_kernel_launches; }
+                                                                                                   zeta, weighted, with_sgd, err_word); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 
@@ -541,8 +543,9 @@ cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstr
 __global__ void __launch_bounds__(256) consensus_partial_kernel(const float* __restrict__ params, const float* __restrict__ grads,
                                                                 long long pstride, long long len4, int K, float lr,
                                                                 const double* __restrict__ zeta, int weighted, int with_sgd,
-                                                                double total, float* __restrict__ out) {
+                                                                double total, float* __restrict__ out, const int32_t* __restrict__ err_word) {
     extern __shared__ float w_sm[];
+    if (err_word && *err_word) return;
     for (int k = threadIdx.x; k < K; k += blockDim.x) w_sm[k] = (float)((weighted ? zeta[k] : 1.0) / total);
     __syncthreads();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -560,25 +563,25 @@ __global__ void __launch_bounds__(256) consensus_partial_kernel(const float* __r
     reinterpret_cast<float4*>(out)[i] = acc;
 }
 __global__ void __launch_bounds__(256) consensus_apply_kernel(float* __restrict__ params, long long pstride, long long len4, int K,
-                                                              const float* __restrict__ in) {
+                                                              const float* __restrict__ in, const int32_t* __restrict__ err_word) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= len4) return;
+    if (i >= len4 || (err_word && *err_word)) return;
     const float4 v = reinterpret_cast<const float4*>(in)[i];
     for (int k = 0; k < K; ++k) reinterpret_cast<float4*>(params + (long long)k * pstride)[i] = v;
 }
 cudaError_t launch_consensus_partial(const float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
-                                     const double* zeta, int weighted, int with_sgd, double total, float* out, cudaStream_t s) {
+                                     const double* zeta, int weighted, int with_sgd, double total, float* out, const int32_t* err_word, cudaStream_t s) {
     const long long len4 = len / 4;
     if (len4 > 0) {
         consensus_partial_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
-                                                                                                       zeta, weighted, with_sgd, total, out);
+                                                                                                       zeta, weighted, with_sgd, total, out, err_word);
         ++g_kernel_launches;
     }
     return cudaGetLastError();
 }
-cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, int K, const float* in, cudaStream_t s) {
+cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, int K, const float* in, const int32_t* err_word, cudaStream_t s) {
     const long long len4 = len / 4;
-    if (len4 > 0) { consensus_apply_kernel<<<(unsigned)((len4 + 255) / 256), 256, 0, s>>>(params, pstride, len4, K, in); ++g_kernel_launches; }
+    if (len4 > 0) { consensus_apply_kernel<<<(unsigned)((len4 + 255) / 256), 256, 0, s>>>(params, pstride, len4, K, in, err_word); ++g_kernel_launches; }
     return cudaGetLastError();
 }
 

@@ -16,9 +16,6 @@
 // order by reduce_chunks, so nothing depends on scheduling.  Every mbarrier wait is bounded: on a time-out the CTA
 // raises the error word and returns.
 #include <algorithm>
-#include <mutex>
-#include <set>
-#include <utility>
 
 #include "gad_internal.h"
 
@@ -140,7 +137,14 @@ narrow_bwd_kernel(const float* __restrict__ H, int ldh, int fi, const float* __r
         const int s = b % kStages;
         const bool ok = bar_wait(ring.bar0 + 8u * (uint32_t)s, (uint32_t)(b / kStages) & 1u);
         if (__syncthreads_or(!ok)) {   // a copy never arrived: report it and stop
-            if (threadIdx.x == 0) atomicExch(err, 90);
+            if (threadIdx.x == 0) {
+                atomicExch(err, 90);
+                // copies of later stages may still be on their way into this CTA's shared memory: give each a short,
+                // bounded chance to land before the memory is released
+                for (int s2 = 0; s2 < kStages; ++s2)
+                    for (uint32_t i = 0; i < 4096u; ++i)
+                        if (bar_try(ring.bar0 + 8u * (uint32_t)s2, 0u) || bar_try(ring.bar0 + 8u * (uint32_t)s2, 1u)) break;
+            }
             return;
         }
         const int nb = min(BR, ch.nrows - b * BR);
@@ -217,20 +221,7 @@ bool narrow_supported(int ldi, int ldo) { return ldo >= 4 && ldo <= 16 && ldi >=
 // per kernel (the instantiations share one function-pointer type, so they are told apart by address).
 template <class Kernel>
 static cudaError_t prepare(Kernel kernel) {
-    static std::mutex lock;
-    static std::set<std::pair<int, const void*>> done;   // (device, kernel): function attributes are per device
-    std::lock_guard<std::mutex> guard(lock);
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    const std::pair<int, const void*> key(dev, reinterpret_cast<const void*>(kernel));
-    if (done.count(key)) return cudaSuccess;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    done.insert(key);
-    return cudaSuccess;
+    return configure_kernel_once(reinterpret_cast<const void*>(kernel), 100 * 1024, true);
 }
 
 static int slabs_for(int ldi) { const int s = (ldi + 127) / 128; return s <= 1 ? 1 : (s <= 2 ? 2 : 4); }

@@ -36,12 +36,21 @@ StaticScratch* g_scratch_ptr[kMaxDevices] = {};
 std::mutex g_setup_mutex;
 
 // Sum of the local degrees and of their squares over one subgraph (exact, in 64-bit integers).
+// Rows of subgraph k, cut to [0, rows): a sub_off array that does not match the matrix must not lead outside it.
+__device__ __forceinline__ void sub_range(const int32_t* __restrict__ sub_off, int k, long long rows, int& r0, int& n) {
+    const long long lo = min(max((long long)sub_off[k], 0ll), rows), hi = min(max((long long)sub_off[k + 1], lo), rows);
+    r0 = (int)lo;
+    n = (int)(hi - lo);
+}
+
 __global__ void __launch_bounds__(256) static_degree_kernel(const int32_t* __restrict__ deg, const int32_t* __restrict__ sub_off,
-                                                            StaticScratch* sc) {
+                                                            long long rows, StaticScratch* sc) {
     __shared__ long long s1[256], s2[256];
     const int k = blockIdx.x;
     long long a = 0, b = 0;
-    for (int r = sub_off[k] + threadIdx.x; r < sub_off[k + 1]; r += blockDim.x) {
+    int first, cnt;
+    sub_range(sub_off, k, rows, first, cnt);
+    for (int r = first + threadIdx.x; r < first + cnt; r += blockDim.x) {
         const long long d = deg[r];
         a += d;
         b += d * d;
@@ -59,10 +68,11 @@ __global__ void __launch_bounds__(256) static_degree_kernel(const int32_t* __res
 // Weighted first and second moments of every feature over one slice of one subgraph's rows, shifted by the
 // subgraph's first row.  Threads: 8 row lanes x 32 column lanes of one float4 each.
 __global__ void __launch_bounds__(256) static_partial_kernel(const float* __restrict__ X, int ld, const int32_t* __restrict__ deg,
-                                                             const int32_t* __restrict__ sub_off, StaticScratch* sc) {
+                                                             const int32_t* __restrict__ sub_off, long long rows, StaticScratch* sc) {
     __shared__ double sm[8][32][8];
     const int k = blockIdx.y, slice = blockIdx.x;
-    const int r0 = sub_off[k], n = sub_off[k + 1] - r0;
+    int r0, n;
+    sub_range(sub_off, k, rows, r0, n);
     const int per = (n + kSlices - 1) / kSlices;
     const int lo = min(n, slice * per), hi = min(n, lo + per);
     const bool uniform = sc->deg_sum[k] == 0;
@@ -99,11 +109,13 @@ __global__ void __launch_bounds__(256) static_partial_kernel(const float* __rest
 }
 
 // zeta_k = S_k / (D_k + beta) from the slice sums, slices added in order.
-__global__ void __launch_bounds__(256) static_final_kernel(int F, int ld, const int32_t* __restrict__ sub_off, float beta,
+__global__ void __launch_bounds__(256) static_final_kernel(int F, int ld, const int32_t* __restrict__ sub_off, long long rows, float beta,
                                                            StaticScratch* sc, float* __restrict__ zeta_out) {
     __shared__ double red[256];
     const int k = blockIdx.x;
-    const long long n = sub_off[k + 1] - sub_off[k];
+    int first, cnt;
+    sub_range(sub_off, k, rows, first, cnt);
+    const long long n = cnt;
     const bool uniform = sc->deg_sum[k] == 0;
     const double D = uniform ? (double)n : (double)sc->deg_sum[k];
     double q = 0.0;
@@ -173,9 +185,9 @@ extern "C" int gad_subgraph_weights_static(const float* X, int64_t rows, int32_t
         sc = g_scratch_ptr[dev];
     }
     cudaStream_t s = (cudaStream_t)stream;
-    static_degree_kernel<<<(unsigned)K, 256, 0, s>>>(deg, sub_off, sc);
-    static_partial_kernel<<<dim3(kSlices, (unsigned)K), 256, 0, s>>>(X, ld, deg, sub_off, sc);
-    static_final_kernel<<<(unsigned)K, 256, 0, s>>>(F, ld, sub_off, beta, sc, zeta_out);
+    static_degree_kernel<<<(unsigned)K, 256, 0, s>>>(deg, sub_off, (long long)rows, sc);
+    static_partial_kernel<<<dim3(kSlices, (unsigned)K), 256, 0, s>>>(X, ld, deg, sub_off, (long long)rows, sc);
+    static_final_kernel<<<(unsigned)K, 256, 0, s>>>(F, ld, sub_off, (long long)rows, beta, sc, zeta_out);
     static_weights_kernel<<<1, 256, 0, s>>>(K, weighted, sc, w_out);
     gad::g_kernel_launches += 4;
     return cudaGetLastError() == cudaSuccess ? GAD_OK : GAD_ERR_CUDA;

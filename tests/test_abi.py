@@ -90,10 +90,10 @@ def test_augment_arguments_are_checked_on_the_host():
     rowptr = np.ascontiguousarray(rowptr, np.int64); col = np.ascontiguousarray(col, np.int32)
     csr = b.gad_csr(int(n), int(rowptr[-1]), b._ptr(rowptr, C.c_int64), b._ptr(col, C.c_int32), None)
 
-    def ws(steps=2, cap=4, alpha=0.01, E=0.05, zc=1.96, nodes=cn):
+    def ws(steps=2, cap=4, alpha=0.01, E=0.05, zc=1.96, nodes=cn, graph=csr):
         cfg = b._AugmentConfig(steps, cap, alpha, E, zc, 0)
         out = C.c_size_t(0)
-        rc = L.gad_augment_workspace_bytes(C.byref(csr), C.c_int32(len(core)), b._ptr(cp, C.c_int64), b._ptr(nodes, C.c_int32),
+        rc = L.gad_augment_workspace_bytes(C.byref(graph), C.c_int32(len(core)), b._ptr(cp, C.c_int64), b._ptr(nodes, C.c_int32),
                                            C.byref(cfg), C.byref(out))
         return rc, out.value
 
@@ -103,3 +103,11 @@ def test_augment_arguments_are_checked_on_the_host():
     bad = cn.copy(); bad[0] = n
     assert ws(nodes=bad)[0] == -2
     assert ws(cap=8)[1] > nbytes                      # room for more walks
+    # the caller's CSR is checked like gad_create checks it: the kernels index with its values
+    badcol = col.copy(); badcol[2] = n
+    assert ws(graph=b.gad_csr(int(n), int(rowptr[-1]), b._ptr(rowptr, C.c_int64), b._ptr(badcol, C.c_int32), None))[0] == -2
+    badcol[2] = -1
+    assert ws(graph=b.gad_csr(int(n), int(rowptr[-1]), b._ptr(rowptr, C.c_int64), b._ptr(badcol, C.c_int32), None))[0] == -2
+    rp = rowptr.copy(); rp[5], rp[6] = rp[6] + 1, rp[5]
+    assert ws(graph=b.gad_csr(int(n), int(rowptr[-1]), b._ptr(rp, C.c_int64), b._ptr(col, C.c_int32), None))[0] == -3
+    assert ws(graph=b.gad_csr(int(n), int(rowptr[-1]) + 1, b._ptr(rowptr, C.c_int64), b._ptr(col, C.c_int32), None))[0] == -1

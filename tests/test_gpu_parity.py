@@ -58,34 +58,61 @@ def check_store(g, st):
     assert ulp.max(initial=0) <= 1
 
 
-def grad_tol(g, ref, tol):
-    """Tolerance for gradients.  A hidden unit whose pre-activation is zero within rounding can land on different
-    sides of the ReLU in fp32 and in the fp64 oracle; both results are valid, but such a unit changes its gradient
-    path by a finite amount.  Units like that must be genuine ties (magnitude <= max(1e-5, tol / 10) of the layer's
-    largest value); when there are any, the gradient comparison is relaxed to max(2 tol, 5e-2), otherwise it is `tol`."""
-    ties, worst = 0, 0.0
+def relu_kink_units(g, ref, tol):
+    """Hidden units that are zero on one side and not on the other.  A unit whose pre-activation is zero within rounding
+    can land on either side of the ReLU in fp32 and in the fp64 oracle; both are valid, but the gradient path differs by
+    a finite amount.  Such units must be genuine ties: magnitude at most max(1e-5, tol / 10) of the layer's largest value.
+    Returns {layer: (rows, cols, on the GPU's side?)}."""
+    out = {}
     for l in range(1, len(g.dims) - 1):
         a, b = g.get_activation(l), ref.activation(l)
         diff = (a == 0) != (b == 0)
         if diff.any():
-            ties += int(diff.sum())
-            worst = max(worst, float(np.max(np.maximum(np.abs(a[diff]), np.abs(b[diff]))) / np.max(np.abs(b))))
-    assert worst <= max(1e-5, 0.1 * tol), "a hidden unit differs across the ReLU and is not a tie (%g)" % worst
-    if ties:
-        print("ReLU ties: %d hidden units within %.1e of zero fall on different sides" % (ties, worst))
-    return tol if ties == 0 else max(2 * tol, 5e-2)
+            worst = float(np.max(np.maximum(np.abs(a[diff]), np.abs(b[diff]))) / np.max(np.abs(b)))
+            assert worst <= max(1e-5, 0.1 * tol), "a hidden unit differs across the ReLU and is not a tie (%g)" % worst
+            rows, cols = np.nonzero(diff)
+            out[l] = (rows, cols, a[rows, cols] != 0)
+    return out
+
+
+def oracle_step(g, ref, tol=TOL, step="train_epoch"):
+    """The oracle's counterpart of the step the library has just run (`step`: train_epoch or forward_backward), with the
+    ReLU decision of units at the kink taken as the library took it: the step is run; if units fell on different
+    sides it is run again from the same state with their branch prescribed (orc_set_relu_branch), until none differ.
+    The comparison that follows needs no widened tolerance.  Returns (the step's result, number of tie units)."""
+    saved = [ref.get_params(k) for k in range(ref.K)]
+    epoch = ref.epoch
+    out = getattr(ref, step)()
+    total = 0
+    for _ in range(4):
+        ties = relu_kink_units(g, ref, tol)
+        if not ties:
+            break
+        for l, (rows, cols, on) in ties.items():
+            total += len(rows)
+            ref.set_relu_branch(l, rows[on], cols[on], 1)
+            ref.set_relu_branch(l, rows[~on], cols[~on], 2)
+        for k in range(ref.K):
+            ref.set_params(k, saved[k])
+        ref.epoch = epoch
+        out = getattr(ref, step)()
+    else:
+        raise AssertionError("units at the ReLU kink keep changing sides")
+    ref.clear_relu_branches()
+    if total:
+        print("ReLU ties: %d hidden units at the kink took the library's branch in the oracle" % total)
+    return out, total
 
 
 def check_epoch(g, ref, tol=TOL, loss_tol=1e-5):
     lg = g.train_epoch()
-    lr = ref.train_epoch()
+    lr, _ = oracle_step(g, ref, tol)
     assert np.max(np.abs(lg - lr)) <= loss_tol + 1e-5 * np.max(np.abs(lr)), (lg, lr)
     L = len(g.dims) - 1
     for l in range(1, L + 1):
         assert rel_err(g.get_activation(l), ref.activation(l)) <= tol, "activation %d" % l
-    gt = grad_tol(g, ref, tol)
     for k in range(g.K):
-        assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt, "grads %d" % k
+        assert rel_err(g.get_grads(k), ref.get_grads(k)) <= tol, "grads %d" % k
         assert rel_err(g.get_params(k), ref.get_params(k)) <= tol, "params %d" % k
 
 
@@ -433,14 +460,17 @@ def test_c2_two_epochs_full_size():
     ref = orc().from_workload(w, theta)
     with pkg().from_workload(w, theta) as g:
         check_store(g, ref.store)
+        ties = 0
         for _ in range(2):
-            lg, lr = g.train_epoch(), ref.train_epoch()
+            lg = g.train_epoch()
+            lr, t = oracle_step(g, ref)
+            ties += t
             assert np.max(np.abs(lg - lr)) <= 1e-4
+        assert ties <= 64, "%d hidden units at the ReLU kink: more than rounding explains" % ties
         L = len(w.dims) - 1
         assert rel_err(g.get_activation(L), ref.activation(L)) <= TOL
-        gt = grad_tol(g, ref, TOL)
         for k in range(g.K):
-            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt, "replica %d (tolerance %g)" % (k, gt)
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL, "replica %d" % k
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
         zg, wg = g.subgraph_weights()
         zr, wr = ref.subgraph_weights()
@@ -480,14 +510,14 @@ def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
     g, ref, st = make_pair(case, dims, 21, lr=0.05, gemm_mode=gemm_mode, flags=flags)
     with g:
         for _ in range(2):
-            lg, lr = g.train_epoch(), ref.train_epoch()
+            lg = g.train_epoch()
+            lr, _ = oracle_step(g, ref, tol)
             assert np.max(np.abs(lg - lr)) <= (1e-4 if gemm_mode == 0 else 5e-2)
         L = len(dims) - 1
         for l in range(1, L + 1):
             assert rel_err(g.get_activation(l), ref.activation(l)) <= tol, "activation %d" % l
-        gt = grad_tol(g, ref, tol)
         for k in range(g.K):
-            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= tol
             assert rel_err(g.get_params(k), ref.get_params(k)) <= tol
         assert rel_err(g.forward(), ref.forward_global(case[0])) <= tol
 
@@ -505,14 +535,14 @@ def test_layers_of_at_most_sixteen_output_columns(flags, dims, dropout):
     g, ref, st = make_pair(case, dims, 31, lr=0.05, dropout=dropout, flags=flags)
     with g:
         for _ in range(2):
-            lg, lr = g.train_epoch(), ref.train_epoch()
+            lg = g.train_epoch()
+            lr, _ = oracle_step(g, ref)
             assert np.max(np.abs(lg - lr)) <= 1e-4
         L = len(dims) - 1
         for l in range(1, L + 1):
             assert rel_err(g.get_activation(l), ref.activation(l)) <= TOL, "activation %d" % l
-        gt = grad_tol(g, ref, TOL)
         for k in range(g.K):
-            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
         assert rel_err(g.forward(), ref.forward_global(case[0])) <= TOL
 
@@ -529,14 +559,14 @@ def test_importance_weights_summed_over_the_layers(dims, dropout):
         zr, wr = ref.subgraph_weights()
         assert np.max(np.abs(wg - wr)) <= 1e-5 and rel_err(zg, zr) <= 1e-5
         for _ in range(3):
-            lg, lr = g.train_epoch(), ref.train_epoch()
+            lg = g.train_epoch()
+            lr, _ = oracle_step(g, ref)
             assert np.max(np.abs(lg - lr)) <= 1e-4
         zg, wg = g.subgraph_weights()
         zr, wr = ref.subgraph_weights()
         assert np.max(np.abs(wg - wr)) <= 1e-5 and rel_err(zg, zr) <= 1e-5
-        gt = grad_tol(g, ref, TOL)
         for k in range(g.K):
-            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= gt
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
 
 
@@ -596,3 +626,51 @@ def test_reduced_precision_mode_on_a_power_law_graph():
                 assert rel_err(g.get_params(k), ref.get_params(k)) <= 5e-2
             # and it is not the fp32 path in disguise: the rounding of the operands shows
             assert rel_err(g.get_activation(L), ref.activation(L)) > 1e-5
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_model_untouched(tiny_signal):
+    """The transforms bound every device-side wait.  gad_debug_expire_wait makes one such wait run out on purpose (a
+    one-thread kernel polling, 1000 times, a barrier nothing arrives at): the kernel returns, the error word is raised,
+    the epoch enqueued behind it skips its update and consensus, the next waiting call returns
+    GAD_ERR_DEVICE_TIMEOUT, and the context goes on working from the unchanged parameters."""
+    w = tiny_signal
+    theta = glorot_params(w.dims, np.random.default_rng(13))
+    ref = orc().from_workload(w, theta)
+    with pkg().from_workload(w, theta) as g:
+        assert np.max(np.abs(g.train_epoch() - ref.train_epoch())) <= 1e-5
+        before = [g.get_params(k) for k in range(g.K)]
+        g.debug_expire_wait(1000)
+        g.train_epoch(wait=False)                       # enqueued behind the failed wait
+        with pytest.raises(pkg().GadError) as e:
+            g.synchronize()
+        assert e.value.code == -7
+        for k in range(g.K):
+            assert np.array_equal(g.get_params(k), before[k])
+        g.synchronize()                                  # reported once, then cleared
+        g.debug_expire_wait(1)
+        with pytest.raises(pkg().GadError) as e:
+            g.get_loss()
+        assert e.value.code == -7
+        # the run continues as if the skipped epoch had not been asked for
+        g.epoch = ref.epoch
+        assert np.max(np.abs(g.train_epoch() - ref.train_epoch())) <= 1e-5
+        for k in range(g.K):
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+        with pytest.raises(pkg().GadError):
+            g.debug_expire_wait(0)
+
+
+def test_set_inputs_rejects_labels_outside_the_classes(tiny):
+    w = tiny
+    theta = glorot_params(w.dims, np.random.default_rng(14))
+    with pkg().from_workload(w, theta) as g:
+        bad = w.labels.copy()
+        bad[7] = w.dims[-1]
+        with pytest.raises(pkg().GadError) as e:
+            g.set_inputs(None, bad)
+        assert e.value.code == -2
+        bad[7] = -1
+        with pytest.raises(pkg().GadError) as e:
+            g.set_inputs(w.X, bad)
+        assert e.value.code == -2
+        assert np.all(np.isfinite(g.train_epoch()))      # nothing was enqueued; the old labels are still in place

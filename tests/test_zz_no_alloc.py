@@ -5,7 +5,8 @@ memory pool, or the call sits in a loop where an allocation (and the device sync
 acceptable.  For them the library offers one entry point that needs no context and no workspace and keeps its
 partial sums in a fixed array inside the library.  This test calls it through the C ABI twice in a row, on two
 different workloads, so the second call runs over whatever the first left in that shared array, and checks both
-results against the regular entry point (gad_subgraph_weights of a context built on the same inputs).
+results against the regular entry point (gad_subgraph_weights of a context built on the same inputs), whose own
+values are compared with the CPU oracle's zeta first.
 
 The file is collected last on purpose, so a failure here cannot hide any other test behind `-x`.
 """
@@ -24,14 +25,21 @@ def built():
 
 
 def reference_and_inputs(w):
-    """zeta / w from the regular entry point, and the same inputs as plain device tensors."""
+    """zeta / w from the regular entry point, and the same inputs as plain device tensors.  The regular entry point's
+    zeta is itself held against the oracle's definition (Section 3.4.1, aggregate reading) here, so this file stands on
+    the oracle and not only on the library's other path."""
     import torch
     import paper_2110_02987_b200 as pkg
+    from oracle import gad_oracle as orc
     theta = glorot_params(w.dims, np.random.default_rng(0))
     with pkg.from_workload(w, theta) as g:
         zeta, wts = g.subgraph_weights()
         st = g.get_store()
         X = g.get_activation(0)                       # input features in store-row order [N' x F]
+    off = st["sub_off"]
+    z_orc = np.array([orc.zeta_aggregate(st["deg"][off[k]:off[k + 1]], X[off[k]:off[k + 1]]) for k in range(len(off) - 1)])
+    assert np.max(np.abs(zeta - z_orc) / z_orc) <= 1e-6
+    assert np.max(np.abs(wts - z_orc / z_orc.sum())) <= 1e-6
     F = X.shape[1]
     ld = (F + 3) // 4 * 4
     Xp = np.zeros((X.shape[0], ld), dtype=np.float32)
