@@ -49,31 +49,69 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples the SM clock and the throttle reasons of one GPU while the timed region runs: through NVML every 20 ms
+    (reading only), or, without the NVML module, through nvidia-smi every 100 ms."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index = index
-        self.rows = []
+        self.rows = []          # [sm MHz, max MHz, {reason names}]
         self.proc = None
+        self.stop = threading.Event()
+        self.thread = None
+
+    def _nvml_loop(self, nv, handle):
+        masks = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown, "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown, "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        mx = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+        while not self.stop.is_set():
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM))
+                bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(handle))
+                self.rows.append([sm, mx, {name for name, m in masks.items() if bits & m}])
+            except Exception:
+                pass
+            self.stop.wait(0.02)
+
+    def _smi_loop(self):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.proc.stdout:
+            r = [t.strip() for t in line.split(",")]
+            try:
+                self.rows.append([float(r[0]), float(r[1]), {n for n, f in zip(names, r[3:7]) if f.lower().startswith("active")}])
+            except (ValueError, IndexError):
+                continue
 
     def __enter__(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            # NVML numbers the GPUs of the machine; CUDA_VISIBLE_DEVICES may renumber them for this process
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            ids = [v.strip() for v in vis.split(",") if v.strip()]
+            handle = None
+            if ids and self.index < len(ids):
+                handle = nv.nvmlDeviceGetHandleByIndex(int(ids[self.index])) if ids[self.index].isdigit() else nv.nvmlDeviceGetHandleByUUID(ids[self.index])
+            if handle is None:
+                handle = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, handle), daemon=True)
+            self.thread.start()
+            return self
+        except Exception:
+            pass
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
                                           "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread = threading.Thread(target=self._smi_loop, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
         return self
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([t.strip() for t in line.split(",")])
-
     def __exit__(self, *a):
+        self.stop.set()
         if self.proc is not None:
             time.sleep(0.15)
             self.proc.terminate()
@@ -81,22 +119,16 @@ class ClockSampler:
                 self.proc.wait(timeout=5)
             except Exception:
                 self.proc.kill()
+        if self.thread is not None:
             self.thread.join(timeout=2)
 
     def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except (ValueError, IndexError):
-                continue
-            for name, flag in zip(names, r[3:7]):
-                if flag.lower().startswith("active"):
-                    reasons.add(name)
+        sm = [r[0] for r in self.rows]
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+        reasons = set().union(*[r[2] for r in self.rows])
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(r[1] for r in self.rows)), "reasons": sorted(reasons),
+                "samples": len(sm)}
 
 
 def max_over_ranks(ms, world, device="cpu"):
@@ -207,23 +239,15 @@ def cpu_baseline(w, theta, budget_s=20.0):
     return {"value": frac / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": "one step: " + sample}
 
 
-def run_micro_consensus(args):
-    """HBM-sized point for the update and consensus kernel: K = 8 replicas of one 4096 x 4096 layer (P = 16.8 M
-    parameters, 0.5 GB per set of copies) over a small graph.  Prints one JSON line: the kernel's time inside an epoch
-    (SGD step + weighted consensus: 12 K P bytes) and inside gad_consensus (consensus alone: 8 K P bytes), against the measured
-    copy rate."""
-    import torch
-    import __graft_entry__ as entry
+def consensus_point(K, D, steps, hbm_peak):
+    """Update + weighted consensus over K copies of one D x D layer: the kernel's time inside an epoch (SGD step and
+    consensus, 12 K P bytes) and inside gad_consensus (consensus alone, 8 K P bytes) by per-kernel CUDA events."""
     from gad_synth.graphs import sbm_graph
     from gad_synth.partition import contiguous_partition, one_hop_halo
     from gad_synth import glorot_params
     import paper_2110_02987_b200 as pkg
-    if not os.path.exists(pkg.LIB_PATH):
-        entry.build()
-    torch.cuda.set_device(0)
-    torch.cuda.set_stream(torch.cuda.Stream())
     rng = np.random.default_rng(0)
-    K, D, bs = 8, int(args.F) if args.F > 128 else 4096, 128
+    bs = 128
     rowptr, col, block = sbm_graph(K, bs, 0.05, 0.002, rng)
     n = K * bs
     X = rng.standard_normal((n, D), dtype=np.float32)
@@ -236,15 +260,16 @@ def run_micro_consensus(args):
     theta = glorot_params((D, D), rng)
     g = pkg.Gad(n, rowptr, col, cp, np.concatenate(core).astype(np.int32), hp,
                 np.concatenate(halo).astype(np.int32) if hp[-1] else np.empty(0, np.int32), X, y, split, (D, D), init_params=theta)
-    hbm_peak, _, peak_kind = measured_peaks()
     for _ in range(3):
         g.train_epoch(wait=False)
     g.profile_enable(True); g.profile_reset()
-    for _ in range(args.steps or 10):
+    for _ in range(steps):
         g.train_epoch(wait=False)
     prof = {e["name"]: e for e in g.profile_read()}
     e = prof["sgd_consensus"]
     ms_in = e["total_ms"] / e["launches"]
+    z = prof["zeta"]
+    ms_zeta = z["total_ms"] / z["launches"]
     g.profile_reset()
     for _ in range(20):
         g.consensus()    # importance weights, then the weighted mean written to all copies
@@ -253,14 +278,153 @@ def run_micro_consensus(args):
     c = prof["consensus"]
     ms_alone = c["total_ms"] / c["launches"]
     P = g.P
-    line = {"micro": "consensus", "K": K, "P": P, "bytes_per_copy_set": 4 * K * P,
+    line = {"micro": "consensus", "K": K, "layer": "%d-%d" % (D, D), "P": P, "bytes_per_copy_set": 4 * K * P,
             "sgd_consensus_in_epoch": {"ms": ms_in, "bytes": e["bytes_per_launch"], "GBps": e["bytes_per_launch"] / ms_in / 1e6,
                                        "frac": e["bytes_per_launch"] / ms_in / 1e6 / hbm_peak},
             "gad_consensus": {"ms": ms_alone, "bytes": 8.0 * K * P, "GBps": 8.0 * K * P / ms_alone / 1e6,
                               "frac": 8.0 * K * P / ms_alone / 1e6 / hbm_peak},
-            "peak": hbm_peak, "peak_source": peak_kind, "unit": "GB/s"}
+            "zeta": {"ms": ms_zeta, "bytes": z["bytes_per_launch"], "GBps": z["bytes_per_launch"] / ms_zeta / 1e6},
+            "peak": hbm_peak, "unit": "GB/s"}
     g.destroy()
+    return line
+
+
+def run_micro_consensus(args):
+    """The update and consensus kernel by itself.  Default: an HBM-sized point, K = 8 replicas of one 4096 x 4096 layer
+    (P = 16.8 M parameters, 0.5 GB per set of copies).  With --F 256 and --K k: k copies of a 256-256 layer (the point the
+    sweep configuration names; 0.26 MB per copy, launch-latency bound).  One JSON line against the measured copy rate."""
+    import torch
+    import __graft_entry__ as entry
+    import paper_2110_02987_b200 as pkg
+    if not os.path.exists(pkg.LIB_PATH):
+        entry.build()
+    torch.cuda.set_device(0)
+    torch.cuda.set_stream(torch.cuda.Stream())
+    hbm_peak, _, peak_kind = measured_peaks()
+    D = int(args.F) if args.F > 128 else 4096
+    line = consensus_point(args.K if args.F > 128 else 8, D, args.steps or 10, hbm_peak)
+    line["peak_source"] = peak_kind
     print(json.dumps(line))
+
+
+def grid_point(w, args, hbm_peak):
+    """One point of the sweep: epochs/s with everything resident, then one pass with per-kernel CUDA events."""
+    import torch
+    from gad_synth import glorot_params
+    import paper_2110_02987_b200 as pkg
+    theta = glorot_params(w.dims, np.random.default_rng(0))
+    g = pkg.from_workload(w, theta, gemm_mode=args.gemm_mode, flags=args.flags)
+    steps = args.steps or 10
+    for _ in range(max(args.warmup, 3)):
+        g.train_epoch(wait=False)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        g.train_epoch(wait=False)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    g.profile_enable(True); g.profile_reset()
+    for _ in range(steps):
+        g.train_epoch(wait=False)
+    prof = {e["name"]: e for e in g.profile_read()}
+    g.profile_enable(False)
+
+    def rate(name):
+        e = prof.get(name)
+        if not e or e["total_ms"] <= 0:
+            return None
+        t = e["total_ms"] / e["launches"]
+        return {"ms": t, "GBps": e["bytes_per_launch"] / t / 1e6, "frac": e["bytes_per_launch"] / t / 1e6 / hbm_peak,
+                "TFLOPs": e["flops_per_launch"] / t / 1e9}
+    F = w.dims[0]
+    line = {"grid": w.name, "mean_deg": w.extra.get("mean_deg"), "F": F, "K": w.K, "n_prime": g.n_prime, "nnz_prime": g.nnz_prime,
+            "epochs_per_s": 1e3 / ms, "ms_per_epoch": ms, "edges_per_s": g.nnz_prime * 1e3 / ms,
+            # the net is F-F-F-16: layer 0 aggregates the features first (forward only), layer 1 transforms first (an F-wide
+            # aggregation forward and its transposed one on the way back), layer 2 runs at 16 columns
+            "spmm_fwd_F": rate("spmm_fwd_l1"), "spmm_bwd_F": rate("spmm_bwd_l1"), "spmm_fwd_F_input": rate("spmm_fwd_l0"),
+            "spmm_fwd_16": rate("spmm_fwd_l2"), "spmm_bwd_16": rate("spmm_bwd_l2"),
+            "gemm_fwd_FxF": rate("gemm_fwd_l1"), "gemm_dw_FxF": rate("gemm_dw_l1"), "gemm_dh_FxF": rate("gemm_dh_l1"), "zeta": rate("zeta"),
+            "sgd_consensus": rate("sgd_consensus"), "dtype": "f32" if args.gemm_mode == 0 else "tf32 operands, f32 accumulate"}
+    g.destroy()
+    return line
+
+
+def run_grid(args):
+    """The sweep configuration as a grid: mean degree {8, 32, 128, 256} x feature width {64, 128, 256, 512} at K = 8, and
+    K in {2, 32, 64} at (mean degree 32, F = 128), on the 1 M-node Chung-Lu graph (each graph drawn once per degree);
+    then the update + consensus kernel over K in {2, 8, 32, 64} copies of a 256-256 layer.  One JSON line per point."""
+    import torch
+    import __graft_entry__ as entry
+    from gad_synth import sweep_family
+    import paper_2110_02987_b200 as pkg
+    if not os.path.exists(pkg.LIB_PATH):
+        entry.build()
+    torch.cuda.set_device(0)
+    torch.cuda.set_stream(torch.cuda.Stream())
+    hbm_peak, _, peak_kind = measured_peaks()
+    degs = [float(d) for d in args.grid_degs.split(",")]
+    Fs = [int(f) for f in args.grid_F.split(",")]
+    for deg in degs:
+        Ks = (8, 2, 32, 64) if deg == 32 and not args.grid_no_K else (8,)
+        for w in sweep_family(deg, Ks, Fs, scale=args.scale):
+            if w.K != 8 and w.dims[0] != 128:
+                continue
+            w.extra["mean_deg"] = deg
+            line = grid_point(w, args, hbm_peak)
+            line["peak"], line["peak_source"] = hbm_peak, peak_kind
+            print(json.dumps(line), flush=True)
+    for K in (2, 8, 32, 64):
+        line = consensus_point(K, 256, 50, hbm_peak)
+        line["peak_source"] = peak_kind
+        print(json.dumps(line), flush=True)
+
+
+def run_micro_gather(args):
+    """Where the aggregation's ceiling lies on this GPU: the library's own SpMM at width F on 1 M-row graphs of mean
+    degree 32 whose neighbours fall within a window of W rows around the row, so the operand rows an SM gathers come
+    from L1 (W = 64: 64 KB at F = 256), from L2 (W = 16 384: 16 MB) or from HBM (W = all rows: 1 GB).  Per window one
+    JSON line: time of the F-wide aggregation, operand bytes gathered per second (4 F bytes per stored entry) and the
+    algorithmic bytes per second."""
+    import torch
+    import __graft_entry__ as entry
+    from gad_synth.graphs import csr_from_pairs
+    from gad_synth import glorot_params
+    import paper_2110_02987_b200 as pkg
+    if not os.path.exists(pkg.LIB_PATH):
+        entry.build()
+    torch.cuda.set_device(0)
+    torch.cuda.set_stream(torch.cuda.Stream())
+    hbm_peak, _, peak_kind = measured_peaks()
+    n, deg, F = int(round((1 << 20) * args.scale)), int(args.mean_deg), int(args.F)
+    rng = np.random.default_rng(0)
+    X = rng.standard_normal((n, F), dtype=np.float32)
+    y = rng.integers(0, 16, size=n).astype(np.int32)
+    split = np.zeros(n, dtype=np.uint8)
+    theta = glorot_params((F, F, 16), rng)
+    for window in [int(x) for x in args.windows.split(",")]:
+        W = n if window <= 0 else min(window, n)
+        u = np.repeat(np.arange(n, dtype=np.int64), deg // 2)
+        v = (u + rng.integers(1, max(2, W // 2 + 1), size=u.shape[0])) % n
+        rowptr, col = csr_from_pairs(n, u, v)
+        cp = np.array([0, n], dtype=np.int64)
+        hp = np.zeros(2, dtype=np.int64)
+        g = pkg.Gad(n, rowptr, col, cp, np.arange(n, dtype=np.int32), hp, np.empty(0, np.int32), X, y, split, (F, F, 16), init_params=theta)
+        for _ in range(3):
+            g.train_epoch(wait=False)
+        g.profile_enable(True); g.profile_reset()
+        for _ in range(args.steps or 10):
+            g.train_epoch(wait=False)
+        prof = {e["name"]: e for e in g.profile_read()}
+        g.profile_enable(False)
+        e = prof["spmm_fwd_l0"]
+        ms = e["total_ms"] / e["launches"]
+        gathered = 4.0 * g.nnz_prime * F
+        print(json.dumps({"micro": "gather", "window_rows": W, "window_bytes": 4 * F * W, "rows": n, "nnz": g.nnz_prime, "F": F,
+                          "ms": ms, "gather_TBps": gathered / ms / 1e9, "algorithmic_GBps": e["bytes_per_launch"] / ms / 1e6,
+                          "frac_of_hbm_peak": e["bytes_per_launch"] / ms / 1e6 / hbm_peak, "peak": hbm_peak, "peak_source": peak_kind}), flush=True)
+        g.destroy()
 
 
 def run_micro_augment(args):
@@ -392,12 +556,23 @@ def main():
     ap.add_argument("--kernels", action="store_true", help="also print the per-kernel table to stderr")
     ap.add_argument("--shard", action="store_true",
                     help="spread the K subgraphs over the ranks (one all-reduce per epoch) instead of running N replicas of the job")
-    ap.add_argument("--micro", default=None, choices=["consensus", "augment"],
+    ap.add_argument("--grid", action="store_true", help="with --workload sweep: the whole degree x width (x K) grid, one JSON line per point")
+    ap.add_argument("--grid-degs", default="8,32,128,256")
+    ap.add_argument("--grid-F", default="64,128,256,512")
+    ap.add_argument("--grid-no-K", action="store_true", help="leave out the K = 2, 32, 64 points")
+    ap.add_argument("--windows", default="64,1024,16384,0", help="--micro gather: neighbour windows in rows (0 = all rows)")
+    ap.add_argument("--micro", default=None, choices=["consensus", "augment", "gather"],
                     help="a single point instead of the epoch benchmark (consensus: K = 8 copies of a 4096 x 4096 layer; "
                          "augment: Algorithm 1 on the workload's partition)")
     args = ap.parse_args()
     if args.micro == "consensus":
         run_micro_consensus(args)
+        return
+    if args.micro == "gather":
+        run_micro_gather(args)
+        return
+    if args.grid:
+        run_grid(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "gad" else args.warmup
     if args.steps is None:

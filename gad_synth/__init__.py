@@ -26,6 +26,7 @@ from .partition import (  # noqa: F401
 from .workloads import (  # noqa: F401
     Workload,
     make_workload,
+    sweep_family,
     glorot_params,
     param_count,
     WORKLOADS,

@@ -133,6 +133,34 @@ def _c3(K, rng, scale):
                "halo .05 of core" % (mean_deg, K))
 
 
+def sweep_family(mean_deg: float, Ks, Fs, *, seed: int = 0, scale: float = 1.0):
+    """The sweep workloads of one mean degree, for every feature width in ``Fs`` and every K in ``Ks``, with the graph
+    drawn once and every partition grown once.  Each yielded workload equals ``make_workload("sweep", mean_deg=...,
+    F=..., K=...)`` bit for bit (the generator draws the graph before the features, and the partition draws nothing)."""
+    rng = np.random.default_rng(seed)
+    n = max(64 * max(Ks), int(round(1_000_000 * scale)))
+    rowptr, col, comm = chung_lu_graph(n, 2.1, mean_deg, 16, 0.7, rng)
+    state = rng.bit_generator.state
+    y = (comm % 16).astype(np.int32)
+    parts = {}
+    for K in Ks:
+        core = bfs_partition(rowptr, col, K)
+        parts[K] = (core, one_hop_halo(rowptr, col, core, frac_of_core=0.05))
+    for F in Fs:
+        rng.bit_generator.state = state
+        X = rng.standard_normal((n, F), dtype=np.float32)
+        split = _split(n, rng)
+        for K in Ks:
+            core, halo = parts[K]
+            w = Workload(
+                name="sweep_d%g_f%d_k%d" % (mean_deg, F, K), n=n, rowptr=rowptr, col=col, X=X, labels=y, split=split, core=core,
+                halo=halo, dims=(F, F, F, 16), lr=0.01, epochs=1,
+                recipe="Chung-Lu gamma=%.1f mean degree %g, %d planted communities (p_intra .7); N(0,1)^%d; "
+                       "K=%d BFS blocks; halo %g of core" % (2.1, mean_deg, 16, F, K, 0.05))
+            w.seed = seed
+            yield w
+
+
 WORKLOADS = ("tiny", "tiny_signal", "c2", "c3k4", "c3k8", "c4", "sweep")
 
 
@@ -159,7 +187,7 @@ def make_workload(name: str, *, seed: int = 0, scale: float = 1.0, **kw) -> Work
         K = int(kw.get("K", 8))
         deg = float(kw.get("mean_deg", 32))
         w = _chung_lu("sweep_d%g_f%d_k%d" % (deg, F, K), 1_000_000, 2.1, deg, 16, 16, F, K, 0.05,
-                      (F, F, 16), 1, rng, scale)
+                      (F, F, F, 16), 1, rng, scale)
     else:
         raise ValueError("unknown workload %r" % name)
     w.seed = seed

@@ -79,8 +79,10 @@ typedef struct {
     int32_t gemm_mode;    /* 0: fp32-accurate transform (SIMT, or tensor cores with every operand split in two);  *
                            * 1: reduced-precision operands with fp32 accumulation: one TF32 pass on the tensor      *
                            *    cores, and the aggregation gathers a bfloat16 copy of its operand (tolerance 5e-2)  */
-    int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form, O(n'^2 F_0) per subgraph       *
-                           * (GAD_ERR_UNSUPPORTED when a subgraph has more than 32768 rows); 2: the aggregate  *
+    int32_t zeta_mode;    /* 0: aggregate distance term; 1: literal pairwise form, O(n'^2 F_0) per subgraph, the  *
+                           * squared distances from a Gram matrix on the tensor cores (any subgraph size; with   *
+                           * flag bit 0 or 4 from the differences on the FP32 ALUs, GAD_ERR_UNSUPPORTED when a    *
+                           * subgraph has more than 32768 rows); 2: the aggregate                               *
                            * term with the sum over layers of the variance equation (Section 3.4.1) kept: the  *
                            * squared distances are summed over the inputs H^(0) .. H^(L-1) of all layers, as   *
                            * the most recent forward pass left them, so zeta changes from epoch to epoch        */
@@ -92,7 +94,11 @@ typedef struct {
                              bit 2: the backward pass of a layer of at most 16 output columns also goes through the
                              tensor-core transforms instead of the streaming FP32 kernel written for it (for
                              comparison);
-                             bit 3: never replay an epoch as a CUDA graph (see gad_train_epoch)                */
+                             bit 3: never replay an epoch as a CUDA graph (see gad_train_epoch);
+                             bit 4: zeta_mode 1 on the FP32 ALUs (difference form) instead of the tensor cores;
+                             bit 5: layers l >= 1 always transform before they aggregate (by default a layer whose
+                             input is narrower than its output aggregates first, sigma((A~ H^(l)) W + b): the same
+                             product in the other order, with both of its SpMMs at the narrower width)              */
 } gad_config;
 
 /* Bytes of device workspace gad_create needs for these inputs.  Host-only; touches no GPU. */
@@ -113,6 +119,11 @@ int gad_workspace_bytes(const gad_csr* g, const gad_partition* part, const gad_c
 int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const float* X, const int32_t* labels,
                const uint8_t* split, const gad_config* cfg, const float* init_params, void* workspace,
                size_t workspace_bytes, void* stream);
+
+/* The parameters gad_create starts from when init_params is NULL, host [P] in the layout above: W_l uniform in (-a, a)
+ * with a = sqrt(6 / (F_l + F_{l+1})) (Glorot), drawn from a splitmix64 stream of `seed`; biases zero.  Host-only.  (The
+ * paper does not say how its models are initialised.) */
+int gad_default_params(int32_t L, const int32_t* dims, uint64_t seed, float* out);
 
 /* One pass of Algorithm 2 (one subgraph per processor): for every replica k
  *   forward   H^(l+1) = sigma(A~_k (H^(l) W_k^(l)) + b_k^(l)), sigma = ReLU (identity on the last layer), with
@@ -280,8 +291,9 @@ int gad_subgraph_weights_static(const float* X, int64_t rows, int32_t F, int32_t
  * first d |B| walks (d = average degree of the boundary nodes) the number of walks n follows the Monte-Carlo error
  * equation, n = (zc sigma / (mean E))^2, at most cap times the first batch; walks are ranked by the sum of I over
  * their outside nodes and their nodes are taken in walk order until alpha (1 + density) |v_i| nodes are selected.
- * The boundary test, the walks, the counts, their statistics and the walk scores run on the GPU; the ranking and
- * the selection loop on the host.  Every random number is mix(seed, subgraph, walk, step) (splitmix64 output
+ * The boundary test, the density count, the walks, the counts, their statistics, the walk scores and the selection of
+ * the leading walks (the few thousand best-ranked ones, all the selection loop normally reaches) run on the GPU; the
+ * order among those and the selection loop, which is sequential by definition, on the host.  Every random number is mix(seed, subgraph, walk, step) (splitmix64 output
  * function), so the result is a pure function of the arguments. */
 typedef struct {
     int32_t steps;   /* walk length l = number of GCN layers, 1 .. 8                                      */
@@ -290,6 +302,9 @@ typedef struct {
     double E;        /* Monte-Carlo error bound; the paper uses 0.05                                       */
     double zc;       /* confidence statistic; 1.96 for the paper's 95 % level                              */
     uint64_t seed;
+    int32_t graph_resident; /* 0: copy g to the device; 1: the caller vouches that an earlier gad_augment call with   *
+                             * this very workspace and the same g (n, nnz, rowptr, col unchanged) left it there:  *
+                             * the copy is skipped (the graph sits at the start of the workspace)                   */
 } gad_augment_config;
 
 /* Bytes of device workspace gad_augment needs.  Host-only. */

@@ -16,7 +16,7 @@ For every subgraph g_i = (v_i, e_i) of a partition of G (steps in the order of A
                      walk that lie outside v_i and are not selected yet are added in walk order until n(g_i) are selected
                      ("depth-first": a selected node is reached from v_i through selected nodes of the same walk)
 
-Readings where the paper is silent (listed in the design doc): the random draws come from a counter-based generator,
+Readings where the paper is silent: the random draws come from a counter-based generator,
 draw(i, j, s) = mix(mix(mix(seed + G (1 + i)) + G (1 + j)) + G (1 + s)) with the splitmix64 output function `mix` and
 its increment G, reduced modulo the number of choices; a node counts once per walk; sigma is the population standard
 deviation; sigma / mean is evaluated from the integer sums of the counts, n = ceil((z_c / E)^2 (m S2 / S1^2 - 1));

@@ -27,7 +27,7 @@ SYMBOLS = (
     "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_subgraph_weights_static", "gad_launch_count",
     "gad_last_error", "gad_destroy", "gad_train_epoch_local", "gad_consensus_floats", "gad_consensus_partial",
     "gad_consensus_apply", "gad_export_params", "gad_get_train_counts", "gad_augment_workspace_bytes", "gad_augment",
-    "gad_augment_last_error", "gad_debug_expire_wait",
+    "gad_augment_last_error", "gad_debug_expire_wait", "gad_default_params",
 )
 
 
@@ -398,42 +398,81 @@ def launch_count() -> int:
 
 class _AugmentConfig(C.Structure):
     _fields_ = [("steps", C.c_int32), ("cap", C.c_int32), ("alpha", C.c_double), ("E", C.c_double), ("zc", C.c_double),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("graph_resident", C.c_int32)]
+
+
+def default_params(dims, seed=0):
+    """gad_default_params: the seeded Glorot-uniform initialisation gad_create uses when it is given none (host-only)."""
+    dims_a = np.asarray(dims, dtype=np.int32)
+    P = int(sum(int(dims_a[l]) * int(dims_a[l + 1]) + int(dims_a[l + 1]) for l in range(len(dims_a) - 1)))
+    out = np.zeros(P, dtype=np.float32)
+    rc = load().gad_default_params(C.c_int32(len(dims_a) - 1), _ptr(dims_a, C.c_int32), C.c_uint64(seed), _ptr(out, C.c_float))
+    if rc != GAD_OK:
+        raise GadError(rc)
+    return out
+
+
+class Augmenter:
+    """gad_augment for one graph and several calls: the device workspace is kept between calls, and from the second call
+    on (same workspace, same graph) the graph is not copied to the device again (``graph_resident``)."""
+
+    def __init__(self, n, rowptr, col):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the GAD library needs a CUDA device (there is no CPU fallback)")
+        self._L = load()
+        self._L.gad_augment_last_error.restype = C.c_char_p
+        self.n = int(n)
+        self.rowptr = _arr(rowptr, np.int64)
+        self.col = _arr(col, np.int32)
+        self._csr = gad_csr(self.n, int(self.rowptr[-1]), _ptr(self.rowptr, C.c_int64), _ptr(self.col, C.c_int32), None)
+        self._ws = None
+        self._ws_bytes = 0
+        self._resident = False
+
+    def _fail(self, rc):
+        raise GadError(rc, (self._L.gad_augment_last_error() or b"").decode())
+
+    def run(self, cores, steps, *, alpha=0.01, E=0.05, zc=1.96, seed=0, cap=4, stream=None):
+        """The replication-node list of every core set (Algorithm 1 of the paper) on the current CUDA device.
+        Returns (list of int32 arrays in selection order, int64 array of the walks drawn per subgraph)."""
+        import torch
+        L = self._L
+        K = len(cores)
+        cp = np.zeros(K + 1, dtype=np.int64)
+        np.cumsum([len(c) for c in cores], out=cp[1:])
+        cn = _arr(np.concatenate(cores) if cp[-1] > 0 else np.empty(0, np.int32), np.int32)
+        cfg = _AugmentConfig(int(steps), int(cap), float(alpha), float(E), float(zc), int(seed), 0)
+        nbytes = C.c_size_t(0)
+        rc = L.gad_augment_workspace_bytes(C.byref(self._csr), C.c_int32(K), _ptr(cp, C.c_int64), _ptr(cn, C.c_int32), C.byref(cfg),
+                                           C.byref(nbytes))
+        if rc != GAD_OK:
+            self._fail(rc)
+        if self._ws is None or int(nbytes.value) > self._ws_bytes:
+            self._ws = torch.empty(int(nbytes.value) + 256, dtype=torch.uint8, device="cuda")
+            self._ws_bytes = int(nbytes.value)
+            self._resident = False
+        cfg.graph_resident = 1 if self._resident else 0
+        aligned = (self._ws.data_ptr() + 255) // 256 * 256
+        st = stream if stream is not None else torch.cuda.current_stream()
+        capacity = int(sum(int(np.floor(alpha * 2.0 * len(c))) for c in cores)) + 1
+        halo_ptr = np.zeros(K + 1, dtype=np.int64)
+        halo = np.zeros(capacity, dtype=np.int32)
+        walks = np.zeros(K, dtype=np.int64)
+        rc = L.gad_augment(C.byref(self._csr), C.c_int32(K), _ptr(cp, C.c_int64), _ptr(cn, C.c_int32), C.byref(cfg), C.c_void_p(aligned),
+                           C.c_size_t(self._ws_bytes), C.c_void_p(st.cuda_stream), _ptr(halo_ptr, C.c_int64), _ptr(halo, C.c_int32),
+                           C.c_int64(capacity), _ptr(walks, C.c_int64))
+        if rc != GAD_OK:
+            self._resident = False
+            self._fail(rc)
+        self._resident = True
+        return [halo[halo_ptr[k]:halo_ptr[k + 1]].copy() for k in range(K)], walks
 
 
 def augment(n, rowptr, col, cores, steps, *, alpha=0.01, E=0.05, zc=1.96, seed=0, cap=4, stream=None):
-    """gad_augment: the replication-node list of every core set (Algorithm 1 of the paper) on the current CUDA device.
-    Returns (list of int32 arrays in selection order, int64 array of the walks drawn per subgraph)."""
-    import torch
-    if not torch.cuda.is_available():
-        raise RuntimeError("the GAD library needs a CUDA device (there is no CPU fallback)")
-    L = load()
-    L.gad_augment_last_error.restype = C.c_char_p
-    rowptr = _arr(rowptr, np.int64)
-    col = _arr(col, np.int32)
-    K = len(cores)
-    cp = np.zeros(K + 1, dtype=np.int64)
-    np.cumsum([len(c) for c in cores], out=cp[1:])
-    cn = _arr(np.concatenate(cores) if cp[-1] > 0 else np.empty(0, np.int32), np.int32)
-    csr = gad_csr(int(n), int(rowptr[-1]), _ptr(rowptr, C.c_int64), _ptr(col, C.c_int32), None)
-    cfg = _AugmentConfig(int(steps), int(cap), float(alpha), float(E), float(zc), int(seed))
-    nbytes = C.c_size_t(0)
-    rc = L.gad_augment_workspace_bytes(C.byref(csr), C.c_int32(K), _ptr(cp, C.c_int64), _ptr(cn, C.c_int32), C.byref(cfg), C.byref(nbytes))
-    if rc != GAD_OK:
-        raise GadError(rc, (L.gad_augment_last_error() or b"").decode())
-    ws = torch.empty(int(nbytes.value) + 256, dtype=torch.uint8, device="cuda")
-    aligned = (ws.data_ptr() + 255) // 256 * 256
-    st = stream if stream is not None else torch.cuda.current_stream()
-    capacity = int(sum(int(np.floor(alpha * 2.0 * len(c))) for c in cores)) + 1
-    halo_ptr = np.zeros(K + 1, dtype=np.int64)
-    halo = np.zeros(capacity, dtype=np.int32)
-    walks = np.zeros(K, dtype=np.int64)
-    rc = L.gad_augment(C.byref(csr), C.c_int32(K), _ptr(cp, C.c_int64), _ptr(cn, C.c_int32), C.byref(cfg), C.c_void_p(aligned),
-                       C.c_size_t(int(nbytes.value)), C.c_void_p(st.cuda_stream), _ptr(halo_ptr, C.c_int64), _ptr(halo, C.c_int32),
-                       C.c_int64(capacity), _ptr(walks, C.c_int64))
-    if rc != GAD_OK:
-        raise GadError(rc, (L.gad_augment_last_error() or b"").decode())
-    return [halo[halo_ptr[k]:halo_ptr[k + 1]].copy() for k in range(K)], walks
+    """gad_augment, one call: the replication-node list of every core set (Algorithm 1 of the paper) on the current CUDA
+    device.  Returns (list of int32 arrays in selection order, int64 array of the walks drawn per subgraph)."""
+    return Augmenter(n, rowptr, col).run(cores, steps, alpha=alpha, E=E, zc=zc, seed=seed, cap=cap, stream=stream)
 
 
 def from_workload(w, init_params, **kw):

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgad.so")
-SOURCES = ["gad_api.cu", "store_host.cpp", "spmm.cu", "gemm_simt.cu", "gemm_tc.cu", "misc_kernels.cu", "zeta_pair.cu", "noalloc.cu", "narrow.cu", "augment.cu"]
+SOURCES = ["gad_api.cu", "store_host.cpp", "spmm.cu", "gemm_simt.cu", "gemm_tc.cu", "misc_kernels.cu", "zeta_pair.cu", "zeta_gram.cu", "noalloc.cu", "narrow.cu", "augment.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC,-fopenmp,-Wall", "--expt-relaxed-constexpr"]
 

@@ -12,6 +12,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <functional>
 #include <numeric>
 #include <string>
 #include <vector>
@@ -60,14 +61,26 @@ __host__ __device__ inline bool first_outside(const uint8_t* inside, const int32
     return true;
 }
 
+// flag[t] = core node t has a neighbour outside the core set; *inner += directed entries between two different core nodes
+// (2 |e_i| of the density definition; an integer sum, so the order of the additions does not matter).
 __global__ void boundary_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ core,
-                                int64_t ncore, const uint8_t* __restrict__ inside, uint8_t* __restrict__ flag) {
+                                int64_t ncore, const uint8_t* __restrict__ inside, uint8_t* __restrict__ flag,
+                                unsigned long long* __restrict__ inner) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= ncore) return;
-    const int32_t v = core[t];
-    uint8_t f = 0;
-    for (int64_t e = rowptr[v]; e < rowptr[v + 1] && !f; ++e) f = inside[col[e]] ? 0 : 1;
-    flag[t] = f;
+    unsigned long long mine = 0;
+    if (t < ncore) {
+        const int32_t v = core[t];
+        uint8_t f = 0;
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+            const int32_t c = col[e];
+            if (!inside[c]) f = 1;
+            else if (c != v) ++mine;
+        }
+        flag[t] = f;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(inner, mine);
 }
 __global__ void mark_kernel(const int32_t* __restrict__ core, int64_t ncore, uint8_t* __restrict__ inside, uint8_t value) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -85,7 +98,7 @@ __global__ void walk_count_kernel(const int64_t* __restrict__ rowptr, const int3
 }
 __global__ void walk_score_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ col, const int32_t* __restrict__ B,
                                   int64_t nB, const uint8_t* __restrict__ inside, uint64_t seed, int sub, int64_t nwalks, int steps,
-                                  const int32_t* __restrict__ count, int64_t* __restrict__ score) {
+                                  const int32_t* __restrict__ count, int64_t* __restrict__ score, unsigned long long* __restrict__ key) {
     const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= nwalks) return;
     int32_t seq[kMaxSteps + 1];
@@ -94,6 +107,36 @@ __global__ void walk_score_kernel(const int64_t* __restrict__ rowptr, const int3
     for (int s = 0; s <= steps; ++s)
         if (first_outside(inside, seq, s)) sc += count[seq[s]];
     score[j] = sc;
+    // ranking key: a better walk (higher score; equal scores: lower index) has the larger key, and no two walks share one
+    if (key) key[j] = ((unsigned long long)sc << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)j);
+}
+
+// Selection of the S largest ranking keys without sorting them all: the keys are unique, so the S-th largest one is found
+// digit by digit (13 bits at a time, from the top), each pass a histogram of the next digit over the keys that share the
+// digits fixed so far; the host reads the 8192 counts and fixes the digit.  A last pass gathers the keys >= that one.
+constexpr int kDigitBits = 13, kDigits = 1 << kDigitBits;
+__global__ void __launch_bounds__(256) key_hist_kernel(const unsigned long long* __restrict__ key, int64_t n, unsigned long long prefix_mask,
+                                                       unsigned long long prefix, int shift, unsigned* __restrict__ hist) {
+    __shared__ unsigned h[kDigits];
+    for (int i = threadIdx.x; i < kDigits; i += blockDim.x) h[i] = 0u;
+    __syncthreads();
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x) {
+        const unsigned long long k = key[j];
+        if ((k & prefix_mask) == prefix) atomicAdd(&h[(unsigned)(k >> shift) & (kDigits - 1)], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kDigits; i += blockDim.x)
+        if (h[i]) atomicAdd(hist + i, h[i]);
+}
+__global__ void __launch_bounds__(256) key_gather_kernel(const unsigned long long* __restrict__ key, int64_t n, unsigned long long least,
+                                                         unsigned long long* __restrict__ out, unsigned long long* __restrict__ n_out, int64_t cap) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    const unsigned long long k = key[j];
+    if (k >= least) {
+        const unsigned long long at = atomicAdd(n_out, 1ull);   // the host sorts what it gets: the order here is free
+        if ((int64_t)at < cap) out[at] = k;
+    }
 }
 // m = visited candidates, S1 = sum of counts, S2 = sum of squared counts
 __global__ void count_stats_kernel(const int32_t* __restrict__ count, int64_t n, unsigned long long* __restrict__ stats) {
@@ -114,7 +157,12 @@ __global__ void count_stats_kernel(const int32_t* __restrict__ count, int64_t n,
         for (int q = 0; q < 3; ++q) atomicAdd(stats + q, sm[q][0]);
 }
 
-struct AugPlan { size_t o_rowptr, o_col, o_inside, o_core, o_flag, o_B, o_count, o_stats, o_score, bytes; int64_t max_core, max_walks; };
+struct AugPlan {
+    size_t o_rowptr, o_col, o_inside, o_core, o_flag, o_B, o_count, o_stats, o_score, o_key, o_hist, o_top, bytes;
+    int64_t max_core, max_walks, max_top;   // max_top: most leading walks ever ranked on the device
+};
+// Leading walks whose order is established first: the selection loop rarely needs more (it then orders all of them).
+inline int64_t leading_walks(int64_t nwalks, int64_t n_rep) { return std::min<int64_t>(nwalks, std::max<int64_t>(1024, 8 * n_rep)); }
 
 size_t take(size_t& cur, size_t bytes) { size_t o = cur; cur += (size_t)round_up((int64_t)std::max<size_t>(bytes, 4), 256); return o; }
 
@@ -145,8 +193,11 @@ int plan_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int
     size_t cur = 0;
     p.o_rowptr = take(cur, 8 * (size_t)(g->n + 1)); p.o_col = take(cur, 4 * (size_t)g->nnz);
     p.o_inside = take(cur, (size_t)g->n); p.o_core = take(cur, 4 * (size_t)p.max_core); p.o_flag = take(cur, (size_t)p.max_core);
-    p.o_B = take(cur, 4 * (size_t)p.max_core); p.o_count = take(cur, 4 * (size_t)g->n); p.o_stats = take(cur, 24);
+    p.o_B = take(cur, 4 * (size_t)p.max_core); p.o_count = take(cur, 4 * (size_t)g->n); p.o_stats = take(cur, 40);
     p.o_score = take(cur, 8 * (size_t)p.max_walks);
+    // n(g_i) <= alpha (1 + d) |v_i| <= 2 alpha |v_i|
+    p.max_top = leading_walks(p.max_walks, (int64_t)std::floor(cfg->alpha * 2.0 * (double)p.max_core));
+    p.o_key = take(cur, 8 * (size_t)p.max_walks); p.o_hist = take(cur, 4 * (size_t)kDigits); p.o_top = take(cur, 8 * (size_t)p.max_top);
     p.bytes = cur;
     return GAD_OK;
 }
@@ -201,14 +252,21 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
     int32_t* d_count = (int32_t*)(ws + p.o_count);
     unsigned long long* d_stats = (unsigned long long*)(ws + p.o_stats);
     int64_t* d_score = (int64_t*)(ws + p.o_score);
+    unsigned long long* d_key = (unsigned long long*)(ws + p.o_key);
+    unsigned* d_hist = (unsigned*)(ws + p.o_hist);
+    unsigned long long* d_top = (unsigned long long*)(ws + p.o_top);
     const int64_t n = g->n;
     const int steps = cfg->steps;
-    AUG_CK(cudaMemcpyAsync(d_rowptr, g->rowptr, 8 * (size_t)(n + 1), cudaMemcpyHostToDevice, s));
-    if (g->nnz > 0) AUG_CK(cudaMemcpyAsync(d_col, g->col, 4 * (size_t)g->nnz, cudaMemcpyHostToDevice, s));
+    if (!cfg->graph_resident) {   // else: an earlier call left this very graph at the start of this workspace
+        AUG_CK(cudaMemcpyAsync(d_rowptr, g->rowptr, 8 * (size_t)(n + 1), cudaMemcpyHostToDevice, s));
+        if (g->nnz > 0) AUG_CK(cudaMemcpyAsync(d_col, g->col, 4 * (size_t)g->nnz, cudaMemcpyHostToDevice, s));
+    }
     AUG_CK(cudaMemsetAsync(d_inside, 0, (size_t)n, s));
     std::vector<uint8_t> inside((size_t)n, 0), flag;
     std::vector<int32_t> B, seq((size_t)steps + 1);
     std::vector<int64_t> score, order;
+    std::vector<unsigned long long> top;
+    std::vector<unsigned> hist((size_t)kDigits);
     std::vector<uint8_t> taken((size_t)n, 0);
     auto grid = [](int64_t work) { return (unsigned)((work + 255) / 256); };
     int64_t out = 0;
@@ -220,17 +278,18 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
         if (ncore > 0) {
             AUG_CK(cudaMemcpyAsync(d_core, core, 4 * (size_t)ncore, cudaMemcpyHostToDevice, s));
             mark_kernel<<<grid(ncore), 256, 0, s>>>(d_core, ncore, d_inside, 1); ++g_kernel_launches;
-            boundary_kernel<<<grid(ncore), 256, 0, s>>>(d_rowptr, d_col, d_core, ncore, d_inside, d_flag); ++g_kernel_launches;
+            AUG_CK(cudaMemsetAsync(d_stats + 3, 0, 16, s));
+            boundary_kernel<<<grid(ncore), 256, 0, s>>>(d_rowptr, d_col, d_core, ncore, d_inside, d_flag, d_stats + 3); ++g_kernel_launches;
             flag.resize((size_t)ncore);
+            unsigned long long inner_dev = 0;
             AUG_CK(cudaMemcpyAsync(flag.data(), d_flag, (size_t)ncore, cudaMemcpyDeviceToHost, s));
+            AUG_CK(cudaMemcpyAsync(&inner_dev, d_stats + 3, 8, cudaMemcpyDeviceToHost, s));
             AUG_CK(cudaStreamSynchronize(s));
             B.clear();
-            int64_t inner_directed = 0;
-            for (int64_t t = 0; t < ncore; ++t) inside[(size_t)core[t]] = 1;
+            const int64_t inner_directed = (int64_t)inner_dev;
             for (int64_t t = 0; t < ncore; ++t) {
+                inside[(size_t)core[t]] = 1;
                 if (flag[(size_t)t]) B.push_back(core[t]);
-                for (int64_t e = g->rowptr[core[t]]; e < g->rowptr[core[t] + 1]; ++e)
-                    inner_directed += (inside[(size_t)g->col[e]] && g->col[e] != core[t]) ? 1 : 0;
             }
             std::sort(B.begin(), B.end());
             const int64_t nB = (int64_t)B.size();
@@ -263,13 +322,15 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
                     count_stats_kernel<<<148 * 4, 256, 0, s>>>(d_count, n, d_stats); ++g_kernel_launches;
                     AUG_CK(cudaMemcpyAsync(st, d_stats, 24, cudaMemcpyDeviceToHost, s));
                 }
+                // a walk's score is at most (steps + 1) nwalks (a node counts once per walk): when score and walk index fit
+                // 32 bits each, the walks get unique 64-bit ranking keys and the leading ones are selected on the device
+                const bool keyed = nwalks > 0 && nwalks < ((int64_t)1 << 32) && (int64_t)(steps + 1) * nwalks < ((int64_t)1 << 31);
                 if (nwalks > 0) {
-                    walk_score_kernel<<<grid(nwalks), 256, 0, s>>>(d_rowptr, d_col, d_B, nB, d_inside, cfg->seed, k, nwalks, steps, d_count, d_score);
+                    walk_score_kernel<<<grid(nwalks), 256, 0, s>>>(d_rowptr, d_col, d_B, nB, d_inside, cfg->seed, k, nwalks, steps, d_count, d_score,
+                                                                   keyed ? d_key : nullptr);
                     ++g_kernel_launches;
                 }
-                score.resize((size_t)nwalks);
-                if (nwalks > 0) AUG_CK(cudaMemcpyAsync(score.data(), d_score, 8 * (size_t)nwalks, cudaMemcpyDeviceToHost, s));
-                AUG_CK(cudaStreamSynchronize(s));
+                AUG_CK(cudaStreamSynchronize(s));   // st (the statistics of the final counts) has arrived
                 // n(g_i) = alpha (1 + d(g_i)) |v_i|, at most the visited candidates
                 int64_t n_rep = 0;
                 if (ncore >= 2) {
@@ -280,17 +341,57 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
                 // walks in descending order of their summed importance (equal scores: ascending index).  Only the best
                 // walks are ever looked at, so the order is established for a leading stretch first and for all
                 // walks only if that stretch does not yield n(g_i) nodes.
-                order.resize((size_t)nwalks);
-                std::iota(order.begin(), order.end(), (int64_t)0);
                 auto better = [&](int64_t a, int64_t b) {
                     return score[(size_t)a] != score[(size_t)b] ? score[(size_t)a] > score[(size_t)b] : a < b;
                 };
-                int64_t sorted = std::min<int64_t>(nwalks, std::max<int64_t>(1024, 8 * n_rep));
-                if (n_rep > 0) std::partial_sort(order.begin(), order.begin() + sorted, order.end(), better);
+                auto order_all = [&]() -> int {   // every score to the host, every walk ranked there
+                    score.resize((size_t)nwalks);
+                    AUG_CK(cudaMemcpyAsync(score.data(), d_score, 8 * (size_t)nwalks, cudaMemcpyDeviceToHost, s));
+                    AUG_CK(cudaStreamSynchronize(s));
+                    order.resize((size_t)nwalks);
+                    std::iota(order.begin(), order.end(), (int64_t)0);
+                    std::sort(order.begin(), order.end(), better);
+                    return GAD_OK;
+                };
+                int64_t sorted = std::min(leading_walks(nwalks, n_rep), p.max_top);
+                if (n_rep > 0 && keyed && sorted < nwalks) {
+                    // the `sorted`-th largest key, digit by digit from the top; then the keys at least that large
+                    int top_bit = 32;
+                    while (top_bit < 63 && (((int64_t)(steps + 1) * nwalks) >> (top_bit - 32)) > 0) ++top_bit;
+                    unsigned long long prefix = 0, prefix_mask = 0;
+                    int64_t remaining = sorted;
+                    for (int d = (top_bit + kDigitBits - 1) / kDigitBits - 1; d >= 0; --d) {
+                        const int shift = d * kDigitBits;
+                        AUG_CK(cudaMemsetAsync(d_hist, 0, 4 * (size_t)kDigits, s));
+                        key_hist_kernel<<<148 * 2, 256, 0, s>>>(d_key, nwalks, prefix_mask, prefix, shift, d_hist); ++g_kernel_launches;
+                        AUG_CK(cudaMemcpyAsync(hist.data(), d_hist, 4 * (size_t)kDigits, cudaMemcpyDeviceToHost, s));
+                        AUG_CK(cudaStreamSynchronize(s));
+                        int b = kDigits - 1;
+                        for (; b > 0 && (int64_t)hist[(size_t)b] < remaining; --b) remaining -= hist[(size_t)b];
+                        prefix |= (unsigned long long)b << shift;
+                        prefix_mask |= (unsigned long long)(kDigits - 1) << shift;
+                    }
+                    AUG_CK(cudaMemsetAsync(d_stats + 4, 0, 8, s));
+                    key_gather_kernel<<<grid(nwalks), 256, 0, s>>>(d_key, nwalks, prefix, d_top, d_stats + 4, p.max_top); ++g_kernel_launches;
+                    unsigned long long got = 0;
+                    top.resize((size_t)sorted);
+                    AUG_CK(cudaMemcpyAsync(&got, d_stats + 4, 8, cudaMemcpyDeviceToHost, s));
+                    AUG_CK(cudaMemcpyAsync(top.data(), d_top, 8 * (size_t)sorted, cudaMemcpyDeviceToHost, s));
+                    AUG_CK(cudaStreamSynchronize(s));
+                    if ((int64_t)got != sorted) return aug_fail(GAD_ERR_CUDA, "selection of the leading walks came out with the wrong count");
+                    std::sort(top.begin(), top.end(), std::greater<unsigned long long>());
+                    order.resize((size_t)sorted);
+                    for (int64_t a = 0; a < sorted; ++a) order[(size_t)a] = (int64_t)(0xFFFFFFFFu - (uint32_t)(top[(size_t)a] & 0xFFFFFFFFull));
+                } else if (n_rep > 0) {
+                    int rc2 = order_all();
+                    if (rc2 != GAD_OK) return rc2;
+                    sorted = nwalks;
+                }
                 const int64_t first = out;
                 for (int64_t a = 0; a < nwalks && out - first < n_rep; ++a) {
-                    if (a == sorted) {   // the leading stretch is used up: order the rest as well
-                        std::sort(order.begin() + sorted, order.end(), better);
+                    if (a == sorted) {   // the leading stretch is used up: order all walks (the leading ones come out the same)
+                        int rc2 = order_all();
+                        if (rc2 != GAD_OK) return rc2;
                         sorted = nwalks;
                     }
                     make_walk(g->rowptr, g->col, B.data(), nB, cfg->seed, k, order[(size_t)a], steps, seq.data());

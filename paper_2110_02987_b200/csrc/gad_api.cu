@@ -59,11 +59,14 @@ struct Plan {
     int32_t maxld = 0;
     std::vector<RowSpan> tiles, chunks, dw_chunks, core_spans;
     std::vector<int32_t> chunk_ptr, dw_chunk_ptr;   // [K+1]
-    std::vector<int64_t> pair_ptr;    // [K+1] tiles of pairs per subgraph (zeta_mode 1), else empty
+    std::vector<int64_t> pair_ptr;    // [K+1] tiles of pairs per subgraph (zeta_mode 1 on the FP32 ALUs), else empty
     size_t o_pair_ptr = 0, o_pair_partial = 0;
+    std::vector<int64_t> gram_ptr;    // [K+1] 128 x 128 tiles of pairs per subgraph (zeta_mode 1 on the tensor cores)
+    size_t o_gram_ptr = 0, o_gram_partial = 0, o_norm2 = 0;
+    bool pair_alu_ok = false;         // every subgraph is small enough for the FP32-ALU pairwise kernel
     int64_t dw_partial = 0;           // floats per chunk
-    bool agg_first0 = false;          // layer 0 aggregates before it transforms
-    size_t o_P = 0;                   // A~ H^(0)  [Np x ld0], only with agg_first0
+    std::vector<uint8_t> agg_first;   // [L] the layer aggregates before it transforms: sigma((A~ H^(l)) W + b)
+    std::vector<size_t> o_P;          // [L] A~ H^(l)  [Np x ld_l] of those layers
     size_t o_counters = 0;            // arrival counters: [loss | K column sums | K zeta]
     // layers l >= 1 of at most 16 output columns take the streaming FP32 kernel on the way back (flag bit 2 switches it off)
     std::vector<uint8_t> narrow;      // [L]
@@ -95,12 +98,13 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     if (!(cfg->dropout >= 0.f && cfg->dropout < 1.f)) { err = "dropout must be in [0,1)"; return GAD_ERR_ARG; }
     if (cfg->gemm_mode != 0 && cfg->gemm_mode != 1) { err = "gemm_mode must be 0 or 1"; return GAD_ERR_ARG; }
     if (cfg->zeta_mode < 0 || cfg->zeta_mode > 2) { err = "zeta_mode must be 0, 1 or 2"; return GAD_ERR_ARG; }
-    if (cfg->zeta_mode == 1)   // O(n'^2 F_0) pairs per subgraph
-        for (int32_t k = 0; k < K; ++k)
-            if (sub_off[k + 1] - sub_off[k] > kZetaPairMaxRows) {
-                err = "zeta_mode 1 (pairwise form) takes subgraphs of at most " + std::to_string(kZetaPairMaxRows) + " rows";
-                return GAD_ERR_UNSUPPORTED;
-            }
+    p.pair_alu_ok = true;
+    for (int32_t k = 0; k < K; ++k)
+        if (sub_off[k + 1] - sub_off[k] > kZetaPairMaxRows) p.pair_alu_ok = false;
+    if (cfg->zeta_mode == 1 && (cfg->flags & (1 | 16)) != 0 && !p.pair_alu_ok) {   // the FP32-ALU form was asked for
+        err = "zeta_mode 1 on the FP32 ALUs (flag bits 0 / 4) takes subgraphs of at most " + std::to_string(kZetaPairMaxRows) + " rows";
+        return GAD_ERR_UNSUPPORTED;
+    }
     if (!(cfg->beta > 0.f)) { err = "beta must be positive"; return GAD_ERR_ARG; }
     p.n = n; p.K = K; p.L = cfg->L; p.nnz = nnz; p.Np = sub_off[K]; p.slots = slots;
     p.dims.assign(cfg->dims, cfg->dims + cfg->L + 1);
@@ -109,7 +113,12 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     for (int l = 0; l <= p.L; ++l) { p.ld[l] = (int32_t)round_up(p.dims[l], 4); p.maxld = std::max(p.maxld, p.ld[l]); }
     // Layer 0 needs no gradient with respect to its input, so aggregating first costs one SpMM at the width F_0 where
     // transforming first costs two at F_1; keeping A~ H^(0) across epochs (flag bit 1) removes that one as well.
-    p.agg_first0 = (cfg->flags & 2) != 0 || p.dims[0] <= 2 * p.dims[1];
+    // A layer l >= 1 needs the gradient with respect to its input either way, so it costs two SpMMs in both orders: at
+    // the width F_l when it aggregates first, at F_{l+1} when it transforms first.  It aggregates first when its input is
+    // the narrower side (flag bit 5 keeps the layers l >= 1 on the transform-first order, for comparison).
+    p.agg_first.assign(p.L, 0);
+    p.agg_first[0] = (cfg->flags & 2) != 0 || p.dims[0] <= 2 * p.dims[1];
+    for (int l = 1; l < p.L; ++l) p.agg_first[l] = (cfg->flags & 32) == 0 && p.dims[l] < p.dims[l + 1];
     p.layers.resize(p.L);
     int64_t oi = 0, oe = 0;
     p.dw_partial = 0;
@@ -170,8 +179,8 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_core_spans = take(cur, sizeof(RowSpan) * p.core_spans.size());
     p.o_H.resize(p.L + 1);
     for (int l = 0; l <= p.L; ++l) p.o_H[l] = take(cur, 4 * Np * (size_t)p.ld[l]);
-    int32_t max_spmm_ld = 4;   // the SpMM runs at the widths F_1 .. F_L, and at F_0 when layer 0 aggregates first
-    for (int l = p.agg_first0 ? 0 : 1; l <= p.L; ++l) max_spmm_ld = std::max(max_spmm_ld, p.ld[l]);
+    int32_t max_spmm_ld = 4;   // a layer's SpMMs run at its input width when it aggregates first, else at its output width
+    for (int l = 0; l < p.L; ++l) max_spmm_ld = std::max(max_spmm_ld, p.ld[p.agg_first[l] ? l : l + 1]);
     p.o_spmm_scratch = take(cur, 4 * (size_t)slots * (size_t)max_spmm_ld);
     if (cfg->gemm_mode == 1) p.o_bf16 = take(cur, 2 * Np * (size_t)max_spmm_ld);
     p.o_G1 = take(cur, 4 * Np * (size_t)p.maxld); p.o_G2 = take(cur, 4 * Np * (size_t)p.maxld);
@@ -194,13 +203,14 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         p.o_wt_hi[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi); p.o_wt_lo[l] = take(cur, 4 * (size_t)K * y.fo * y.ldi);
     }
     p.o_counters = take(cur, 4 * (size_t)(1 + 2 * K));
-    if (p.agg_first0) p.o_P = take(cur, 4 * Np * (size_t)p.ld[0]);
+    p.o_P.assign(p.L, 0);
+    for (int l = 0; l < p.L; ++l)
+        if (p.agg_first[l]) p.o_P[l] = take(cur, 4 * Np * (size_t)p.ld[l]);
     p.narrow.assign(p.L, 0);
     int64_t narrow_partial = 0;
     for (int l = 0; l < p.L; ++l) {
         const Layer& y = p.layers[l];
-        const bool agg_first = l == 0 && p.agg_first0;
-        p.narrow[l] = (cfg->flags & 5) == 0 && l > 0 && !agg_first && narrow_supported(y.ldi, y.ldo);
+        p.narrow[l] = (cfg->flags & 5) == 0 && l > 0 && !p.agg_first[l] && narrow_supported(y.ldi, y.ldo);
         if (p.narrow[l]) narrow_partial = std::max(narrow_partial, (int64_t)y.fi * y.ldw + y.ldi);
     }
     if (narrow_partial > 0) {
@@ -215,11 +225,18 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         p.o_nchunk_ptr = take(cur, 4 * (size_t)(K + 1));
         p.o_nw_partial = take(cur, 4 * p.nchunks.size() * (size_t)narrow_partial);
     }
-    if (cfg->zeta_mode == 1) {
+    if (cfg->zeta_mode == 1 && p.pair_alu_ok) {
         p.pair_ptr.assign(K + 1, 0);
         for (int32_t k = 0; k < K; ++k) p.pair_ptr[k + 1] = p.pair_ptr[k] + zeta_pair_tiles(sub_off[k + 1] - sub_off[k]);
         p.o_pair_ptr = take(cur, 8 * (size_t)(K + 1));
         p.o_pair_partial = take(cur, 8 * (size_t)p.pair_ptr[K]);
+    }
+    if (cfg->zeta_mode == 1 && (cfg->flags & (1 | 16)) == 0) {
+        p.gram_ptr.assign(K + 1, 0);
+        for (int32_t k = 0; k < K; ++k) p.gram_ptr[k + 1] = p.gram_ptr[k] + zeta_gram_tiles(sub_off[k + 1] - sub_off[k]);
+        p.o_gram_ptr = take(cur, 8 * (size_t)(K + 1));
+        p.o_gram_partial = take(cur, 8 * (size_t)zeta_gram_partials(kGramMaxCtas, K));
+        p.o_norm2 = take(cur, 4 * Np);
     }
     p.bytes = cur;
     return GAD_OK;
@@ -228,6 +245,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
 }  // namespace
 
 struct gad_ctx {
+    struct alignas(64) TMap { unsigned char bytes[128]; };
     cudaStream_t stream = nullptr;
     char* ws = nullptr;
     Plan p;
@@ -254,8 +272,9 @@ struct gad_ctx {
     struct EpochGraph { cudaGraphExec_t exec = nullptr; int64_t kernels = 0; bool failed = false; } graphs[2];
     int64_t direct_epochs = 0;      // epochs enqueued launch by launch so far (the first one also sets up the kernels)
     bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
+    bool use_gram = false;          // zeta_mode 1 through the Gram-matrix kernel on the tensor cores
+    TMap map_x;                     // H^(0) as 128-row boxes, for that kernel
     int num_sms = 1;
-    struct alignas(64) TMap { unsigned char bytes[128]; };
     std::vector<TMap> maps;         // per layer: forward A, B_hi, B_lo; input-gradient A, B_hi, B_lo
 
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -349,13 +368,12 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
         const Layer& y = p.layers[l];
         Epilogue ep{params, p.pstride, y.b_int, ctx->at<int32_t>(p.o_sub_off), p.K, l < p.L - 1 ? 1 : 0,
                     train ? ctx->cfg.dropout : 0.f, ctx->cfg.seed, ctx->epoch, l};
-        const bool agg_first = l == 0 && p.agg_first0;
-        if (agg_first) {
-            // A~ (X W) = (A~ X) W: aggregate at the input width, finish the layer in the transform's epilogue
-            if (!(ctx->hoist && ctx->P_valid)) {
+        if (p.agg_first[l]) {
+            // A~ (H W) = (A~ H) W: aggregate at the input width, finish the layer in the transform's epilogue
+            if (!(l == 0 && ctx->hoist && ctx->P_valid)) {
                 GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
-                        [&] { return launch_spmm(ctx->A, ctx->H(0), y.ldi, ctx->at<float>(p.o_P), y.ldi, y.fi, nullptr, bf16_of(ctx), ctx->stream); });
-                ctx->P_valid = true;
+                        [&] { return launch_spmm(ctx->A, ctx->H(l), y.ldi, ctx->at<float>(p.o_P[l]), y.ldi, y.fi, nullptr, bf16_of(ctx), ctx->stream); });
+                if (l == 0) ctx->P_valid = true;
             }
             const ActEpi act = make_act(ep, 0);
             if (split_pending) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
@@ -364,7 +382,7 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
                     return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 2, passes, y.fi, y.fo,
                                                ctx->H(l + 1), y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, &act,
                                                ctx->at<int32_t>(p.o_flags) + 1, ctx->num_sms, ctx->stream);
-                return launch_gemm_rows_simt(2, ctx->at<float>(p.o_P), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, ctx->H(l + 1), y.ldo,
+                return launch_gemm_rows_simt(2, ctx->at<float>(p.o_P[l]), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, ctx->H(l + 1), y.ldo,
                                              ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, &act, ctx->stream);
             });
             continue;
@@ -390,6 +408,16 @@ int zeta_pass(gad_ctx* ctx, cudaStream_t s) {
     if (ctx->cfg.zeta_mode == 2 && !ctx->acts_valid) {   // asked for before any pass has run: an inference pass provides the activations
         int rc = forward_pass(ctx, false, ctx->stream);
         if (rc != GAD_OK) return rc;
+    }
+    if (ctx->cfg.zeta_mode == 1 && ctx->use_gram) {
+        const double pairs = 128.0 * 128.0 * (double)p.gram_ptr[p.K];
+        GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 2), 2.0 * pairs * p.dims[0], [&] {
+            return launch_zeta_gram(&ctx->map_x, ctx->H(0), p.ld[0], p.dims[0], p.Np, ctx->at<int32_t>(p.o_deg), ctx->at<int32_t>(p.o_sub_off),
+                                    ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_gram_ptr), p.gram_ptr[p.K], p.K, ctx->cfg.beta,
+                                    ctx->at<float>(p.o_norm2), ctx->at<double>(p.o_gram_partial), ctx->at<double>(p.o_zeta),
+                                    ctx->at<int32_t>(p.o_flags) + 1, std::min(ctx->num_sms, kGramMaxCtas), s);
+        });
+        return GAD_OK;
     }
     if (ctx->cfg.zeta_mode == 1) {
         const double pairs = 64.0 * 64.0 * (double)p.pair_ptr[p.K];
@@ -448,7 +476,7 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
             if (ss != ctx->stream) GAD_CK(cudaEventRecord(ctx->ev_bias, ss));
         }
         bias_done = false;
-        const bool agg_first = l == 0 && p.agg_first0;   // then dW = (A~ X)^T dPre and nothing flows further back
+        const bool agg_first = p.agg_first[l] != 0;   // then dW = (A~ H^(l))^T dPre, and dH^(l) = A~^T (dPre W^T)
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
                     [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, bf16_of(ctx), ctx->stream); });
@@ -478,12 +506,30 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
                 ctx->use_tc ? launch_gemm_tn_tc(&ctx->maps[kMapsPerLayer * l + 6], &ctx->maps[kMapsPerLayer * l + 7],
                                                 ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fi, y.fo, y.ldw, dw_chunks, ndw,
                                                 ctx->at<float>(p.o_dw_partial), ctx->at<int32_t>(p.o_flags) + 1, ctx->stream)
-                            : launch_gemm_tn_simt(agg_first ? ctx->at<float>(p.o_P) : ctx->H(l), y.ldi, y.fi, agg_first ? G1 : G2, y.ldo,
+                            : launch_gemm_tn_simt(agg_first ? ctx->at<float>(p.o_P[l]) : ctx->H(l), y.ldi, y.fi, agg_first ? G1 : G2, y.ldo,
                                                   y.fo, dw_chunks, ndw, ctx->at<float>(p.o_dw_partial), y.ldw, ctx->stream);
             if (e != cudaSuccess) return e;
             return launch_reduce_chunks(ctx->at<float>(p.o_dw_partial), (int64_t)y.fi * y.ldw, dw_chunk_ptr, p.K, grads, p.pstride,
                                         y.w_int, (int64_t)y.fi * y.ldw, ctx->stream);
         });
+        if (l > 0 && agg_first) {
+            // dP = dPre W^T (no mask yet: the ReLU of layer l-1 sits below the aggregation), dH^(l) = A~^T dP, then the mask
+            GAD_RUN("gemm_dh", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
+                if (ctx->use_tc)
+                    return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 3], &ctx->maps[kMapsPerLayer * l + 4], &ctx->maps[kMapsPerLayer * l + 5], 1,
+                                               ctx->cfg.gemm_mode == 0 ? 3 : 1, y.fo, y.fi, G2, y.ldi, ctx->at<RowSpan>(p.o_tiles),
+                                               (int)p.tiles.size(), nullptr, 0, 1.f, nullptr, ctx->at<int32_t>(p.o_flags) + 1,
+                                               ctx->num_sms, ctx->stream);
+                return launch_gemm_rows_simt(1, G1, y.ldo, y.fo, params, p.pstride, y.w_int, y.ldw, y.fi, G2, y.ldi,
+                                             ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr, ctx->stream);
+            });
+            if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));   // the column sums have read dPre
+            GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
+                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G2, y.ldi, G1, y.ldi, y.fi, nullptr, bf16_of(ctx), ctx->stream); });
+            GAD_RUN("relu_mask", l, 12.0 * p.Np * y.fi, 1.0 * p.Np * y.fi,
+                    [&] { return launch_relu_mask(G1, ctx->H(l), y.ldi, p.Np, scale, ctx->stream); });
+            continue;
+        }
         if (l > 0 && ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
         if (l > 0)
             GAD_RUN("gemm_dh", l, 4.0 * p.Np * (2.0 * y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
@@ -520,6 +566,22 @@ uint64_t host_mix64(uint64_t z) {
     z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ULL;
     z = (z ^ (z >> 27)) * 0x94d049bb133111ebULL;
     return z ^ (z >> 31);
+}
+
+// Default initialisation in the caller-visible layout [W_0, b_0, W_1, b_1, ...]: W_l uniform in (-a, a), a = sqrt(6 / (F_l +
+// F_{l+1})) (Glorot), the i-th weight overall from the 53 top bits of mix(seed + G i) (splitmix64 stream); biases zero.
+void default_params(const std::vector<int32_t>& dims, uint64_t seed, float* out) {
+    uint64_t ctr = 0;
+    int64_t o = 0;
+    for (size_t l = 0; l + 1 < dims.size(); ++l) {
+        const int64_t fi = dims[l], fo = dims[l + 1];
+        const double a = std::sqrt(6.0 / (double)(fi + fo));
+        for (int64_t i = 0; i < fi * fo; ++i) {
+            const uint64_t h = host_mix64(seed + 0x9e3779b97f4a7c15ULL * (++ctr));
+            out[o++] = (float)((2.0 * ((h >> 11) * (1.0 / 9007199254740992.0)) - 1.0) * a);
+        }
+        for (int64_t j = 0; j < fo; ++j) out[o++] = 0.f;
+    }
 }
 
 int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col,
@@ -654,7 +716,7 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         (rc = upload(ctx, p.o_tiles, p.tiles)) || (rc = upload(ctx, p.o_chunks, p.chunks)) ||
         (rc = upload(ctx, p.o_chunk_ptr, p.chunk_ptr)) || (rc = upload(ctx, p.o_dw_chunks, p.dw_chunks)) ||
         (rc = upload(ctx, p.o_dw_chunk_ptr, p.dw_chunk_ptr)) || (rc = upload(ctx, p.o_core_spans, p.core_spans)) ||
-        (rc = upload(ctx, p.o_pair_ptr, p.pair_ptr)) || (rc = upload(ctx, p.o_nchunks, p.nchunks)) ||
+        (rc = upload(ctx, p.o_pair_ptr, p.pair_ptr)) || (rc = upload(ctx, p.o_gram_ptr, p.gram_ptr)) || (rc = upload(ctx, p.o_nchunks, p.nchunks)) ||
         (rc = upload(ctx, p.o_nchunk_ptr, p.nchunk_ptr)))
         return rc;
     // features: graph order -> staging -> store-row order with zero pad columns
@@ -662,19 +724,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     GAD_CK(launch_gather_rows(ctx->at<float>(p.o_stage), p.dims[0], ctx->at<int32_t>(p.o_gid), p.Np, ctx->H(0), p.ld[0], ctx->stream));
     // parameters: K identical padded copies
     std::vector<float> ext((size_t)p.P);
-    if (init_params) {
-        std::memcpy(ext.data(), init_params, sizeof(float) * (size_t)p.P);
-    } else {
-        uint64_t ctr = 0;
-        for (const Layer& y : p.layers) {
-            const double a = std::sqrt(6.0 / (y.fi + y.fo));
-            for (int64_t i = 0; i < (int64_t)y.fi * y.fo; ++i) {
-                uint64_t h = host_mix64(cfg->seed + 0x9e3779b97f4a7c15ULL * (++ctr));
-                ext[y.w_ext + i] = (float)((2.0 * ((h >> 11) * (1.0 / 9007199254740992.0)) - 1.0) * a);
-            }
-            for (int j = 0; j < y.fo; ++j) ext[y.b_ext + j] = 0.f;
-        }
-    }
+    if (init_params) std::memcpy(ext.data(), init_params, sizeof(float) * (size_t)p.P);
+    else default_params(p.dims, cfg->seed, ext.data());
     ctx->host_block.assign((size_t)p.pstride, 0.f);
     pack_params(p, ext.data(), ctx->host_block.data());
     for (int32_t k = 0; k < p.K; ++k)
@@ -691,6 +742,14 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         ctx->num_sms = prop.multiProcessorCount;
         ctx->use_tc = (cfg->flags & 1) == 0 && prop.major == 10 && p.Np > 0;
     }
+    if (ctx->cfg.zeta_mode == 1) {
+        ctx->use_gram = ctx->use_tc && !p.gram_ptr.empty();
+        if (ctx->use_gram && !tc_make_map(&ctx->map_x, ctx->H(0), p.dims[0], p.Np, 0, 4ull * p.ld[0], 0, 128))
+            return fail(ctx, GAD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+        if (!ctx->use_gram && !p.pair_alu_ok)
+            return fail(ctx, GAD_ERR_UNSUPPORTED, "zeta_mode 1 without the tensor-core kernel takes subgraphs of at most " +
+                                                      std::to_string(kZetaPairMaxRows) + " rows");
+    }
     if (ctx->use_tc) {
         ctx->maps.resize((size_t)kMapsPerLayer * p.L);
         bool ok = true;
@@ -702,13 +761,13 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
             GAD_CK(cudaMemsetAsync(ctx->ws + p.o_wt_lo[l], 0, 4 * (size_t)p.K * y.fo * y.ldi, ctx->stream));
             gad_ctx::TMap* m = &ctx->maps[(size_t)kMapsPerLayer * l];
             // forward: A = H^(l) [Np x fi], B = W^T copies [K][fo][fi]
-            const bool agg_first = l == 0 && p.agg_first0;   // then the transform and the weight gradient read A~ H^(0), and dW reads dPre (G1)
-            float* Hin = agg_first ? ctx->at<float>(p.o_P) : ctx->H(l);
+            const bool agg_first = p.agg_first[l] != 0;   // then the transform and the weight gradient read A~ H^(l), dW and dH read dPre (G1)
+            float* Hin = agg_first ? ctx->at<float>(p.o_P[l]) : ctx->H(l);
             ok = ok && tc_make_map(&m[0], Hin, y.fi, p.Np, 0, 4ull * y.ldi, 0, 128);
             ok = ok && tc_make_map(&m[1], ctx->at<float>(p.o_wt_hi[l]), y.fi, y.fo, p.K, 4ull * y.ldi, 4ull * y.fo * y.ldi, tc_bn_for(y.fo));
             ok = ok && tc_make_map(&m[2], ctx->at<float>(p.o_wt_lo[l]), y.fi, y.fo, p.K, 4ull * y.ldi, 4ull * y.fo * y.ldi, tc_bn_for(y.fo));
             // input gradient: A = dZ [Np x fo] (in G2), B = W copies [K][fi][fo]
-            ok = ok && tc_make_map(&m[3], ctx->at<float>(p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 128);
+            ok = ok && tc_make_map(&m[3], ctx->at<float>(agg_first ? p.o_G1 : p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 128);
             ok = ok && tc_make_map(&m[4], ctx->at<float>(p.o_w_hi[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
             ok = ok && tc_make_map(&m[5], ctx->at<float>(p.o_w_lo[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
             // weight gradient: 32-row tiles of H^(l) and of dZ (in G2)
@@ -723,6 +782,14 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     GAD_CK(cudaStreamSynchronize(ctx->stream));
     guard.ok = true;
     *out = ctx;
+    return GAD_OK;
+}
+
+int gad_default_params(int32_t L, const int32_t* dims, uint64_t seed, float* out) {
+    if (L < 1 || !dims || !out) return GAD_ERR_ARG;
+    for (int l = 0; l <= L; ++l)
+        if (dims[l] < 1) return GAD_ERR_ARG;
+    default_params(std::vector<int32_t>(dims, dims + L + 1), seed, out);
     return GAD_OK;
 }
 

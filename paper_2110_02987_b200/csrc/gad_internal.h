@@ -205,6 +205,15 @@ cudaError_t launch_zeta_pair(const float* X, int ld, int F, const int32_t* deg, 
 
 // `err_word` (may be null): when a kernel of the epoch has reported a bounded wait that ran out, the gradients are not to
 // be trusted and the three consensus kernels leave the parameters (and `out`) untouched.
+// The same zeta_k with the squared distances from a Gram matrix on the tensor cores (zeta_gram.cu): tiles of 128 x 128 pairs,
+// tile_ptr[k] = first tile of subgraph k, any subgraph size.  norm2: [rows] floats; partial: zeta_gram_partials doubles.
+constexpr int kGramMaxCtas = 256;
+int64_t zeta_gram_tiles(int64_t rows);
+int64_t zeta_gram_partials(int num_ctas, int K);
+cudaError_t launch_zeta_gram(const void* mapX, const float* X, int ld, int F, long long rows, const int32_t* deg, const int32_t* sub_off,
+                             const int64_t* deg_sum, const int64_t* tile_ptr, int64_t ntiles, int K, float beta, float* norm2,
+                             double* partial, double* zeta, int32_t* err, int num_sms, cudaStream_t s);
+
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, const int32_t* err_word, cudaStream_t s);
 // One context's share of a consensus over several contexts: out = sum_k w_k (theta_k - lr grad_k) with w_k = zeta_k / total
@@ -217,6 +226,10 @@ cudaError_t launch_consensus_apply(float* params, int64_t pstride, int64_t len, 
 // reports it in `err` like a transform would (role 99).  For testing the time-out path; returns at once.
 cudaError_t launch_expire_wait(int32_t* err, uint32_t polls, cudaStream_t s);
 cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_f, float* w_f, cudaStream_t s);
+
+// G[r][c] = H[r][c] > 0 ? G[r][c] * scale : 0 over rows x ld values (the ReLU and dropout scale of the layer below, applied
+// to an input gradient that was aggregated after its transform).
+cudaError_t launch_relu_mask(float* G, const float* H, int ld, int64_t rows, float scale, cudaStream_t s);
 
 cudaError_t launch_gather_rows(const float* Xg, int F, const int32_t* gid, int64_t Np, float* H0, int ld,
                                cudaStream_t s);

@@ -83,7 +83,7 @@ gemm_rows_kernel(const float* __restrict__ A, int lda, int Kd, const float* __re
             int n = n0 + tx * TN + j;
             if (n >= ldc) continue;
             float4 v = make_float4(acc[i][j], acc[i][j + 1], acc[i][j + 2], acc[i][j + 3]);
-            if (MODE == 1) {
+            if (MODE == 1 && Hmask) {   // without a mask: plain A W^T
                 float4 h = *reinterpret_cast<const float4*>(Hmask + row * ldh + n);
                 v.x = h.x > 0.f ? v.x * scale : 0.f;
                 v.y = h.y > 0.f ? v.y * scale : 0.f;

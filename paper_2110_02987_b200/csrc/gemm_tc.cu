@@ -20,12 +20,13 @@
 
 #include "epilogue.cuh"
 #include "gad_internal.h"
+#include "tc_common.cuh"
 
 namespace gad {
 
 namespace {
 
-constexpr int BM = 128, BK = 32, STAGES = 3, BN_MAX = 128;
+constexpr int BK = 32, STAGES = 3, BN_MAX = 128;
 constexpr int A_BYTES = BM * BK * 4;                      // 16 KiB
 constexpr int B_BYTES = BN_MAX * BK * 4;                  // 16 KiB
 constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;    // A_hi | A_lo | B_hi | B_lo
@@ -38,101 +39,8 @@ constexpr int SPLIT_WARPS = 8;                            // warps that split th
 constexpr int EPI_WARP0 = 2 + SPLIT_WARPS;                // first epilogue warp (a multiple of 2, see the lane quarters)
 constexpr int ROWS_THREADS = 32 * (EPI_WARP0 + EPI_WARPS);
 constexpr int SMEM_BYTES_ROWS = SMEM_BYTES + EPI_BYTES;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int ACC_COLS = 256;                             // widest output tile of the rows kernel (one MMA: N <= 256)
 constexpr int TMEM_COLS = 2 * ACC_COLS;                   // two accumulators: all 512 columns of the SM's tensor memory
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.b32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the wait ran out or another role of this CTA has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, int32_t* err, int code,
-                                          uint32_t limit = WAIT_LIMIT) {
-    for (uint32_t i = 0; i < limit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-    }
-    *abort_flag = 1u;
-    atomicExch(err, code);
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
-                 : "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major tile written by TMA with the 128-byte swizzle: rows of 128 bytes,
-// groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2 (128B swizzle).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
-           ((uint64_t)2 << 61);
-}
-// Instruction descriptor: fp32 accumulator, TF32 A and B, both K-major, N and M of the MMA.
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-__device__ __forceinline__ void mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n"
-        "}\n" ::"r"(tmem_d),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, "
-        "%25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
-          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-
-// Nearest value with a 10-bit mantissa (ties away from zero), i.e. exactly representable in TF32.
-// Infinities, NaNs and the few finite values that would round up to infinity pass through unchanged.
-__device__ __forceinline__ float tf32_round(float x) {
-    const uint32_t b = __float_as_uint(x);
-    const uint32_t r = (b + 0x1000u) & 0xFFFFE000u;
-    // keep NaNs (whose payload the addition could carry into the sign bit) and anything that would become infinite
-    return __uint_as_float((b & 0x7FFFFFFFu) < 0x7F7FF000u ? r : b);
-}
 
 struct TcArgs {
     const RowSpan* tiles;
@@ -314,7 +222,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int n = n0 + c0 + sub_c;
                 // the eight mask loads of this lane go out together, ahead of the accumulator read and of any store
                 float4 hm[8];
-                if (a.mode == 1) {
+                const bool masked = a.mode == 1 && a.Hmask != nullptr;   // mode 1 without a mask: plain A W^T
+                if (masked) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const int r = q * 32 + 4 * i + sub_r;
@@ -336,7 +245,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int i = 0; i < 8; ++i) {
                     const float* src = tr + (4 * i + sub_r) * 33 + sub_c;
                     o[i] = make_float4(src[0], src[1], src[2], src[3]);
-                    if (a.mode == 1) {
+                    if (masked) {
                         o[i].x = hm[i].x > 0.f ? o[i].x * a.scale : 0.f;
                         o[i].y = hm[i].y > 0.f ? o[i].y * a.scale : 0.f;
                         o[i].z = hm[i].z > 0.f ? o[i].z * a.scale : 0.f;

@@ -599,6 +599,24 @@ cudaError_t launch_weights(const double* zeta, int K, int weighted, float* zeta_
     return cudaGetLastError();
 }
 
+__global__ void __launch_bounds__(256) relu_mask_kernel(float4* __restrict__ G, const float4* __restrict__ H, long long n4, float scale) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 g = G[i];
+    const float4 h = H[i];
+    g.x = h.x > 0.f ? g.x * scale : 0.f; g.y = h.y > 0.f ? g.y * scale : 0.f;
+    g.z = h.z > 0.f ? g.z * scale : 0.f; g.w = h.w > 0.f ? g.w * scale : 0.f;
+    G[i] = g;
+}
+cudaError_t launch_relu_mask(float* G, const float* H, int ld, int64_t rows, float scale, cudaStream_t s) {
+    const long long n4 = (long long)rows * (ld / 4);
+    if (n4 > 0) {
+        relu_mask_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(reinterpret_cast<float4*>(G), reinterpret_cast<const float4*>(H), n4, scale);
+        ++g_kernel_launches;
+    }
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------------------------------------
 // Gathers between graph-node order and store-row order.
 // ---------------------------------------------------------------------------------------------

@@ -85,13 +85,8 @@ __device__ __forceinline__ Item load_item(const int4* __restrict__ items, int id
 // A group fetches a batch of entries at a time (the next batch is requested before this one is used), hands them
 // round with shuffles and has all their operand rows in flight before the multiply-adds; a slot past the end of the
 // item re-reads the item's own operand row with weight 0.  A last batch at most half full takes a half batch.
-#ifndef GAD_SPMM_NBATCH
-#define GAD_SPMM_NBATCH 8
-#endif
-#ifndef GAD_SPMM_NMINB
-#define GAD_SPMM_NMINB 3
-#endif
-constexpr int kNarrowBatch = GAD_SPMM_NBATCH;
+constexpr int kNarrowBatch = 8;      // entries a lane group has in flight
+constexpr int kNarrowMinBlocks = 3;  // resident CTAs of 256 threads asked of the compiler
 template <int GROUP> struct NarrowCfg { static constexpr int EPL = kNarrowBatch / GROUP > 0 ? kNarrowBatch / GROUP : 1; };
 
 template <int GROUP, int NB, bool BF>
@@ -115,7 +110,7 @@ __device__ __forceinline__ void narrow_batch(float4& acc, const uint2 (&mine)[Na
 }
 
 template <int GROUP, bool EPI, bool BF>
-__global__ void __launch_bounds__(256, GAD_SPMM_NMINB)
+__global__ void __launch_bounds__(256, kNarrowMinBlocks)
 spmm_items_narrow_kernel(const uint2* __restrict__ ecv, const int4* __restrict__ items, int nitems, const float* __restrict__ Z, int ldz,
                          float* __restrict__ out, int ldo, float* __restrict__ scratch, int F4, EpiDev ep) {
     constexpr int NB = kNarrowBatch, EPL = NarrowCfg<GROUP>::EPL;   // entries per batch, entries a lane fetches per batch
@@ -266,22 +261,10 @@ __device__ __forceinline__ void gather_tail(float4 (&acc)[NV], const uint2* st, 
 
 // Operand rows in flight per lane and resident warps asked of the compiler: short items make the chain
 // item -> entries -> operand rows the cost, and more resident warps hide it better than more loads per warp.
-#ifndef GAD_SPMM_UU1
-#define GAD_SPMM_UU1 2
-#endif
-#ifndef GAD_SPMM_MINB1
-#define GAD_SPMM_MINB1 16
-#endif
-#ifndef GAD_SPMM_UU2
-#define GAD_SPMM_UU2 2
-#endif
-#ifndef GAD_SPMM_MINB2
-#define GAD_SPMM_MINB2 10
-#endif
 constexpr int kItemWarps = 4;
 template <int NV> struct ItemCfg {
-    static constexpr int UU = NV == 1 ? GAD_SPMM_UU1 : (NV == 2 ? GAD_SPMM_UU2 : (NV <= 4 ? 2 : 1));
-    static constexpr int MINB = NV == 1 ? GAD_SPMM_MINB1 : (NV == 2 ? GAD_SPMM_MINB2 : (NV <= 4 ? 6 : 4));   // CTAs of 4 warps per SM
+    static constexpr int UU = NV <= 4 ? 2 : 1;
+    static constexpr int MINB = NV == 1 ? 16 : (NV == 2 ? 10 : (NV <= 4 ? 6 : 4));   // CTAs of 4 warps per SM
 };
 
 template <int NV, bool EPI, bool OFF32, bool BF, bool PAIR>

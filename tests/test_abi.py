@@ -111,3 +111,24 @@ def test_augment_arguments_are_checked_on_the_host():
     rp = rowptr.copy(); rp[5], rp[6] = rp[6] + 1, rp[5]
     assert ws(graph=b.gad_csr(int(n), int(rowptr[-1]), b._ptr(rp, C.c_int64), b._ptr(col, C.c_int32), None))[0] == -3
     assert ws(graph=b.gad_csr(int(n), int(rowptr[-1]) + 1, b._ptr(rowptr, C.c_int64), b._ptr(col, C.c_int32), None))[0] == -1
+
+
+def test_default_initialisation_is_seeded_glorot_uniform():
+    """gad_default_params (what gad_create uses when no parameters are passed in): every weight inside the Glorot range
+    of its layer, spread over it like a uniform variable, biases zero, a pure function of the seed."""
+    dims = (40, 64, 7)
+    a = pkg.default_params(dims, seed=3)
+    assert np.array_equal(a, pkg.default_params(dims, seed=3))
+    assert not np.array_equal(a, pkg.default_params(dims, seed=4))
+    o = 0
+    for fi, fo in zip(dims[:-1], dims[1:]):
+        W, b = a[o:o + fi * fo], a[o + fi * fo:o + fi * fo + fo]
+        o += fi * fo + fo
+        lim = np.sqrt(6.0 / (fi + fo))
+        assert np.all(np.abs(W) < lim) and np.all(b == 0.0)
+        assert abs(W.mean()) < 4 * lim / np.sqrt(3 * W.size)            # mean 0, variance lim^2 / 3
+        assert abs(W.var() - lim * lim / 3) < 0.1 * lim * lim / 3
+        assert np.unique(W).size > 0.99 * W.size
+    assert o == a.size
+    with pytest.raises(GadError):
+        pkg.default_params((4, 0, 2))

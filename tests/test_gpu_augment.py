@@ -68,3 +68,39 @@ def test_augmented_subgraphs_train_like_the_oracle():
         for _ in range(3):
             assert np.max(np.abs(g.train_epoch() - ref.train_epoch())) <= 1e-4
         assert rel_err(g.get_params(0), ref.get_params(0)) <= 1e-4
+
+
+def test_leading_walks_that_do_not_suffice():
+    """The device hands the host only the best-ranked walks (here 1024 of about 9000).  3000 core nodes that all touch one
+    outside hub and one private outside node each: every top-ranked walk ends on the hub, so the leading stretch yields a
+    single replication node and the ranking of all walks has to follow - with the same lists as the oracle."""
+    m = 3000
+    hub = m
+    src = np.concatenate([np.arange(m), np.full(m, hub), np.arange(m), m + 1 + np.arange(m)])
+    dst = np.concatenate([np.full(m, hub), np.arange(m), m + 1 + np.arange(m), np.arange(m)])
+    ring = np.arange(m)
+    src = np.concatenate([src, ring, (ring + 1) % m]); dst = np.concatenate([dst, (ring + 1) % m, ring])
+    n = 2 * m + 1
+    order = np.lexsort((dst, src))
+    src, dst = src[order], dst[order]
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(np.bincount(src, minlength=n), out=rowptr[1:])
+    cores = [np.arange(m, dtype=np.int32), np.arange(m, n, dtype=np.int32)]
+    got, info = _both(n, rowptr, dst.astype(np.int32), cores, 1, alpha=0.05, seed=9)
+    assert len(got[0]) > 100 and info[0]["n"] > 1024
+
+
+def test_a_second_call_reuses_the_graph_on_the_device():
+    """Augmenter keeps its workspace: from the second call on the graph is not uploaded again (graph_resident), whatever
+    the partition, the seed or the walk length of that call; a call that needs a larger workspace uploads it afresh."""
+    import paper_2110_02987_b200 as pkg
+    from oracle import augment_oracle as aug
+    w = make_workload("c2", scale=0.03)
+    a = pkg.Augmenter(w.n, w.rowptr, w.col)
+    for K, steps, seed, cap in ((4, 2, 0, 4), (4, 3, 5, 4), (6, 2, 1, 2), (2, 2, 2, 8)):
+        cores = bfs_partition(w.rowptr, w.col, K)
+        got, walks = a.run(cores, steps, alpha=0.03, seed=seed, cap=cap)
+        want, info = aug.augment(w.n, w.rowptr, w.col, cores, steps, alpha=0.03, seed=seed, cap=cap)
+        assert walks.tolist() == [it["n"] for it in info]
+        for x, y in zip(got, want):
+            assert np.array_equal(x, y)

@@ -206,12 +206,15 @@ def test_importance_weights_and_consensus(tiny):
         assert np.allclose(g.subgraph_weights()[1], 0.25)
 
 
+@pytest.mark.parametrize("flags", [0, 16])
 @pytest.mark.parametrize("seed,n,K,F", [(0, 70, 3, 6), (1, 700, 2, 37), (2, 3000, 3, 64), (3, 1500, 1, 130)])
-def test_pairwise_importance_weights(seed, n, K, F):
-    """zeta_mode 1: the printed formula taken literally, sum_{i<j} p_i p_j / (|x_i - x_j| + beta), over tiles of
-    64 x 64 pairs with ragged last tiles, against the oracle's double loop; then an epoch whose consensus uses them."""
+def test_pairwise_importance_weights(seed, n, K, F, flags):
+    """zeta_mode 1: the printed formula taken literally, sum_{i<j} p_i p_j / (|x_i - x_j| + beta), against the oracle's
+    double loop; then an epoch whose consensus uses them.  flags 0: squared distances from a Gram matrix on the tensor
+    cores, tiles of 128 x 128 pairs; flags 16: from the differences on the FP32 ALUs, tiles of 64 x 64.  Ragged last
+    tiles, subgraphs of less than one tile, feature widths that are not multiples of the MMA's K."""
     case = small_random_case(seed, n=n, K=K, p=min(0.15, 8.0 / n))
-    g, ref, st = make_pair(case, (F, 8, 3), seed, lr=0.1, zeta_mode=1)
+    g, ref, st = make_pair(case, (F, 8, 3), seed, lr=0.1, zeta_mode=1, flags=flags)
     with g:
         zg, wg = g.subgraph_weights()
         zr, wr = ref.subgraph_weights()
@@ -220,12 +223,14 @@ def test_pairwise_importance_weights(seed, n, K, F):
         check_epoch(g, ref)
 
 
-def test_pairwise_importance_of_identical_points_is_the_closed_form():
-    """All features equal: every distance is 0 and zeta = S / beta with S = (1 - sum p^2) / 2."""
+@pytest.mark.parametrize("flags", [0, 16])
+def test_pairwise_importance_of_identical_points_is_the_closed_form(flags):
+    """All features equal: every distance is 0 and zeta = S / beta with S = (1 - sum p^2) / 2.  (For the Gram-matrix
+    kernel this is the worst case of its cancellation: every pair is recomputed from the differences.)"""
     case = small_random_case(5, n=300, K=2, p=0.05)
     n = case[0]
     X = np.ones((n, 12), dtype=np.float32) * 0.75
-    g, ref, st = make_pair(case, (12, 5, 3), 5, X=X, zeta_mode=1, beta=0.5)
+    g, ref, st = make_pair(case, (12, 5, 3), 5, X=X, zeta_mode=1, beta=0.5, flags=flags)
     with g:
         zg, _ = g.subgraph_weights()
     for k in range(st.K):
@@ -674,3 +679,73 @@ def test_set_inputs_rejects_labels_outside_the_classes(tiny):
             g.set_inputs(w.X, bad)
         assert e.value.code == -2
         assert np.all(np.isfinite(g.train_epoch()))      # nothing was enqueued; the old labels are still in place
+
+
+def test_pairwise_importance_of_near_duplicates_and_offset_features():
+    """The Gram form |x|^2 + |y|^2 - 2 x.y cancels for rows that are close compared with their norms.  Features with a
+    large common offset (every pair is close in that sense) and a block of near-duplicate rows must still give the
+    oracle's zeta: such pairs take the difference form."""
+    case = small_random_case(41, n=600, K=2, p=0.02)
+    n = case[0]
+    rng = np.random.default_rng(41)
+    X = (rng.standard_normal((n, 20)) + 40.0).astype(np.float32)
+    X[100:200] = X[100] + 1e-3 * rng.standard_normal((100, 20)).astype(np.float32)
+    g, ref, st = make_pair(case, (20, 5, 3), 41, X=X, zeta_mode=1)
+    with g:
+        zg, wg = g.subgraph_weights()
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(zg - zr)) <= 2e-6 * np.max(zr)
+        assert np.max(np.abs(wg - wr)) <= 2e-6
+
+
+def test_pairwise_importance_of_a_large_subgraph():
+    """One subgraph of 36 000 rows (more than the 32 768 the FP32-ALU kernel takes; 282 x 282 / 2 tiles, the last ones
+    ragged) and one of 5 000, against the oracle's pair loop (6.6e8 pairs); twice, for run-to-run equality."""
+    rng = np.random.default_rng(43)
+    n, F = 41000, 24
+    src = rng.integers(0, n, size=4 * n)
+    dst = rng.integers(0, n, size=4 * n)
+    keep = src != dst
+    src, dst = np.concatenate([src[keep], dst[keep]]), np.concatenate([dst[keep], src[keep]])
+    order = np.lexsort((dst, src))
+    src, dst = src[order], dst[order]
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(np.bincount(src, minlength=n), out=rowptr[1:])
+    core = [np.arange(0, 36000, dtype=np.int32), np.arange(36000, n, dtype=np.int32)]
+    halo = [np.empty(0, np.int32), np.empty(0, np.int32)]
+    X = rng.standard_normal((n, F)).astype(np.float32)
+    X[:, :3] *= 4.0
+    g, ref, st = make_pair((n, rowptr, dst.astype(np.int32), None, core, halo), (F, 6, 3), 43, X=X, zeta_mode=1)
+    with g:
+        zg, wg = g.subgraph_weights()
+        zg2, _ = g.subgraph_weights()
+        assert np.array_equal(zg, zg2)
+        zr, wr = ref.subgraph_weights()
+        assert np.max(np.abs(zg - zr)) <= 2e-6 * np.max(zr)
+        assert np.max(np.abs(wg - wr)) <= 2e-6
+    with pytest.raises(pkg().GadError) as e:           # the FP32-ALU form keeps its limit
+        make_pair((n, rowptr, dst.astype(np.int32), None, core, halo), (F, 6, 3), 43, X=X, zeta_mode=1, flags=16)
+    assert e.value.code == -9
+
+
+@pytest.mark.parametrize("flags", [0, 1, 32])
+@pytest.mark.parametrize("dims,dropout", [((16, 8, 256, 4), 0.0), ((12, 40, 9, 64, 5), 0.3), ((20, 6, 30, 140, 3), 0.0)])
+def test_layers_beyond_the_first_choose_the_order_of_aggregation_and_transform(flags, dims, dropout):
+    """A layer l >= 1 whose input is narrower than its output aggregates first, sigma((A~ H^(l)) W + b): forward SpMM at
+    the input width, dW = (A~ H^(l))^T dPre, dH^(l) = A~^T (dPre W^T) followed by the ReLU mask of the layer below.  On
+    the tensor cores, on the FP32 ALUs (flags bit 0), and with the choice switched off (flags bit 5): all against the
+    oracle, which always computes A~ (H W)."""
+    case = small_random_case(71, n=700, K=3, p=0.012, directed=(flags == 1))
+    g, ref, st = make_pair(case, dims, 71, lr=0.05, dropout=dropout, flags=flags)
+    with g:
+        for _ in range(2):
+            lg = g.train_epoch()
+            lr, _ = oracle_step(g, ref)
+            assert np.max(np.abs(lg - lr)) <= 1e-4
+        L = len(dims) - 1
+        for l in range(1, L + 1):
+            assert rel_err(g.get_activation(l), ref.activation(l)) <= TOL, "activation %d" % l
+        for k in range(g.K):
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
+        assert rel_err(g.forward(), ref.forward_global(case[0])) <= TOL
