@@ -115,9 +115,13 @@ __global__ void walk_score_kernel(const int64_t* __restrict__ rowptr, const int3
 // digit by digit (13 bits at a time, from the top), each pass a histogram of the next digit over the keys that share the
 // digits fixed so far; the host reads the 8192 counts and fixes the digit.  A last pass gathers the keys >= that one.
 constexpr int kDigitBits = 13, kDigits = 1 << kDigitBits;
-__global__ void __launch_bounds__(256) key_hist_kernel(const unsigned long long* __restrict__ key, int64_t n, unsigned long long prefix_mask,
-                                                       unsigned long long prefix, int shift, unsigned* __restrict__ hist) {
+// sel = {digits fixed so far, their mask, rank still to find among the keys that share them}: kept on the device, so the passes
+// follow each other without the host in between.
+struct KeySelect { unsigned long long prefix, mask; long long remaining; };
+__global__ void __launch_bounds__(256) key_hist_kernel(const unsigned long long* __restrict__ key, int64_t n, const KeySelect* __restrict__ sel,
+                                                       int shift, unsigned* __restrict__ hist) {
     __shared__ unsigned h[kDigits];
+    const unsigned long long prefix = sel->prefix, prefix_mask = sel->mask;
     for (int i = threadIdx.x; i < kDigits; i += blockDim.x) h[i] = 0u;
     __syncthreads();
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x) {
@@ -128,10 +132,50 @@ __global__ void __launch_bounds__(256) key_hist_kernel(const unsigned long long*
     for (int i = threadIdx.x; i < kDigits; i += blockDim.x)
         if (h[i]) atomicAdd(hist + i, h[i]);
 }
-__global__ void __launch_bounds__(256) key_gather_kernel(const unsigned long long* __restrict__ key, int64_t n, unsigned long long least,
+// One CTA of 1024 threads: the digit whose bin holds the key of rank `remaining` (counted from the largest digit down),
+// fixed in *sel; the histogram is cleared for the next pass.
+__global__ void __launch_bounds__(1024) key_digit_kernel(unsigned* __restrict__ hist, KeySelect* __restrict__ sel, int shift) {
+    __shared__ long long part[1024];
+    __shared__ int chosen;
+    __shared__ long long chosen_rem;
+    constexpr int PER = kDigits / 1024;
+    const int t = threadIdx.x;                 // thread t owns the bins kDigits-1 - PER t .. kDigits - PER (t + 1), largest first
+    unsigned mine[PER];
+    long long s = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { mine[i] = hist[kDigits - 1 - (PER * t + i)]; s += mine[i]; }
+    part[t] = s;
+    if (t == 0) { chosen = 0; chosen_rem = 1; }
+    __syncthreads();
+    // keys in the bins of the threads before this one (inclusive scan by doubling, then made exclusive)
+    for (int o = 1; o < 1024; o <<= 1) {
+        const long long add = t >= o ? part[t - o] : 0;
+        __syncthreads();
+        part[t] += add;
+        __syncthreads();
+    }
+    const long long before = part[t] - s, remaining = sel->remaining;
+    if (before < remaining && remaining <= before + s) {   // exactly one thread: the bins are disjoint and ordered
+        long long r = remaining - before;
+        int i = 0;
+        for (; i < PER - 1 && (long long)mine[i] < r; ++i) r -= mine[i];
+        chosen = kDigits - 1 - (PER * t + i);
+        chosen_rem = r;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < PER; ++i) hist[PER * t + i] = 0u;
+    if (t == 0) {
+        sel->prefix |= (unsigned long long)chosen << shift;
+        sel->mask |= (unsigned long long)(kDigits - 1) << shift;
+        sel->remaining = chosen_rem;
+    }
+}
+__global__ void __launch_bounds__(256) key_gather_kernel(const unsigned long long* __restrict__ key, int64_t n, const KeySelect* __restrict__ sel,
                                                          unsigned long long* __restrict__ out, unsigned long long* __restrict__ n_out, int64_t cap) {
     const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
+    const unsigned long long least = sel->prefix;
     const unsigned long long k = key[j];
     if (k >= least) {
         const unsigned long long at = atomicAdd(n_out, 1ull);   // the host sorts what it gets: the order here is free
@@ -193,7 +237,7 @@ int plan_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int
     size_t cur = 0;
     p.o_rowptr = take(cur, 8 * (size_t)(g->n + 1)); p.o_col = take(cur, 4 * (size_t)g->nnz);
     p.o_inside = take(cur, (size_t)g->n); p.o_core = take(cur, 4 * (size_t)p.max_core); p.o_flag = take(cur, (size_t)p.max_core);
-    p.o_B = take(cur, 4 * (size_t)p.max_core); p.o_count = take(cur, 4 * (size_t)g->n); p.o_stats = take(cur, 40);
+    p.o_B = take(cur, 4 * (size_t)p.max_core); p.o_count = take(cur, 4 * (size_t)g->n); p.o_stats = take(cur, 64);
     p.o_score = take(cur, 8 * (size_t)p.max_walks);
     // n(g_i) <= alpha (1 + d) |v_i| <= 2 alpha |v_i|
     p.max_top = leading_walks(p.max_walks, (int64_t)std::floor(cfg->alpha * 2.0 * (double)p.max_core));
@@ -266,7 +310,6 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
     std::vector<int32_t> B, seq((size_t)steps + 1);
     std::vector<int64_t> score, order;
     std::vector<unsigned long long> top;
-    std::vector<unsigned> hist((size_t)kDigits);
     std::vector<uint8_t> taken((size_t)n, 0);
     auto grid = [](int64_t work) { return (unsigned)((work + 255) / 256); };
     int64_t out = 0;
@@ -287,11 +330,22 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
             AUG_CK(cudaStreamSynchronize(s));
             B.clear();
             const int64_t inner_directed = (int64_t)inner_dev;
-            for (int64_t t = 0; t < ncore; ++t) {
-                inside[(size_t)core[t]] = 1;
-                if (flag[(size_t)t]) B.push_back(core[t]);
+            // boundary nodes in ascending node id: sorted, or, when the core set is a fair share of the graph, read off a
+            // byte map over the node ids (one pass over n bytes instead of a sort)
+            if (n <= 16 * ncore) {
+                for (int64_t t = 0; t < ncore; ++t) {
+                    inside[(size_t)core[t]] = 1;
+                    if (flag[(size_t)t]) taken[(size_t)core[t]] = 1;
+                }
+                for (int64_t v = 0; v < n; ++v)
+                    if (taken[(size_t)v]) { B.push_back((int32_t)v); taken[(size_t)v] = 0; }
+            } else {
+                for (int64_t t = 0; t < ncore; ++t) {
+                    inside[(size_t)core[t]] = 1;
+                    if (flag[(size_t)t]) B.push_back(core[t]);
+                }
+                std::sort(B.begin(), B.end());
             }
-            std::sort(B.begin(), B.end());
             const int64_t nB = (int64_t)B.size();
             if (nB > 0) {
                 int64_t n0 = 0;
@@ -358,21 +412,17 @@ int gad_augment(const gad_csr* g, int32_t K, const int64_t* core_ptr, const int3
                     // the `sorted`-th largest key, digit by digit from the top; then the keys at least that large
                     int top_bit = 32;
                     while (top_bit < 63 && (((int64_t)(steps + 1) * nwalks) >> (top_bit - 32)) > 0) ++top_bit;
-                    unsigned long long prefix = 0, prefix_mask = 0;
-                    int64_t remaining = sorted;
+                    KeySelect* d_sel = reinterpret_cast<KeySelect*>(d_stats + 5);
+                    const KeySelect sel0{0ull, 0ull, (long long)sorted};
+                    AUG_CK(cudaMemcpyAsync(d_sel, &sel0, sizeof sel0, cudaMemcpyHostToDevice, s));
+                    AUG_CK(cudaMemsetAsync(d_hist, 0, 4 * (size_t)kDigits, s));
                     for (int d = (top_bit + kDigitBits - 1) / kDigitBits - 1; d >= 0; --d) {
                         const int shift = d * kDigitBits;
-                        AUG_CK(cudaMemsetAsync(d_hist, 0, 4 * (size_t)kDigits, s));
-                        key_hist_kernel<<<148 * 2, 256, 0, s>>>(d_key, nwalks, prefix_mask, prefix, shift, d_hist); ++g_kernel_launches;
-                        AUG_CK(cudaMemcpyAsync(hist.data(), d_hist, 4 * (size_t)kDigits, cudaMemcpyDeviceToHost, s));
-                        AUG_CK(cudaStreamSynchronize(s));
-                        int b = kDigits - 1;
-                        for (; b > 0 && (int64_t)hist[(size_t)b] < remaining; --b) remaining -= hist[(size_t)b];
-                        prefix |= (unsigned long long)b << shift;
-                        prefix_mask |= (unsigned long long)(kDigits - 1) << shift;
+                        key_hist_kernel<<<148 * 2, 256, 0, s>>>(d_key, nwalks, d_sel, shift, d_hist); ++g_kernel_launches;
+                        key_digit_kernel<<<1, 1024, 0, s>>>(d_hist, d_sel, shift); ++g_kernel_launches;
                     }
                     AUG_CK(cudaMemsetAsync(d_stats + 4, 0, 8, s));
-                    key_gather_kernel<<<grid(nwalks), 256, 0, s>>>(d_key, nwalks, prefix, d_top, d_stats + 4, p.max_top); ++g_kernel_launches;
+                    key_gather_kernel<<<grid(nwalks), 256, 0, s>>>(d_key, nwalks, d_sel, d_top, d_stats + 4, p.max_top); ++g_kernel_launches;
                     unsigned long long got = 0;
                     top.resize((size_t)sorted);
                     AUG_CK(cudaMemcpyAsync(&got, d_stats + 4, 8, cudaMemcpyDeviceToHost, s));

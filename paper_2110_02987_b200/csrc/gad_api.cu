@@ -62,7 +62,7 @@ struct Plan {
     std::vector<int64_t> pair_ptr;    // [K+1] tiles of pairs per subgraph (zeta_mode 1 on the FP32 ALUs), else empty
     size_t o_pair_ptr = 0, o_pair_partial = 0;
     std::vector<int64_t> gram_ptr;    // [K+1] 128 x 128 tiles of pairs per subgraph (zeta_mode 1 on the tensor cores)
-    size_t o_gram_ptr = 0, o_gram_partial = 0, o_norm2 = 0;
+    size_t o_gram_ptr = 0, o_gram_partial = 0, o_norm2 = 0, o_xhi = 0, o_xlo = 0;
     bool pair_alu_ok = false;         // every subgraph is small enough for the FP32-ALU pairwise kernel
     int64_t dw_partial = 0;           // floats per chunk
     std::vector<uint8_t> agg_first;   // [L] the layer aggregates before it transforms: sigma((A~ H^(l)) W + b)
@@ -237,6 +237,7 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
         p.o_gram_ptr = take(cur, 8 * (size_t)(K + 1));
         p.o_gram_partial = take(cur, 8 * (size_t)zeta_gram_partials(kGramMaxCtas, K));
         p.o_norm2 = take(cur, 4 * Np);
+        p.o_xhi = take(cur, 4 * Np * (size_t)p.ld[0]); p.o_xlo = take(cur, 4 * Np * (size_t)p.ld[0]);
     }
     p.bytes = cur;
     return GAD_OK;
@@ -273,7 +274,7 @@ struct gad_ctx {
     int64_t direct_epochs = 0;      // epochs enqueued launch by launch so far (the first one also sets up the kernels)
     bool use_tc = false;            // tensor-core transforms (tcgen05) instead of the SIMT ones
     bool use_gram = false;          // zeta_mode 1 through the Gram-matrix kernel on the tensor cores
-    TMap map_x;                     // H^(0) as 128-row boxes, for that kernel
+    TMap map_xhi, map_xlo;          // the TF32 split of H^(0) as 128-row boxes, for that kernel
     int num_sms = 1;
     std::vector<TMap> maps;         // per layer: forward A, B_hi, B_lo; input-gradient A, B_hi, B_lo
 
@@ -412,8 +413,9 @@ int zeta_pass(gad_ctx* ctx, cudaStream_t s) {
     if (ctx->cfg.zeta_mode == 1 && ctx->use_gram) {
         const double pairs = 128.0 * 128.0 * (double)p.gram_ptr[p.K];
         GAD_RUN("zeta", -1, 4.0 * p.Np * (p.dims[0] + 2), 2.0 * pairs * p.dims[0], [&] {
-            return launch_zeta_gram(&ctx->map_x, ctx->H(0), p.ld[0], p.dims[0], p.Np, ctx->at<int32_t>(p.o_deg), ctx->at<int32_t>(p.o_sub_off),
-                                    ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_gram_ptr), p.gram_ptr[p.K], p.K, ctx->cfg.beta,
+            return launch_zeta_gram(&ctx->map_xhi, &ctx->map_xlo, ctx->H(0), p.ld[0], p.dims[0], p.Np, ctx->at<int32_t>(p.o_deg),
+                                    ctx->at<int32_t>(p.o_sub_off), ctx->at<int64_t>(p.o_deg_sum), ctx->at<int64_t>(p.o_gram_ptr),
+                                    p.gram_ptr[p.K], p.K, ctx->cfg.beta, ctx->at<float>(p.o_xhi), ctx->at<float>(p.o_xlo),
                                     ctx->at<float>(p.o_norm2), ctx->at<double>(p.o_gram_partial), ctx->at<double>(p.o_zeta),
                                     ctx->at<int32_t>(p.o_flags) + 1, std::min(ctx->num_sms, kGramMaxCtas), s);
         });
@@ -744,7 +746,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     }
     if (ctx->cfg.zeta_mode == 1) {
         ctx->use_gram = ctx->use_tc && !p.gram_ptr.empty();
-        if (ctx->use_gram && !tc_make_map(&ctx->map_x, ctx->H(0), p.dims[0], p.Np, 0, 4ull * p.ld[0], 0, 128))
+        if (ctx->use_gram && !(tc_make_map(&ctx->map_xhi, ctx->at<float>(p.o_xhi), p.dims[0], p.Np, 0, 4ull * p.ld[0], 0, 128) &&
+                               tc_make_map(&ctx->map_xlo, ctx->at<float>(p.o_xlo), p.dims[0], p.Np, 0, 4ull * p.ld[0], 0, 128)))
             return fail(ctx, GAD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
         if (!ctx->use_gram && !p.pair_alu_ok)
             return fail(ctx, GAD_ERR_UNSUPPORTED, "zeta_mode 1 without the tensor-core kernel takes subgraphs of at most " +

@@ -206,13 +206,14 @@ cudaError_t launch_zeta_pair(const float* X, int ld, int F, const int32_t* deg, 
 // `err_word` (may be null): when a kernel of the epoch has reported a bounded wait that ran out, the gradients are not to
 // be trusted and the three consensus kernels leave the parameters (and `out`) untouched.
 // The same zeta_k with the squared distances from a Gram matrix on the tensor cores (zeta_gram.cu): tiles of 128 x 128 pairs,
-// tile_ptr[k] = first tile of subgraph k, any subgraph size.  norm2: [rows] floats; partial: zeta_gram_partials doubles.
+// tile_ptr[k] = first tile of subgraph k, any subgraph size.  Xhi, Xlo: [rows x ld] floats each (TF32 split of X, written
+// by the call; mapHi / mapLo are their 128-row-box descriptors); norm2: [rows] floats; partial: zeta_gram_partials doubles.
 constexpr int kGramMaxCtas = 256;
 int64_t zeta_gram_tiles(int64_t rows);
 int64_t zeta_gram_partials(int num_ctas, int K);
-cudaError_t launch_zeta_gram(const void* mapX, const float* X, int ld, int F, long long rows, const int32_t* deg, const int32_t* sub_off,
-                             const int64_t* deg_sum, const int64_t* tile_ptr, int64_t ntiles, int K, float beta, float* norm2,
-                             double* partial, double* zeta, int32_t* err, int num_sms, cudaStream_t s);
+cudaError_t launch_zeta_gram(const void* mapHi, const void* mapLo, const float* X, int ld, int F, long long rows, const int32_t* deg,
+                             const int32_t* sub_off, const int64_t* deg_sum, const int64_t* tile_ptr, int64_t ntiles, int K, float beta,
+                             float* Xhi, float* Xlo, float* norm2, double* partial, double* zeta, int32_t* err, int num_sms, cudaStream_t s);
 
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, const int32_t* err_word, cudaStream_t s);
