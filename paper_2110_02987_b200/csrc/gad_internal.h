@@ -48,14 +48,14 @@ int store_sizes(const gad_csr* g, const gad_partition* part, int64_t* Np, int64_
 
 // Work lists of the SpMM launch (host side).  A row of at most `part_entries` entries is one item; a longer row is
 // cut into parts of `part_entries` entries, each an item with a scratch slot of its own, and gets an entry
-// fin = {row, first scratch slot, slots, subgraph of the row}.  The part length starts at kMinPart and doubles (up to kMaxPart)
-// until the cut rows need at most one scratch slot per two store rows; a row that would still need more than
-// kMaxSlotsPerRow parts gets longer parts of its own.
+// fin = {row, first scratch slot, slots, subgraph of the row}.  The part length starts at kMinPart, or at a quarter of the
+// entries an average resident warp gets if that is more, and doubles (up to kMaxPart) until the cut rows need at most one
+// scratch slot per two store rows; a row that would still need more than kMaxSlotsPerRow parts gets longer parts of its own.
 // items = {row, low 32 bits of the first entry's position in the store, (high bits << 16) | entries, scratch slot
 // or -1 for an uncut row}, subgraph by subgraph and inside a subgraph binned by floor(log2(entries)), longest bin
 // first, ascending row inside a bin.  `perm` (uncut rows in that order) and `parts` are the intermediate lists the
 // items are built from.
-constexpr int64_t kMinPart = 64, kMaxPart = 1024, kMaxSlotsPerRow = 32;
+constexpr int64_t kMinPart = 64, kMaxPart = 8192, kMaxSlotsPerRow = 32;
 struct RowWork {
     std::vector<int32_t> perm;
     std::vector<int4> parts, fin, items;
