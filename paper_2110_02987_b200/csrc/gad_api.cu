@@ -774,8 +774,8 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
             ok = ok && tc_make_map(&m[4], ctx->at<float>(p.o_w_hi[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
             ok = ok && tc_make_map(&m[5], ctx->at<float>(p.o_w_lo[l]), y.fo, y.fi, p.K, 4ull * y.ldw, 4ull * y.fi * y.ldw, tc_bn_for(y.fi));
             // weight gradient: 32-row tiles of H^(l) and of dZ (in G2)
-            ok = ok && tc_make_map(&m[6], Hin, y.fi, p.Np, 0, 4ull * y.ldi, 0, 32, true);
-            ok = ok && tc_make_map(&m[7], ctx->at<float>(agg_first ? p.o_G1 : p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, 32, true);
+            ok = ok && tc_make_map(&m[6], Hin, y.fi, p.Np, 0, 4ull * y.ldi, 0, tc_tn_rows(), true);
+            ok = ok && tc_make_map(&m[7], ctx->at<float>(agg_first ? p.o_G1 : p.o_G2), y.fo, p.Np, 0, 4ull * y.ldo, 0, tc_tn_rows(), true);
         }
         if (!ok) return fail(ctx, GAD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     }

@@ -146,6 +146,7 @@ cudaError_t launch_gemm_rows_simt(int mode, const float* A, int lda, int Kd, con
 // tc_make_map (A: [rows x Kd]; B, B_lo: [K][N][Kd] copies written by launch_split_weights); passes = 3 gives fp32
 // accuracy by operand splitting, passes = 1 plain TF32 operands.  err receives a role code if a bounded wait runs out.
 int tc_bn_for(int n_cols);
+int tc_tn_rows();   // rows of the row-box descriptors the weight-gradient kernel reads (mapH / mapZ of launch_gemm_tn_tc)
 bool tc_make_map(void* out_map, const void* base, uint64_t inner, uint64_t rows, uint64_t outer, uint64_t row_stride_bytes,
                  uint64_t outer_stride_bytes, uint32_t box_rows, bool mn_major = false);
 cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w_int, int fi, int fo, int ldw, int ldkt, int K,
@@ -154,7 +155,7 @@ cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* 
                                 float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
                                 const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s);
 
-// Tensor-core version of launch_gemm_tn_simt; mapH / mapZ are 32-row-box descriptors of H^(l) and dZ.
+// Tensor-core version of launch_gemm_tn_simt; mapH / mapZ are row-box descriptors (tc_tn_rows rows) of H^(l) and dZ.
 cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,
                               int nchunks, float* partial, int32_t* err, cudaStream_t s);
 

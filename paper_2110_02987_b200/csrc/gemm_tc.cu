@@ -187,10 +187,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const int i = tt + 32 * SPLIT_WARPS * j;
                         const float4 v = hi[i];
                         float4 h, l;
-                        h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
-                        h.y = tf32_round(v.y); l.y = tf32_round(v.y - h.y);
-                        h.z = tf32_round(v.z); l.z = tf32_round(v.z - h.z);
-                        h.w = tf32_round(v.w); l.w = tf32_round(v.w - h.w);
+                        h.x = tf32_hi(v.x); l.x = tf32_round(v.x - h.x);
+                        h.y = tf32_hi(v.y); l.y = tf32_round(v.y - h.y);
+                        h.z = tf32_hi(v.z); l.z = tf32_round(v.z - h.z);
+                        h.w = tf32_hi(v.w); l.w = tf32_round(v.w - h.w);
                         hi[i] = h;
                         lo[i] = l;
                     }
@@ -293,7 +293,7 @@ __global__ void split_weights_kernel(const float* __restrict__ params, long long
     if (idx >= (long long)fi * ldw) return;
     const int i = (int)(idx / ldw), j = (int)(idx % ldw);
     const float w = params[(long long)k * pstride + w_int + idx];
-    const float h = tf32_round(w), l = tf32_round(w - h);
+    const float h = tf32_hi(w), l = tf32_round(w - h);
     w_hi[(long long)k * fi * ldw + idx] = h;
     w_lo[(long long)k * fi * ldw + idx] = l;
     if (j < fo) {
@@ -319,10 +319,16 @@ struct TnArgs {
     int32_t* err;
 };
 
+// Rows of the reduction per ring stage of the weight-gradient kernel (a multiple of 8, the K of one MMA).  With 32 rows the
+// ring holds two stages at 256 output columns; 16 rows (four stages) measured the same on the 2.5 M-row workload (2.37 vs
+// 2.49 ms at 256 x 256, but 1.41 vs 1.26 ms at 256 x 47) and slower on the small one: the stage count is not what limits it.
+constexpr int TBK = 32;
+constexpr int TN_BLOCK_BYTES = TBK * 128;                 // one block: TBK rows x 32 values
+constexpr int TN_A_BYTES = 4 * TN_BLOCK_BYTES;            // 128 output rows = 4 blocks
 // MN-major TF32 tile: layout type 1 (128-byte swizzle of 32-byte units, repeating every 4 rows = 512 bytes), blocks of
-// 32 values 4096 bytes apart (leading byte offset), groups of 4 rows 512 bytes apart (stride byte offset).
+// 32 values TN_BLOCK_BYTES apart (leading byte offset), groups of 4 rows 512 bytes apart (stride byte offset).
 __device__ __forceinline__ uint64_t smem_desc_mn(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(4096 >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) | ((uint64_t)1 << 46) |
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(TN_BLOCK_BYTES >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) | ((uint64_t)1 << 46) |
            ((uint64_t)1 << 61);
 }
 
@@ -334,10 +340,10 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
     uint8_t* sm = smem_raw + pad;
     const uint32_t sm_addr = raw_addr + pad;
-    // a stage holds the H tile and its low half (16 KiB each) and the dZ tile of BN columns with its low half
+    // a stage holds the H tile and its low half and the dZ tile of BN columns with its low half, TBK rows each
     const int nb_blocks = (a.BN + 31) / 32;                    // 32-value blocks of the B tile
-    const uint32_t b_bytes = (uint32_t)nb_blocks * 4096u;
-    const uint32_t stage_bytes = 2u * A_BYTES + 2u * b_bytes;
+    const uint32_t b_bytes = (uint32_t)nb_blocks * TN_BLOCK_BYTES;
+    const uint32_t stage_bytes = 2u * TN_A_BYTES + 2u * b_bytes;
     const int nst = min(MAX_STAGES, (int)(RING_BYTES / stage_bytes));
     const uint32_t bars = sm_addr + RING_BYTES;
     auto full = [&](int s) { return bars + 8u * s; };
@@ -350,7 +356,7 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), NSPLIT); mbar_init(empty(s), 1); }
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(xfull(s), NSPLIT / 32); mbar_init(empty(s), 1); }   // one arrival per splitting warp
         mbar_init(tfull, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -368,8 +374,8 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
     const RowSpan c = a.chunks[blockIdx.x / tiles_per_chunk];
     const int tile = blockIdx.x % tiles_per_chunk;
     const int m0 = (tile / a.ntn) * BM, n0 = (tile % a.ntn) * a.BN;
-    const int nkb = (c.nrows + BK - 1) / BK;
-    const uint32_t tx_bytes = (uint32_t)(4 + nb_blocks) * 4096u;
+    const int nkb = (c.nrows + TBK - 1) / TBK;
+    const uint32_t tx_bytes = (uint32_t)(4 + nb_blocks) * TN_BLOCK_BYTES;
     bool ok = true;
 
     if (warp == 0 && lane == 0) {
@@ -379,9 +385,9 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             if (!(ok = mbar_wait(empty(stage), phase ^ 1u, abort_flag, a.err, 11))) break;
             mbar_expect_tx(full(stage), tx_bytes);
             const uint32_t base = sm_addr + stage * stage_bytes;
-            const int r = c.row0 + kb * BK;
-            for (int j = 0; j < 4; ++j) tma_load_2d(base + j * 4096, &tmH, m0 + 32 * j, r, full(stage));
-            for (int j = 0; j < nb_blocks; ++j) tma_load_2d(base + 2 * A_BYTES + j * 4096, &tmZ, n0 + 32 * j, r, full(stage));
+            const int r = c.row0 + kb * TBK;
+            for (int j = 0; j < 4; ++j) tma_load_2d(base + j * TN_BLOCK_BYTES, &tmH, m0 + 32 * j, r, full(stage));
+            for (int j = 0; j < nb_blocks; ++j) tma_load_2d(base + 2 * TN_A_BYTES + j * TN_BLOCK_BYTES, &tmZ, n0 + 32 * j, r, full(stage));
             if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
     } else if (warp == 1 && lane == 0) {
@@ -393,14 +399,14 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             if (!(ok = mbar_wait(xfull(stage), phase, abort_flag, a.err, 14))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t base = sm_addr + stage * stage_bytes;
-            const int nks = min(BK / 8, (c.nrows - kb * BK + 7) / 8);
-            const uint64_t a_hi = smem_desc_mn(base), a_lo = smem_desc_mn(base + A_BYTES);
-            const uint64_t b_hi = smem_desc_mn(base + 2 * A_BYTES), b_lo = smem_desc_mn(base + 2 * A_BYTES + b_bytes);
+            const int nks = min(TBK / 8, (c.nrows - kb * TBK + 7) / 8);
+            const uint64_t a_hi = smem_desc_mn(base), a_lo = smem_desc_mn(base + TN_A_BYTES);
+            const uint64_t b_hi = smem_desc_mn(base + 2 * TN_A_BYTES), b_lo = smem_desc_mn(base + 2 * TN_A_BYTES + b_bytes);
             // the next group of 8 rows is 1024 bytes = 64 descriptor units further on; a full block is unrolled so that
             // the issuing thread spends few instructions between two MMAs
-            if (nks == BK / 8 && a.passes > 1) {
+            if (nks == TBK / 8 && a.passes > 1) {
 #pragma unroll
-                for (int ks = 0; ks < BK / 8; ++ks) {
+                for (int ks = 0; ks < TBK / 8; ++ks) {
                     mma_tf32(tmem_base, a_hi + 64 * ks, b_hi + 64 * ks, idesc, ks == 0 ? (kb != 0 ? 1u : 0u) : 1u);
                     mma_tf32(tmem_base, a_hi + 64 * ks, b_lo + 64 * ks, idesc, 1u);
                     mma_tf32(tmem_base, a_lo + 64 * ks, b_hi + 64 * ks, idesc, 1u);
@@ -424,31 +430,34 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
         const int tt = threadIdx.x - 64;
         int stage = 0;
         uint32_t phase = 0;
-        const int nf4 = (4 + nb_blocks) * 256;                // float4 values of the stage's A and B tiles
+        constexpr int BF4 = TN_BLOCK_BYTES / 16;              // float4 values of one block
+        const int nf4 = (4 + nb_blocks) * BF4;                // float4 values of the stage's A and B tiles
         for (int kb = 0; kb < nkb; ++kb) {
-            if (!(ok = mbar_wait(full(stage), phase, abort_flag, a.err, 15))) break;
-            const int rows_valid = min(BK, c.nrows - kb * BK);
-            if (a.passes > 1 || rows_valid < BK) {
+            // (the vote keeps the warp together: lanes may see a time-out or an abort at different polls)
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(full(stage), phase, abort_flag, a.err, 15)))) break;
+            const int rows_valid = min(TBK, c.nrows - kb * TBK);
+            if (a.passes > 1 || rows_valid < TBK) {
                 uint8_t* sb = sm + stage * stage_bytes;
                 for (int i = tt; i < nf4; i += NSPLIT) {
-                    const int blk = i >> 8, in = i & 255;                         // block of 32 values, float4 inside it
+                    const int blk = i / BF4, in = i % BF4;                        // block of 32 values, float4 inside it
                     const int row = in >> 3;                                      // 8 float4 per 128-byte row
-                    const int byte_off = (blk < 4 ? blk * 4096 : 2 * A_BYTES + (blk - 4) * 4096) + in * 16;
+                    const int byte_off = (blk < 4 ? blk * TN_BLOCK_BYTES : 2 * TN_A_BYTES + (blk - 4) * TN_BLOCK_BYTES) + in * 16;
                     float4* hi = reinterpret_cast<float4*>(sb + byte_off);
-                    float4* lo = reinterpret_cast<float4*>(sb + byte_off + (blk < 4 ? (uint32_t)A_BYTES : b_bytes));
+                    float4* lo = reinterpret_cast<float4*>(sb + byte_off + (blk < 4 ? (uint32_t)TN_A_BYTES : b_bytes));
                     float4 v = *hi;
                     if (row >= rows_valid) v = make_float4(0.f, 0.f, 0.f, 0.f);
                     float4 h, l;
-                    h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
-                    h.y = tf32_round(v.y); l.y = tf32_round(v.y - h.y);
-                    h.z = tf32_round(v.z); l.z = tf32_round(v.z - h.z);
-                    h.w = tf32_round(v.w); l.w = tf32_round(v.w - h.w);
+                    h.x = tf32_hi(v.x); l.x = tf32_round(v.x - h.x);
+                    h.y = tf32_hi(v.y); l.y = tf32_round(v.y - h.y);
+                    h.z = tf32_hi(v.z); l.z = tf32_round(v.z - h.z);
+                    h.w = tf32_hi(v.w); l.w = tf32_round(v.w - h.w);
                     *hi = a.passes > 1 ? h : v;
                     if (a.passes > 1) *lo = l;
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
-            mbar_arrive(xfull(stage));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(xfull(stage));
             if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
     }
@@ -515,6 +524,7 @@ EncodeTiledFn encode_fn() {
 
 // Output columns per tile: one MMA covers up to 256, and an M = 128, K = 8 TF32 MMA costs about the same for any N, so
 // the widest tile that the ring still holds twice is the cheapest.
+int tc_tn_rows() { return TBK; }
 int tc_bn_for(int n_cols) { return n_cols <= 16 ? 16 : n_cols <= 32 ? 32 : n_cols <= 64 ? 64 : n_cols <= 128 ? 128 : 256; }
 
 // fp32 tensor [outer (z)] x [rows (y)] x [inner (x)], box = 32 floats x box_rows x 1, zero fill outside.  K-major

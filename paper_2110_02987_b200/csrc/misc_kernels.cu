@@ -504,6 +504,34 @@ __device__ __forceinline__ void consensus_weights(const double* __restrict__ zet
     __syncthreads();
 }
 
+// sum_k w_k (theta_k - lr grad_k) for the four parameters at float4 index i, k ascending.  The copies are read eight at a time,
+// all sixteen loads of a batch issued before the first is used: with many copies of a small model (K = 64 copies of a
+// 256-256 layer are 50 MB spread over 65 CTAs) the kernel is a chain of dependent loads otherwise.
+__device__ __forceinline__ float4 weighted_sum(const float* __restrict__ params, const float* __restrict__ grads, long long pstride,
+                                               long long i, int K, float lr, int with_sgd, const float* w_sm) {
+    constexpr int B = 8;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k0 = 0; k0 < K; k0 += B) {
+        float4 p[B], g[B];
+#pragma unroll
+        for (int t = 0; t < B; ++t) {
+            const int k = min(k0 + t, K - 1);   // past the end: the last copy again, with weight 0 below
+            p[t] = reinterpret_cast<const float4*>(params + (long long)k * pstride)[i];
+            g[t] = with_sgd ? reinterpret_cast<const float4*>(grads + (long long)k * pstride)[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int t = 0; t < B; ++t) {
+            if (k0 + t < K) {
+                const float w = w_sm[k0 + t];
+                float4 q = p[t];
+                if (with_sgd) { q.x = fmaf(-lr, g[t].x, q.x); q.y = fmaf(-lr, g[t].y, q.y); q.z = fmaf(-lr, g[t].z, q.z); q.w = fmaf(-lr, g[t].w, q.w); }
+                acc.x = fmaf(w, q.x, acc.x); acc.y = fmaf(w, q.y, acc.y); acc.z = fmaf(w, q.z, acc.z); acc.w = fmaf(w, q.w, acc.w);
+            }
+        }
+    }
+    return acc;
+}
+
 // theta_k <- theta_k - lr * grad_k (each replica's own step, update equation of Section 3.3), then
 // theta_k <- sum_j w_j theta_j for every k (weighted global consensus, Section 3.4.2).  One float4 per thread.
 __global__ void __launch_bounds__(256) sgd_consensus_kernel(float* __restrict__ params, const float* __restrict__ grads,
@@ -515,23 +543,15 @@ __global__ void __launch_bounds__(256) sgd_consensus_kernel(float* __restrict__ 
     consensus_weights(zeta, K, weighted, w_sm);
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= len4) return;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k = 0; k < K; ++k) {
-        float4 p = reinterpret_cast<const float4*>(params + (long long)k * pstride)[i];
-        if (with_sgd) {
-            float4 g = reinterpret_cast<const float4*>(grads + (long long)k * pstride)[i];
-            p.x = fmaf(-lr, g.x, p.x); p.y = fmaf(-lr, g.y, p.y); p.z = fmaf(-lr, g.z, p.z); p.w = fmaf(-lr, g.w, p.w);
-        }
-        const float w = w_sm[k];
-        acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y); acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
-    }
+    const float4 acc = weighted_sum(params, grads, pstride, i, K, lr, with_sgd, w_sm);
     for (int k = 0; k < K; ++k) reinterpret_cast<float4*>(params + (long long)k * pstride)[i] = acc;
 }
 cudaError_t launch_sgd_consensus(float* params, const float* grads, int64_t pstride, int64_t len, int K, float lr,
                                  const double* zeta, int weighted, int with_sgd, const int32_t* err_word, cudaStream_t s) {
     const long long len4 = len / 4;
     if (len4 > 0) {
-        sgd_consensus_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
+        const int threads = len4 >= 148 * 256 * 4 ? 256 : 64;   // a small model is spread over more CTAs
+        sgd_consensus_kernel<<<(unsigned)((len4 + threads - 1) / threads), threads, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
                                                                                                    zeta, weighted, with_sgd, err_word); ++g_kernel_launches; }
     return cudaGetLastError();
 }
@@ -550,16 +570,7 @@ __global__ void __launch_bounds__(256) consensus_partial_kernel(const float* __r
     __syncthreads();
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= len4) return;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k = 0; k < K; ++k) {
-        float4 p = reinterpret_cast<const float4*>(params + (long long)k * pstride)[i];
-        if (with_sgd) {
-            float4 g = reinterpret_cast<const float4*>(grads + (long long)k * pstride)[i];
-            p.x = fmaf(-lr, g.x, p.x); p.y = fmaf(-lr, g.y, p.y); p.z = fmaf(-lr, g.z, p.z); p.w = fmaf(-lr, g.w, p.w);
-        }
-        const float w = w_sm[k];
-        acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y); acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
-    }
+    const float4 acc = weighted_sum(params, grads, pstride, i, K, lr, with_sgd, w_sm);
     reinterpret_cast<float4*>(out)[i] = acc;
 }
 __global__ void __launch_bounds__(256) consensus_apply_kernel(float* __restrict__ params, long long pstride, long long len4, int K,
@@ -573,7 +584,8 @@ cudaError_t launch_consensus_partial(const float* params, const float* grads, in
                                      const double* zeta, int weighted, int with_sgd, double total, float* out, const int32_t* err_word, cudaStream_t s) {
     const long long len4 = len / 4;
     if (len4 > 0) {
-        consensus_partial_kernel<<<(unsigned)((len4 + 255) / 256), 256, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
+        const int threads = len4 >= 148 * 256 * 4 ? 256 : 64;
+        consensus_partial_kernel<<<(unsigned)((len4 + threads - 1) / threads), threads, (size_t)K * sizeof(float), s>>>(params, grads, pstride, len4, K, lr,
                                                                                                        zeta, weighted, with_sgd, total, out, err_word);
         ++g_kernel_launches;
     }

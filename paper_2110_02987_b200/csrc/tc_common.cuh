@@ -95,13 +95,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "memory");
 }
 
-// Nearest value with a 10-bit mantissa (ties away from zero), i.e. exactly representable in TF32.
-// Infinities, NaNs and the few finite values that would round up to infinity pass through unchanged.
+// Nearest value with a 10-bit mantissa (ties away from zero), i.e. exactly representable in TF32: one conversion
+// instruction.  tf32_round is for values that cannot overflow (the lo parts, weights); tf32_hi also keeps a finite value
+// finite (the few values within 2^-11 of the largest float would round up to infinity: they are clamped to the largest
+// TF32 value, and x - hi then carries the rest).  NaN and infinity stay non-finite through hi or lo.
 __device__ __forceinline__ float tf32_round(float x) {
-    const uint32_t b = __float_as_uint(x);
-    const uint32_t r = (b + 0x1000u) & 0xFFFFE000u;
-    // keep NaNs (whose payload the addition could carry into the sign bit) and anything that would become infinite
-    return __uint_as_float((b & 0x7FFFFFFFu) < 0x7F7FF000u ? r : b);
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+__device__ __forceinline__ float tf32_hi(float x) {
+    return copysignf(fminf(fabsf(tf32_round(x)), __uint_as_float(0x7F7FE000u)), x);
 }
 
 }  // namespace

@@ -312,10 +312,10 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict
         const float4 v = __ldg(x + f4);
         s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s); s = fmaf(v.z, v.z, s); s = fmaf(v.w, v.w, s);
         float4 h, l;
-        h.x = tf32_round(v.x); l.x = tf32_round(v.x - h.x);
-        h.y = tf32_round(v.y); l.y = tf32_round(v.y - h.y);
-        h.z = tf32_round(v.z); l.z = tf32_round(v.z - h.z);
-        h.w = tf32_round(v.w); l.w = tf32_round(v.w - h.w);
+        h.x = tf32_hi(v.x); l.x = tf32_round(v.x - h.x);
+        h.y = tf32_hi(v.y); l.y = tf32_round(v.y - h.y);
+        h.z = tf32_hi(v.z); l.z = tf32_round(v.z - h.z);
+        h.w = tf32_hi(v.w); l.w = tf32_round(v.w - h.w);
         xh[f4] = h;
         xl[f4] = l;
     }
