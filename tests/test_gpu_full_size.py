@@ -24,9 +24,9 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-4
 
 
-@functools.lru_cache(maxsize=1)
+@functools.lru_cache(maxsize=2)
 def workload(name):
-    """The last workload built stays in memory: the tests of one configuration follow each other."""
+    """The two workloads built last stay in memory (a few GB): the tests of c4 and c3k8 alternate."""
     if name.startswith("sweep"):
         _, deg, F, K = name.split("_")
         return make_workload("sweep", mean_deg=float(deg[1:]), F=int(F[1:]), K=int(K[1:]))
