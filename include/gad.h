@@ -237,6 +237,12 @@ int gad_set_inputs(gad_ctx* ctx, const float* X, const int32_t* labels);
 int gad_read_loss_async(gad_ctx* ctx, float* loss_out);
 int gad_synchronize(gad_ctx* ctx);
 
+/* Self-check of the device store (no counterpart in the paper; it stands in for a memory checker): one kernel tests every
+ * index the aggregation kernels form - rows, entry ranges, scratch slots of the work lists, and every stored column against
+ * the row range of its own subgraph (the store is block-diagonal) - for the store and, if there is one, its transposed copy.
+ * *violations receives the count; returns GAD_ERR_RANGE if it is not zero.  Waits for the stream. */
+int gad_check_store(gad_ctx* ctx, int64_t* violations);
+
 /* For testing the time-out path without hanging anything (no counterpart in the paper): enqueues a one-thread kernel
  * that waits, with the same bounded wait the tensor-core transforms use and a limit of `polls` polls (1 .. 65536), on
  * a barrier that nothing ever arrives at.  The wait runs out, the kernel raises the context's error word and returns;

@@ -27,7 +27,7 @@ SYMBOLS = (
     "gad_profile_reset", "gad_profile_count", "gad_profile_read", "gad_subgraph_weights_static", "gad_launch_count",
     "gad_last_error", "gad_destroy", "gad_train_epoch_local", "gad_consensus_floats", "gad_consensus_partial",
     "gad_consensus_apply", "gad_export_params", "gad_get_train_counts", "gad_augment_workspace_bytes", "gad_augment",
-    "gad_augment_last_error", "gad_debug_expire_wait", "gad_default_params",
+    "gad_augment_last_error", "gad_debug_expire_wait", "gad_default_params", "gad_check_store",
 )
 
 
@@ -335,6 +335,13 @@ class Gad:
     @epoch.setter
     def epoch(self, e):
         self._ck(self._L.gad_set_epoch(self._h, C.c_int64(e)))
+
+    def check_store(self):
+        """gad_check_store: every index of the device store and its work lists tested against its range; returns the
+        number of violations (0) or raises."""
+        v = C.c_int64(0)
+        self._ck(self._L.gad_check_store(self._h, C.byref(v)))
+        return int(v.value)
 
     def debug_expire_wait(self, polls=1000):
         """gad_debug_expire_wait: makes one bounded device-side wait run out (for testing the time-out path)."""

@@ -1111,6 +1111,25 @@ int gad_synchronize(gad_ctx* ctx) {
     return GAD_OK;
 }
 
+int gad_check_store(gad_ctx* ctx, int64_t* violations) {
+    if (!ctx || !violations) return GAD_ERR_ARG;
+    const Plan& p = ctx->p;
+    // two 64-bit words of the loss-partial buffer serve as the counters (nothing of an epoch is in flight after the wait below)
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    unsigned long long* bad = ctx->at<unsigned long long>(p.o_loss_partial);
+    const unsigned long long init[2] = {0ull, ~0ull};
+    GAD_CK(cudaMemcpyAsync(bad, init, 16, cudaMemcpyHostToDevice, ctx->stream));
+    GAD_CK(launch_check_store(ctx->A, p.nnz, p.slots, ctx->at<int32_t>(p.o_sub_off), p.K, bad, ctx->stream));
+    if (!ctx->symmetric) GAD_CK(launch_check_store(ctx->At, p.nnz, p.slots, ctx->at<int32_t>(p.o_sub_off), p.K, bad, ctx->stream));
+    unsigned long long out[2] = {0, 0};
+    GAD_CK(cudaMemcpyAsync(out, bad, 16, cudaMemcpyDeviceToHost, ctx->stream));
+    GAD_CK(cudaStreamSynchronize(ctx->stream));
+    *violations = (int64_t)out[0];
+    if (out[0]) return fail(ctx, GAD_ERR_RANGE, "store self-check: " + std::to_string(out[0]) + " index violations, first at work-list position " +
+                                                    std::to_string(out[1] - 1));
+    return GAD_OK;
+}
+
 int gad_debug_expire_wait(gad_ctx* ctx, uint32_t polls) {
     if (!ctx || polls < 1 || polls > 65536) return GAD_ERR_ARG;
     GAD_CK(launch_expire_wait(ctx->at<int32_t>(ctx->p.o_flags) + 1, polls, ctx->stream));

@@ -136,6 +136,11 @@ inline ActEpi make_act(const Epilogue& e, int col0) {
 cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F,
                         const Epilogue* epi, void* bf16_scratch, cudaStream_t s);
 
+// Tests every index of a device store and its work lists against its range (see check_store_kernel); bad[0] += violations,
+// bad[1] = min(bad[1], first offending work-list position + 1).
+cudaError_t launch_check_store(const SparseDev& A, long long nnz, long long slots, const int32_t* sub_off, int K, unsigned long long* bad,
+                               cudaStream_t s);
+
 // mode 0: C = A * W_k (W row-major [Kd x N], ld ldw); mode 1: C = (A * W_k^T) masked by Hmask > 0, scaled
 // (W row-major [N x Kd]); mode 2: C = sigma(A * W_k + b_k) with dropout as `act` says.  Tiles never cross a subgraph.
 cudaError_t launch_gemm_rows_simt(int mode, const float* A, int lda, int Kd, const float* params, int64_t pstride,

@@ -372,6 +372,50 @@ static cudaError_t dispatch(const SparseDev& A, const float* Z, int ldz, float* 
     return cudaSuccess;
 }
 
+// Self-check of a device store before any kernel trusts it: every index the aggregation kernels will form is tested
+// against its range - an item's row, its entry range inside the store, its scratch slot, every column inside the row's own
+// subgraph (the store is block-diagonal), and the slot runs of the cut rows.  bad[0] counts violations, bad[1] keeps the
+// smallest offending item / cut-row index + 1.  Stands in for a memory checker on the store and its work lists.
+__global__ void __launch_bounds__(256) check_store_kernel(const uint2* __restrict__ ecv, long long nnz, const int4* __restrict__ items, int nitems,
+                                                          const int4* __restrict__ fin, int nfin, long long slots, long long nrows,
+                                                          const int32_t* __restrict__ sub_off, int K, unsigned long long* __restrict__ bad) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long mine = 0;
+    if (t < nitems) {
+        const int4 it = items[t];
+        const long long pos = ((long long)((uint32_t)it.z >> 16) << 32) | (long long)(uint32_t)it.y;
+        const int len = (int)((uint32_t)it.z & 0xFFFFu);
+        const bool head_ok = it.x >= 0 && it.x < nrows && pos >= 0 && pos + len <= nnz && (it.w == -1 || (it.w >= 0 && it.w < slots));
+        if (!head_ok) ++mine;
+        else {
+            const int k = find_sub(sub_off, K, it.x);
+            for (int e = 0; e < len; ++e) {
+                const uint32_t c = ecv[pos + e].x;
+                if ((long long)c < sub_off[k] || (long long)c >= sub_off[k + 1]) ++mine;
+            }
+        }
+    } else if (t < (long long)nitems + nfin) {
+        const int4 f = fin[t - nitems];
+        if (!(f.x >= 0 && f.x < nrows && f.y >= 0 && f.z >= 1 && (long long)f.y + f.z <= slots && f.w >= 0 && f.w < K &&
+              f.x >= sub_off[f.w] && f.x < sub_off[f.w + 1]))
+            ++mine;
+    }
+    if (mine) {
+        atomicAdd(bad, mine);
+        atomicMin(bad + 1, (unsigned long long)t + 1ull);
+    }
+}
+
+cudaError_t launch_check_store(const SparseDev& A, long long nnz, long long slots, const int32_t* sub_off, int K, unsigned long long* bad,
+                               cudaStream_t s) {
+    const long long work = (long long)A.nitems + A.nfin;
+    if (work > 0) {
+        check_store_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(A.ecv, nnz, A.items, A.nitems, A.fin, A.nfin, slots, A.nrows, sub_off, K, bad);
+        ++g_kernel_launches;
+    }
+    return cudaGetLastError();
+}
+
 // fp32 -> bfloat16 (round to nearest even; NaN stays NaN), four values per thread.
 __global__ void __launch_bounds__(256) to_bf16_kernel(const float4* __restrict__ in, uint2* __restrict__ out, long long n4) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;

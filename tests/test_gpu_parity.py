@@ -47,6 +47,7 @@ def make_pair(case, dims, seed=0, X=None, **kw):
 
 
 def check_store(g, st):
+    assert g.check_store() == 0          # the library's own index check of the device store and its work lists
     s = g.get_store()
     assert np.array_equal(s["rowptr"], st.rowptr)
     assert np.array_equal(s["col"], st.col)
