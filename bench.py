@@ -32,6 +32,9 @@ UNIT = "epochs/s"
 # capture summarised under profiles/; keyed by (workload, profile entry).  A kernel changed since its capture
 # has no entry (reported as null).
 NCU_TRAFFIC = {
+    # spmm_items_kernel<2,1,...> (14.21 GB read + 2.60 GB written) + spmm_finish_kernel (2 MB), profiles/spmm_c4_dram.md
+    ("c4", "spmm_fwd_l1"): 16.80e9,
+    ("c4", "spmm_bwd_l1"): 17.01e9,
     # spmm_items_kernel (76.8 MB read + 33.6 MB written) + spmm_finish_kernel (14.9 MB read), profiles/spmm_items_c2.md
     ("c2", "spmm_fwd_l0"): 125.3e6,
 }
@@ -166,7 +169,7 @@ def oracle_sample(w, theta, seconds_per_step):
         sub.core, sub.halo = [core0[:m]], [np.empty(0, dtype=np.int32)]
         return orc.from_workload(sub, theta)
 
-    m0 = int(min(len(core0), 2000))
+    m0 = int(min(len(core0), 8000))
     pilot = prefix_model(m0)
     pilot.train_epoch()                      # page everything in
     t0 = time.perf_counter()
@@ -175,7 +178,8 @@ def oracle_sample(w, theta, seconds_per_step):
     pilot.close()
     if per_row * rows_all <= seconds_per_step:
         return orc.from_workload(w, theta), 1.0, "whole epochs of the workload"
-    m = int(min(len(core0), max(m0, seconds_per_step / per_row)))
+    # a longer prefix has more entries per row and leaves the caches: allow for twice the pilot's time per row
+    m = int(min(len(core0), max(m0, seconds_per_step / (2.0 * per_row))))
     frac = m / float(rows_all)
     return prefix_model(m), frac, ("the first %d core rows of subgraph 0 of %d as a block of their own (%.4f of the %d store rows) "
                                    "per step, sized from a %d-row pilot; epochs/s = that fraction / time per step"
@@ -184,7 +188,7 @@ def oracle_sample(w, theta, seconds_per_step):
 
 def run_reference(args, rank):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only): every step a bounded sample of the workload,
-    sized so that warm-up and timed steps together take about two minutes."""
+    sized so that warm-up and timed steps together take one to two minutes."""
     if rank != 0:
         return
     from gad_synth import make_workload, glorot_params
@@ -194,7 +198,7 @@ def run_reference(args, rank):
     theta = glorot_params(w.dims, np.random.default_rng(0))
     cores = orc.threads()
     total_steps = args.steps + args.warmup
-    m, frac, sample = oracle_sample(w, theta, 120.0 / max(total_steps, 1))
+    m, frac, sample = oracle_sample(w, theta, 90.0 / max(total_steps, 1))
     for _ in range(args.warmup):
         m.train_epoch()
     t0 = time.perf_counter()
