@@ -27,6 +27,17 @@ __device__ __forceinline__ bool dropout_keep(uint64_t row_key, int col, uint32_t
     return (uint32_t)(h >> 40) >= thr24;
 }
 
+// fp32 -> bfloat16 bits (round to nearest even; NaN stays a quiet NaN).
+__device__ __forceinline__ uint32_t bf16_bits(float x) {
+    const uint32_t b = __float_as_uint(x);
+    if ((b & 0x7fffffffu) > 0x7f800000u) return (b >> 16) | 0x40u;
+    return (b + 0x7fffu + ((b >> 16) & 1u)) >> 16;
+}
+// Four consecutive values as four bfloat16 (value i in bits 16 i .. 16 i + 15 of the 64 bits).
+__device__ __forceinline__ uint2 bf16_pack4(float4 v) {
+    return make_uint2(bf16_bits(v.x) | (bf16_bits(v.y) << 16), bf16_bits(v.z) | (bf16_bits(v.w) << 16));
+}
+
 // ReLU that lets NaN through (fmaxf would turn it into 0).
 __device__ __forceinline__ float relu_nan(float x) { return x > 0.f ? x : (x <= 0.f ? 0.f : x); }
 

@@ -373,7 +373,7 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
             // A~ (H W) = (A~ H) W: aggregate at the input width, finish the layer in the transform's epilogue
             if (!(l == 0 && ctx->hoist && ctx->P_valid)) {
                 GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
-                        [&] { return launch_spmm(ctx->A, ctx->H(l), y.ldi, ctx->at<float>(p.o_P[l]), y.ldi, y.fi, nullptr, bf16_of(ctx), ctx->stream); });
+                        [&] { return launch_spmm(ctx->A, ctx->H(l), y.ldi, ctx->at<float>(p.o_P[l]), y.ldi, y.fi, nullptr, bf16_of(ctx), false, ctx->stream); });
                 if (l == 0) ctx->P_valid = true;
             }
             const ActEpi act = make_act(ep, 0);
@@ -389,16 +389,18 @@ int forward_pass(gad_ctx* ctx, bool train, cudaStream_t ss) {
             continue;
         }
         if (split_pending) { GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_split, 0)); split_pending = false; }
+        // reduced-precision mode: the transform writes the bfloat16 operand copy the aggregation gathers, and nothing else
+        void* zb = ctx->use_tc ? bf16_of(ctx) : nullptr;
         GAD_RUN("gemm_fwd", l, 4.0 * p.Np * (y.fi + y.fo) + 4.0 * p.K * y.fi * y.fo, 2.0 * p.Np * y.fi * y.fo, [&] {
             if (ctx->use_tc)
                 return launch_gemm_rows_tc(&ctx->maps[kMapsPerLayer * l + 0], &ctx->maps[kMapsPerLayer * l + 1], &ctx->maps[kMapsPerLayer * l + 2], 0, passes, y.fi, y.fo, Z,
                                            y.ldo, ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr,
-                                           ctx->at<int32_t>(p.o_flags) + 1, ctx->num_sms, ctx->stream);
+                                           ctx->at<int32_t>(p.o_flags) + 1, ctx->num_sms, ctx->stream, zb);
             return launch_gemm_rows_simt(0, ctx->H(l), y.ldi, y.fi, params, p.pstride, y.w_int, y.ldw, y.fo, Z, y.ldo,
                                          ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr, ctx->stream);
         });
         GAD_RUN("spmm_fwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
-                [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, bf16_of(ctx), ctx->stream); });
+                [&] { return launch_spmm(ctx->A, Z, y.ldo, ctx->H(l + 1), y.ldo, y.fo, &ep, bf16_of(ctx), zb != nullptr, ctx->stream); });
     }
     ctx->acts_valid = true;
     return GAD_OK;
@@ -481,7 +483,7 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
         const bool agg_first = p.agg_first[l] != 0;   // then dW = (A~ H^(l))^T dPre, and dH^(l) = A~^T (dPre W^T)
         if (!agg_first)
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
-                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, bf16_of(ctx), ctx->stream); });
+                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, bf16_of(ctx), false, ctx->stream); });
         if (ctx->use_tc && p.narrow[l]) {
             // one pass over H^(l) and dZ gives both dW and dPre of the layer below (it writes G1: the column sums come first)
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
@@ -527,7 +529,7 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
             });
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));   // the column sums have read dPre
             GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
-                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G2, y.ldi, G1, y.ldi, y.fi, nullptr, bf16_of(ctx), ctx->stream); });
+                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G2, y.ldi, G1, y.ldi, y.fi, nullptr, bf16_of(ctx), false, ctx->stream); });
             GAD_RUN("relu_mask", l, 12.0 * p.Np * y.fi, 1.0 * p.Np * y.fi,
                     [&] { return launch_relu_mask(G1, ctx->H(l), y.ldi, p.Np, scale, ctx->stream); });
             continue;

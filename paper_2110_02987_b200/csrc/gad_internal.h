@@ -132,9 +132,9 @@ inline ActEpi make_act(const Epilogue& e, int col0) {
 // Kernel launchers (each enqueues on `s` and returns the cudaGetLastError of its launches)
 // ---------------------------------------------------------------------------------------------
 // bf16_scratch: null, or device room for nrows x ldz bfloat16 values: the operand is then copied there in bfloat16 and
-// gathered from the copy (reduced-precision mode).
+// gathered from the copy (reduced-precision mode); with bf16_ready the copy is there already (written by the producer).
 cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F,
-                        const Epilogue* epi, void* bf16_scratch, cudaStream_t s);
+                        const Epilogue* epi, void* bf16_scratch, bool bf16_ready, cudaStream_t s);
 
 // Tests every index of a device store and its work lists against its range (see check_store_kernel); bad[0] += violations,
 // bad[1] = min(bad[1], first offending work-list position + 1).
@@ -156,9 +156,11 @@ bool tc_make_map(void* out_map, const void* base, uint64_t inner, uint64_t rows,
                  uint64_t outer_stride_bytes, uint32_t box_rows, bool mn_major = false);
 cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w_int, int fi, int fo, int ldw, int ldkt, int K,
                                  float* w_hi, float* w_lo, float* wt_hi, float* wt_lo, cudaStream_t s);
+// Cbf16 (mode 0 only, may be null): the result goes there as bfloat16 [rows x ldc] INSTEAD of to C - the operand copy the
+// reduced-precision aggregation gathers, written by its producer.
 cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* mapBlo, int mode, int passes, int Kd, int n_cols,
                                 float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
-                                const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s);
+                                const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s, void* Cbf16 = nullptr);
 
 // Tensor-core version of launch_gemm_tn_simt; mapH / mapZ are row-box descriptors (tc_tn_rows rows) of H^(l) and dZ.
 cudaError_t launch_gemm_tn_tc(const void* mapH, const void* mapZ, int passes, int M, int n_cols, int ldw, const RowSpan* chunks,

@@ -46,6 +46,7 @@ struct TcArgs {
     const RowSpan* tiles;
     int ntiles_rows, ntn, BN, Kd;
     float* C;
+    uint2* Cbf;   // mode 0: the result as bfloat16 (four values per uint2) instead of C, or null
     int ldc;
     const float* Hmask;
     int ldh;
@@ -256,7 +257,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int r = q * 32 + 4 * i + sub_r;
-                    if (r < sp.nrows && n < a.ldc) *reinterpret_cast<float4*>(a.C + ((long long)sp.row0 + r) * a.ldc + n) = o[i];
+                    if (r < sp.nrows && n < a.ldc) {
+                        if (a.Cbf) a.Cbf[(((long long)sp.row0 + r) * a.ldc + n) >> 2] = bf16_pack4(o[i]);
+                        else *reinterpret_cast<float4*>(a.C + ((long long)sp.row0 + r) * a.ldc + n) = o[i];
+                    }
                 }
                 __syncwarp();
             }
@@ -564,16 +568,16 @@ cudaError_t launch_split_weights(const float* params, int64_t pstride, int64_t w
 
 cudaError_t launch_gemm_rows_tc(const void* mapA, const void* mapB, const void* mapBlo, int mode, int passes, int Kd, int n_cols,
                                 float* C, int ldc, const RowSpan* tiles, int ntiles, const float* Hmask, int ldh, float scale,
-                                const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s) {
+                                const ActEpi* act, int32_t* err, int num_sms, cudaStream_t s, void* Cbf16) {
     if (ntiles <= 0) return cudaSuccess;
-    if (mode == 2 && !act) return cudaErrorInvalidValue;
+    if ((mode == 2 && !act) || (Cbf16 && mode != 0)) return cudaErrorInvalidValue;
     {
         cudaError_t e = configure_kernel_once(reinterpret_cast<const void*>(gemm_tc_kernel), SMEM_BYTES_ROWS, false);
         if (e != cudaSuccess) return e;
     }
     TcArgs a;
     a.tiles = tiles; a.ntiles_rows = ntiles; a.BN = tc_bn_for(n_cols); a.ntn = (ldc + a.BN - 1) / a.BN; a.Kd = Kd;
-    a.C = C; a.ldc = ldc; a.Hmask = Hmask; a.ldh = ldh; a.scale = scale; a.mode = mode; a.passes = passes; a.err = err;
+    a.C = C; a.Cbf = reinterpret_cast<uint2*>(Cbf16); a.ldc = ldc; a.Hmask = Hmask; a.ldh = ldh; a.scale = scale; a.mode = mode; a.passes = passes; a.err = err;
     a.act = act ? *act : ActEpi{};
     const long long total = (long long)ntiles * a.ntn;
     const unsigned grid = (unsigned)(total < num_sms ? total : num_sms);

@@ -420,22 +420,17 @@ cudaError_t launch_check_store(const SparseDev& A, long long nnz, long long slot
 __global__ void __launch_bounds__(256) to_bf16_kernel(const float4* __restrict__ in, uint2* __restrict__ out, long long n4) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n4) return;
-    const float4 v = in[i];
-    auto cvt = [](float x) -> uint32_t {
-        const uint32_t b = __float_as_uint(x);
-        if ((b & 0x7fffffffu) > 0x7f800000u) return (b >> 16) | 0x40u;   // NaN: keep it quiet
-        return (b + 0x7fffu + ((b >> 16) & 1u)) >> 16;
-    };
-    out[i] = make_uint2(cvt(v.x) | (cvt(v.y) << 16), cvt(v.z) | (cvt(v.w) << 16));
+    out[i] = bf16_pack4(in[i]);
 }
 
 // F up to 1024 columns per pass (8 float4 per lane); wider operands are processed in column slabs.
 // With `bf16_scratch` (room for nrows x ldz bfloat16) the operand is first copied there in bfloat16 and gathered from
-// that copy: the reduced-precision mode, in which the gather moves half the bytes.
+// that copy: the reduced-precision mode, in which the gather moves half the bytes.  `bf16_ready`: the producing kernel has
+// written that copy already (and Z itself is not read).
 cudaError_t launch_spmm(const SparseDev& A, const float* Z, int ldz, float* out, int ldo, int F, const Epilogue* epi,
-                        void* bf16_scratch, cudaStream_t s) {
+                        void* bf16_scratch, bool bf16_ready, cudaStream_t s) {
     const int F4_all = (int)(round_up(F, 4) / 4);
-    if (bf16_scratch && A.nrows > 0) {
+    if (bf16_scratch && !bf16_ready && A.nrows > 0) {
         const long long n4 = (long long)A.nrows * (ldz / 4);
         to_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float4*>(Z), reinterpret_cast<uint2*>(bf16_scratch), n4);
         ++g_kernel_launches;
