@@ -61,3 +61,23 @@ def test_reference_arm_prints_the_contract_line():
     assert line["impl"] == "reference" and line["unit"] == "epochs/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"] == {"value": line["value"], "unit": "epochs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+
+
+def test_oracle_sample_is_sized_from_a_pilot_and_never_times_the_whole_workload():
+    """With a step budget far below one epoch the reference arm takes the leading core rows of subgraph 0 as a block of
+    their own and scales by their share of the store rows; with a generous budget it runs whole epochs."""
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    import bench
+    from gad_synth import make_workload, glorot_params
+    w = make_workload("c2", scale=0.2)
+    theta = glorot_params(w.dims, np.random.default_rng(0))
+    m, frac, sample = bench.oracle_sample(w, theta, 1e-4)
+    rows_all = sum(len(c) + len(h) for c, h in zip(w.core, w.halo))
+    assert 0.0 < frac < 1.0 and "pilot" in sample
+    assert m.store.K == 1 and m.store.n_prime == round(frac * rows_all) and m.store.n_prime >= 2000
+    assert np.all(np.isfinite(m.train_epoch()))
+    m.close()
+    m, frac, sample = bench.oracle_sample(w, theta, 1e9)
+    assert frac == 1.0 and m.store.K == w.K
+    m.close()

@@ -576,7 +576,7 @@ def test_importance_weights_summed_over_the_layers(dims, dropout):
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
 
 
-@pytest.mark.parametrize("dims,zeta_mode", [((24, 40, 5), 0), ((130, 128, 16), 0), ((12, 20, 9, 4), 2)])
+@pytest.mark.parametrize("dims,zeta_mode", [((24, 40, 5), 0), ((130, 128, 16), 0), ((12, 20, 9, 4), 2), ((40, 12, 64, 5), 1)])
 def test_epochs_replayed_as_a_graph_equal_epochs_enqueued_one_by_one(dims, zeta_mode):
     """On a stream of its own the library captures the epoch's launches after the first epoch and replays them as one
     CUDA graph; flags bit 3 keeps the launches one by one.  Same kernels in the same order: the results must agree
@@ -750,3 +750,21 @@ def test_layers_beyond_the_first_choose_the_order_of_aggregation_and_transform(f
             assert rel_err(g.get_grads(k), ref.get_grads(k)) <= TOL
             assert rel_err(g.get_params(k), ref.get_params(k)) <= TOL
         assert rel_err(g.forward(), ref.forward_global(case[0])) <= TOL
+
+
+def test_reduced_precision_mode_with_a_layer_that_aggregates_first():
+    """gemm_mode 1 through a net whose middle layer aggregates first (8 -> 200): the bfloat16 operand copies are made by
+    the conversion pass for that layer's two aggregations and by the transform's epilogue for the others.  Bar: 5e-2."""
+    case = small_random_case(73, n=900, K=3, p=0.01)
+    dims = (150, 8, 200, 6)
+    g, ref, st = make_pair(case, dims, 73, lr=0.05, gemm_mode=1)
+    with g:
+        for _ in range(2):
+            lg = g.train_epoch()
+            lr, _ = oracle_step(g, ref, 5e-2)
+            assert np.max(np.abs(lg - lr)) <= 5e-2
+        for l in range(1, len(dims)):
+            assert rel_err(g.get_activation(l), ref.activation(l)) <= 5e-2, "activation %d" % l
+        for k in range(g.K):
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= 5e-2
+            assert rel_err(g.get_params(k), ref.get_params(k)) <= 5e-2
