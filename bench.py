@@ -682,8 +682,9 @@ def main():
         # the entry's algorithmic bytes 8 nnz' + 8 N' + 8 N' F
         F_run = (top["bytes_per_launch"] - 8.0 * g.nnz_prime - 8.0 * g.n_prime) / (8.0 * g.n_prime)
         roofline["gather"] = {"bytes": 4.0 * g.nnz_prime * F_run, "GBps": 4.0 * g.nnz_prime * F_run / (avg_ms * 1e-3) / 1e9,
-                              "note": "operand rows requested by the gather (4 F bytes per entry) / time: the L2 -> SM fill path, "
-                                      "64 B per clock and SM (18.6 TB/s at 1.965 GHz), bounds this kernel, not HBM"}
+                              "note": "operand rows the gather moves on the chip (4 F bytes per stored entry) / time; this kernel's measured "
+                                      "ceilings at F = 256 (bench.py --micro gather): 23.3 TB/s with the rows L1-resident, 20.5 TB/s "
+                                      "L2-resident; the SM's L1 / shared-memory data stage moves 128 B per clock (37 TB/s at 1.965 GHz)"}
     kernels = [{"name": e["name"], "ms_per_step": e["total_ms"] / prof_steps, "share": e["total_ms"] / total_prof,
                 "GBps": e["bytes_per_launch"] * e["launches"] / (e["total_ms"] * 1e-3) / 1e9 if e["total_ms"] > 0 else None,
                 "TFLOPs": e["flops_per_launch"] * e["launches"] / (e["total_ms"] * 1e-3) / 1e12 if e["total_ms"] > 0 else None}
