@@ -44,7 +44,7 @@ extern "C" {
 #define GAD_ERR_NONFINITE (-6)      /* a loss came out NaN or infinite (reported, never trapped)            */
 #define GAD_ERR_DEVICE_TIMEOUT (-7) /* a bounded device-side wait ran out                                   */
 #define GAD_ERR_CUDA (-8)           /* a CUDA call failed; see gad_last_error                               */
-#define GAD_ERR_UNSUPPORTED (-9)    /* a documented option that this build does not implement               */
+#define GAD_ERR_UNSUPPORTED (-9)    /* a documented option that this library does not implement             */
 
 typedef struct gad_ctx gad_ctx;
 
