@@ -6,11 +6,12 @@
 // Both are C[rows x N] = A[rows x Kd] * B_k^T with A row-major (Kd contiguous) and B_k stored as N rows of Kd
 // contiguous values, i.e. both operands K-major.  Row tiles never cross a subgraph, so a tile uses one replica's B.
 //
-// fp32 accuracy from TF32 tensor cores: every operand value x is split into hi = x rounded to a 10-bit mantissa
-// (exactly representable in TF32) and lo = x - hi, rounded the same way, and the product is accumulated as
-// A_hi B_hi + A_hi B_lo + A_lo B_hi in fp32 (the dropped A_lo B_lo term and the rounding of lo are ~2^-22 relative).  B is split once per
-// epoch by a small kernel; A tiles are split in shared memory by four warps of the GEMM kernel.  With passes = 1
-// only A B is issued on the unsplit operands (TF32 operand precision).
+// fp32 accuracy from TF32 tensor cores: every operand value x is split into hi, a value with a 10-bit mantissa
+// (exactly representable in TF32), and lo = x - hi rounded to TF32, and the product is accumulated as
+// A_hi B_hi + A_hi B_lo + A_lo B_hi in fp32 (the dropped A_lo B_lo term and the rounding of lo are ~2^-20 relative).  B is split once per
+// epoch by a small kernel (hi = x rounded).  For A the tile as loaded is its own hi part, because the tensor core
+// ignores the low 13 mantissa bits of an fp32 operand (hi = x truncated); eight warps of the GEMM kernel write only
+// the lo tile beside it.  With passes = 1 only A B is issued on the unsplit operands (TF32 operand precision).
 //
 // One persistent CTA per SM, 18 warps: warp 0 issues TMA loads (128B-swizzled tiles) through a 3-stage ring,
 // warps 2-9 split the A tile, warp 1 issues tcgen05.mma, warps 10-17 drain the accumulator (tcgen05.ld, two warps
@@ -171,7 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     } else if (warp >= 2 && warp < EPI_WARP0) {
-        // ---------------- A split: hi = x rounded to TF32, lo = x - hi ----------------
+        // ---------------- A split: lo = x - (x as the tensor core reads it) ----------------
         const int tt = threadIdx.x - 64;
         int stage = 0;
         uint32_t phase = 0;
@@ -186,14 +187,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll 4
                     for (int j = 0; j < A_BYTES / 16 / (32 * SPLIT_WARPS); ++j) {
                         const int i = tt + 32 * SPLIT_WARPS * j;
-                        const float4 v = hi[i];
-                        float4 h, l;
-                        h.x = tf32_hi(v.x); l.x = tf32_round(v.x - h.x);
-                        h.y = tf32_hi(v.y); l.y = tf32_round(v.y - h.y);
-                        h.z = tf32_hi(v.z); l.z = tf32_round(v.z - h.z);
-                        h.w = tf32_hi(v.w); l.w = tf32_round(v.w - h.w);
-                        hi[i] = h;
-                        lo[i] = l;
+                        const float4 v = hi[i];   // stays where it is: the MMA reads it as the hi part
+                        lo[i] = make_float4(tf32_rest(v.x), tf32_rest(v.y), tf32_rest(v.z), tf32_rest(v.w));
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
                 }
@@ -311,7 +306,7 @@ __global__ void split_weights_kernel(const float* __restrict__ params, long long
 // H[r][m] dZ[r][n].  The reduction index is the row, so both operands are "MN-major": a tile of 32 rows x 32
 // values (128 bytes per row, swizzled in 32-byte units) is one block of the canonical layout, blocks of 32 values
 // are 4096 bytes apart (leading byte offset), groups of 4 rows 512 bytes apart (stride byte offset), and one MMA
-// (K = 8) consumes 8 rows.  Both operands are activations, so both are split into hi / lo in shared memory;
+// (K = 8) consumes 8 rows.  Both operands are activations, so both get a lo tile written beside them in shared memory;
 // rows past the end of the chunk are zeroed there.  One CTA per (chunk, 128 x BN output tile).
 // ---------------------------------------------------------------------------------------------
 struct TnArgs {
@@ -430,7 +425,7 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
         }
         if (ok) mma_commit(tfull);
     } else if (warp >= 2) {
-        // split both operand tiles into hi / lo and zero the rows past the end of the chunk
+        // write the lo tile of both operands and zero the rows past the end of the chunk
         const int tt = threadIdx.x - 64;
         int stage = 0;
         uint32_t phase = 0;
@@ -448,15 +443,12 @@ gemm_tn_tc_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant
                     const int byte_off = (blk < 4 ? blk * TN_BLOCK_BYTES : 2 * TN_A_BYTES + (blk - 4) * TN_BLOCK_BYTES) + in * 16;
                     float4* hi = reinterpret_cast<float4*>(sb + byte_off);
                     float4* lo = reinterpret_cast<float4*>(sb + byte_off + (blk < 4 ? (uint32_t)TN_A_BYTES : b_bytes));
-                    float4 v = *hi;
-                    if (row >= rows_valid) v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    float4 h, l;
-                    h.x = tf32_hi(v.x); l.x = tf32_round(v.x - h.x);
-                    h.y = tf32_hi(v.y); l.y = tf32_round(v.y - h.y);
-                    h.z = tf32_hi(v.z); l.z = tf32_round(v.z - h.z);
-                    h.w = tf32_hi(v.w); l.w = tf32_round(v.w - h.w);
-                    *hi = a.passes > 1 ? h : v;
-                    if (a.passes > 1) *lo = l;
+                    float4 v = *hi;   // a valid row stays where it is: the MMA reads it as the hi part
+                    if (row >= rows_valid) {
+                        v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        *hi = v;
+                    }
+                    if (a.passes > 1) *lo = make_float4(tf32_rest(v.x), tf32_rest(v.y), tf32_rest(v.z), tf32_rest(v.w));
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }

@@ -107,6 +107,12 @@ __device__ __forceinline__ float tf32_round(float x) {
 __device__ __forceinline__ float tf32_hi(float x) {
     return copysignf(fminf(fabsf(tf32_round(x)), __uint_as_float(0x7F7FE000u)), x);
 }
+// What is left of x once the tensor core has read it as TF32: the MMA ignores the low 13 bits of an fp32 operand, so
+// an unsplit tile already is its own hi part (x with those bits cleared) and only lo = x - hi, exact in fp32 and then
+// rounded to TF32, has to be written.  Infinity gives NaN here (inf - inf), which keeps a non-finite result non-finite.
+__device__ __forceinline__ float tf32_rest(float x) {
+    return tf32_round(x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u));
+}
 
 }  // namespace
 
