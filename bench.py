@@ -357,7 +357,8 @@ def grid_point(w, args, hbm_peak):
 
 def run_grid(args):
     """The sweep configuration as a grid: mean degree {8, 32, 128, 256} x feature width {64, 128, 256, 512} at K = 8, and
-    K in {2, 32, 64} at (mean degree 32, F = 128), on the 1 M-node Chung-Lu graph (each graph drawn once per degree);
+    K in {2, 32, 64} at (mean degree 32, F = 128) or, with --grid-all-K, at every degree and width (64 points), on the
+    1 M-node Chung-Lu graph (each graph drawn once per degree);
     then the update + consensus kernel over K in {2, 8, 32, 64} copies of a 256-256 layer.  One JSON line per point."""
     import torch
     import __graft_entry__ as entry
@@ -371,9 +372,9 @@ def run_grid(args):
     degs = [float(d) for d in args.grid_degs.split(",")]
     Fs = [int(f) for f in args.grid_F.split(",")]
     for deg in degs:
-        Ks = (8, 2, 32, 64) if deg == 32 and not args.grid_no_K else (8,)
+        Ks = (8, 2, 32, 64) if args.grid_all_K or (deg == 32 and not args.grid_no_K) else (8,)
         for w in sweep_family(deg, Ks, Fs, scale=args.scale):
-            if w.K != 8 and w.dims[0] != 128:
+            if w.K != 8 and w.dims[0] != 128 and not args.grid_all_K:
                 continue
             w.extra["mean_deg"] = deg
             line = grid_point(w, args, hbm_peak)
@@ -574,6 +575,7 @@ def main():
     ap.add_argument("--grid-degs", default="8,32,128,256")
     ap.add_argument("--grid-F", default="64,128,256,512")
     ap.add_argument("--grid-no-K", action="store_true", help="leave out the K = 2, 32, 64 points")
+    ap.add_argument("--grid-all-K", action="store_true", help="K = 2, 8, 32, 64 at every degree and width: all 64 points")
     ap.add_argument("--windows", default="64,1024,16384,0", help="--micro gather: neighbour windows in rows (0 = all rows)")
     ap.add_argument("--micro", default=None, choices=["consensus", "augment", "gather"],
                     help="a single point instead of the epoch benchmark (consensus: K = 8 copies of a 4096 x 4096 layer; "
