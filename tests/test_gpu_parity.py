@@ -528,6 +528,31 @@ def test_transform_paths_tensor_core_and_simt(gemm_mode, flags, tol, dims):
         assert rel_err(g.forward(), ref.forward_global(case[0])) <= tol
 
 
+def test_split_transform_keeps_the_bits_below_tf32():
+    """The fp32-accurate transforms hand the tensor core the activation tile as loaded and add the product with
+    lo = x - (x without its 13 lowest mantissa bits): right only if the tensor core drops those bits of an fp32 operand
+    rather than rounding them.  Features whose 13 lowest mantissa bits are all ones make the difference as large as it
+    gets (rounding would move every one of them up by a TF32 ulp, 5e-4 to 1e-3 of the value, always away from zero);
+    on a graph without edges (A~ = I) layer 0 is the transform alone.  Bar: 2e-5 of the largest entry, forward (row
+    kernel) and weight gradient (reduction over rows): several times what the split leaves, and far below the 7e-4 that
+    rounded hi parts under the same lo parts give on these inputs (worked out in fp64 on the host)."""
+    n, K, dims = 700, 2, (256, 256, 8)
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    col = np.empty(0, dtype=np.int32)
+    core = [np.arange(0, 350, dtype=np.int32), np.arange(350, n, dtype=np.int32)]
+    halo = [np.empty(0, np.int32), np.empty(0, np.int32)]
+    X = np.random.default_rng(5).standard_normal((n, dims[0])).astype(np.float32)
+    X = (X.view(np.uint32) | np.uint32(0x1FFF)).view(np.float32)
+    g, ref, st = make_pair((n, rowptr, col, None, core, halo), dims, 5, X=X, lr=0.05)
+    with g:
+        lg = g.train_epoch()
+        lr, _ = oracle_step(g, ref, 2e-5)
+        assert np.max(np.abs(lg - lr)) <= 1e-5
+        assert rel_err(g.get_activation(1), ref.activation(1)) <= 2e-5
+        for k in range(K):
+            assert rel_err(g.get_grads(k), ref.get_grads(k)) <= 2e-5
+
+
 @pytest.mark.parametrize("flags", [0, 4])
 @pytest.mark.parametrize("dims,dropout", [((40, 128, 16), 0.0), ((30, 200, 12), 0.0), ((24, 500, 7), 0.3), ((100, 8, 3), 0.0),
                                           ((16, 130, 16, 4), 0.25), ((12, 256, 5), 0.0), ((9, 516, 4), 0.0), ((20, 100, 10), 0.0), ((12, 128, 16, 100, 8), 0.0)])
