@@ -98,7 +98,12 @@ typedef struct {
                              bit 4: zeta_mode 1 on the FP32 ALUs (difference form) instead of the tensor cores;
                              bit 5: layers l >= 1 always transform before they aggregate (by default a layer whose
                              input is narrower than its output aggregates first, sigma((A~ H^(l)) W + b): the same
-                             product in the other order, with both of its SpMMs at the narrower width)              */
+                             product in the other order, with both of its SpMMs at the narrower width);
+                             bit 6: the last layer's backward aggregation reads every row (by default it runs over a
+                             copy of the transposed store without the entries that read a row carrying no loss - a
+                             replicated node, or a core node outside the training split, where d loss / d logits is
+                             zero (the loss of Section 3.3 is taken over the subgraph's own training nodes): the same
+                             sums without their zero terms; the copy costs up to 8 bytes per stored entry)           */
 } gad_config;
 
 /* Bytes of device workspace gad_create needs for these inputs.  Host-only; touches no GPU. */

@@ -77,6 +77,7 @@ struct Plan {
     size_t o_bf16 = 0;                // [Np x widest SpMM operand] bfloat16 copy of the operand (gemm_mode 1), else unused
     size_t bytes = 0;
     // offsets into the workspace
+    size_t o_growptr = 0, o_gecv = 0, o_gfin = 0, o_gitems = 0;   // the loss rows' store (see gad_ctx::Ag)
     size_t o_rowptr, o_ecv, o_fin, o_items, o_trowptr, o_tecv, o_tfin, o_titems, o_spmm_scratch, o_sub_off, o_gid, o_deg, o_label, o_train,
         o_deg_sum, o_deg_sq, o_inv_ntrain, o_tiles, o_chunks, o_chunk_ptr, o_dw_chunks, o_dw_chunk_ptr, o_core_spans, o_G1, o_G2, o_params, o_grads,
         o_dw_partial, o_cs_partial, o_loss_partial, o_zeta_partial, o_zeta, o_loss, o_flags, o_zeta_f, o_w_f, o_stage,
@@ -170,6 +171,11 @@ int make_plan(Plan& p, int32_t n, int32_t K, const std::vector<int32_t>& sub_off
     p.o_trowptr = take(cur, 8 * (Np + 1)); p.o_tecv = take(cur, 8 * (size_t)nnz);
     p.o_tfin = take(cur, 16 * max_fin);
     p.o_titems = take(cur, 16 * (Np + max_parts));
+    if (!(cfg->flags & 64)) {
+        p.o_growptr = take(cur, 8 * (Np + 1)); p.o_gecv = take(cur, 8 * (size_t)nnz);
+        p.o_gfin = take(cur, 16 * max_fin);
+        p.o_gitems = take(cur, 16 * (Np + max_parts));
+    }
     p.o_sub_off = take(cur, 4 * (size_t)(K + 1)); p.o_gid = take(cur, 4 * Np); p.o_deg = take(cur, 4 * Np);
     p.o_label = take(cur, 4 * Np); p.o_train = take(cur, Np);
     p.o_deg_sum = take(cur, 8 * (size_t)K); p.o_deg_sq = take(cur, 8 * (size_t)K); p.o_inv_ntrain = take(cur, 4 * (size_t)K);
@@ -254,6 +260,12 @@ struct gad_ctx {
     std::string err;
     bool symmetric = false;
     SparseDev A, At;
+    // The transposed store without the entries that read a row carrying no loss (a replicated node, or a core node that
+    // is not a training node): d loss / d logits is zero there, so the backward aggregation of the last layer gathers
+    // only the rest and adds the same numbers in the same order.  Built once (the split is fixed at creation).
+    SparseDev Ag;
+    bool use_loss_rows = false;
+    int64_t nnz_loss_rows = 0;
     int64_t epoch = 0;
     std::vector<int32_t> sub_off, gid;
     std::vector<int64_t> ntrain;
@@ -335,7 +347,7 @@ int run(gad_ctx* ctx, const char* name, int layer, double bytes, double flops, F
 // Room for the bfloat16 copy of an aggregation's operand: the reduced-precision mode gathers from that copy.
 void* bf16_of(gad_ctx* ctx) { return ctx->cfg.gemm_mode == 1 ? (void*)(ctx->ws + ctx->p.o_bf16) : nullptr; }
 
-double spmm_bytes(const Plan& p, int F) { return 8.0 * p.nnz + 8.0 * p.Np + 8.0 * (double)p.Np * F; }
+double spmm_bytes(const Plan& p, int F, int64_t nnz = -1) { return 8.0 * (nnz < 0 ? p.nnz : nnz) + 8.0 * p.Np + 8.0 * (double)p.Np * F; }
 
 // Inside a training epoch the kernels that depend on little (operand split of the weights, zeta, bias gradients) go
 // to a second stream and run beside the aggregation / transform sequence; events order them against it.  While
@@ -469,6 +481,10 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
     bool bias_done = false;   // the layer above was narrow: its fused kernel has already summed this layer's dPre columns
     for (int l = p.L - 1; l >= 0; --l) {
         const Layer& y = p.layers[l];
+        // the store of this layer's backward aggregation, and its entries
+        const bool loss_rows = ctx->use_loss_rows && l == p.L - 1;
+        const SparseDev& Ab = loss_rows ? ctx->Ag : (ctx->symmetric ? ctx->A : ctx->At);
+        const int64_t nnz_b = loss_rows ? ctx->nnz_loss_rows : p.nnz;
         if (!bias_done) {
             // db reads dPre (G1) beside the kernels that follow; the next writer of G1 waits for it
             int rc = hand_over(ctx, ctx->stream, ss, ctx->ev_g1);
@@ -482,8 +498,8 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
         bias_done = false;
         const bool agg_first = p.agg_first[l] != 0;   // then dW = (A~ H^(l))^T dPre, and dH^(l) = A~^T (dPre W^T)
         if (!agg_first)
-            GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo), 2.0 * p.nnz * y.fo,
-                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G1, y.ldo, G2, y.ldo, y.fo, nullptr, bf16_of(ctx), false, ctx->stream); });
+            GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fo, nnz_b), 2.0 * nnz_b * y.fo,
+                    [&] { return launch_spmm(Ab, G1, y.ldo, G2, y.ldo, y.fo, nullptr, bf16_of(ctx), false, ctx->stream); });
         if (ctx->use_tc && p.narrow[l]) {
             // one pass over H^(l) and dZ gives both dW and dPre of the layer below (it writes G1: the column sums come first)
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));
@@ -528,8 +544,8 @@ int backward_pass(gad_ctx* ctx, cudaStream_t ss) {
                                              ctx->at<RowSpan>(p.o_tiles), (int)p.tiles.size(), nullptr, 0, 1.f, nullptr, ctx->stream);
             });
             if (ss != ctx->stream) GAD_CK(cudaStreamWaitEvent(ctx->stream, ctx->ev_bias, 0));   // the column sums have read dPre
-            GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fi), 2.0 * p.nnz * y.fi,
-                    [&] { return launch_spmm(ctx->symmetric ? ctx->A : ctx->At, G2, y.ldi, G1, y.ldi, y.fi, nullptr, bf16_of(ctx), false, ctx->stream); });
+            GAD_RUN("spmm_bwd", l, spmm_bytes(p, y.fi, nnz_b), 2.0 * nnz_b * y.fi,
+                    [&] { return launch_spmm(Ab, G2, y.ldi, G1, y.ldi, y.fi, nullptr, bf16_of(ctx), false, ctx->stream); });
             GAD_RUN("relu_mask", l, 12.0 * p.Np * y.fi, 1.0 * p.Np * y.fi,
                     [&] { return launch_relu_mask(G1, ctx->H(l), y.ldi, p.Np, scale, ctx->stream); });
             continue;
@@ -590,7 +606,8 @@ void default_params(const std::vector<int32_t>& dims, uint64_t seed, float* out)
 
 int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::vector<int64_t>& rowptr, const std::vector<int32_t>& col,
                   const std::vector<float>& val,
-                  size_t o_rowptr, size_t o_ecv, size_t o_fin, size_t o_items, SparseDev& out) {
+                  size_t o_rowptr, size_t o_ecv, size_t o_fin, size_t o_items, SparseDev& out, int64_t forced_part = 0,
+                  int64_t* part_entries = nullptr) {
     const Plan& p = ctx->p;
     std::vector<uint2> ecv(col.size());
     for (size_t e = 0; e < col.size(); ++e) {
@@ -599,7 +616,8 @@ int upload_sparse(gad_ctx* ctx, const std::vector<int32_t>& sub_off, const std::
         ecv[e] = make_uint2((uint32_t)col[e], bits);
     }
     RowWork work;
-    bin_rows(rowptr, sub_off, work);
+    bin_rows(rowptr, sub_off, work, forced_part);
+    if (part_entries) *part_entries = work.part_entries;
     if (work.slots > p.slots) return fail(ctx, GAD_ERR_OOM, "SpMM scratch slots exceed the planned count");
     GAD_CK(cudaMemcpyAsync(ctx->ws + o_rowptr, rowptr.data(), 8 * rowptr.size(), cudaMemcpyHostToDevice, ctx->stream));
     if (!ecv.empty()) GAD_CK(cudaMemcpyAsync(ctx->ws + o_ecv, ecv.data(), 8 * ecv.size(), cudaMemcpyHostToDevice, ctx->stream));
@@ -688,10 +706,11 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
     ctx->sub_off = st.sub_off;
     ctx->gid = st.gid;
 
-    rc = upload_sparse(ctx, st.sub_off, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_fin, p.o_items, ctx->A);
+    int64_t part_t = 0;   // part length of the store the backward aggregation reads
+    rc = upload_sparse(ctx, st.sub_off, st.rowptr, st.col, st.val, p.o_rowptr, p.o_ecv, p.o_fin, p.o_items, ctx->A, 0, &part_t);
     if (rc != GAD_OK) return rc;
     if (!st.symmetric) {
-        rc = upload_sparse(ctx, st.sub_off, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tfin, p.o_titems, ctx->At);
+        rc = upload_sparse(ctx, st.sub_off, st.t_rowptr, st.t_col, st.t_val, p.o_trowptr, p.o_tecv, p.o_tfin, p.o_titems, ctx->At, 0, &part_t);
         if (rc != GAD_OK) return rc;
     }
     // per-row labels and loss mask, per-subgraph degree sums and training counts
@@ -713,6 +732,25 @@ int gad_create(gad_ctx** out, const gad_csr* g, const gad_partition* part, const
         }
         inv_ntrain[k] = ctx->ntrain[k] > 0 ? 1.f / (float)ctx->ntrain[k] : 0.f;
         ctx->ntrain_total += ctx->ntrain[k];
+    }
+    if (!(cfg->flags & 64)) {
+        // the transposed store restricted to the columns that carry loss, rows cut as the full one cuts them (so its
+        // scratch slots are no more than the planned ones)
+        const std::vector<int64_t>& rp = st.symmetric ? st.rowptr : st.t_rowptr;
+        const std::vector<int32_t>& cl = st.symmetric ? st.col : st.t_col;
+        const std::vector<float>& vl = st.symmetric ? st.val : st.t_val;
+        std::vector<int64_t> grp((size_t)p.Np + 1, 0);
+        std::vector<int32_t> gcl;
+        std::vector<float> gvl;
+        for (int64_t r = 0; r < p.Np; ++r) {
+            for (int64_t e = rp[r]; e < rp[r + 1]; ++e)
+                if (train[(size_t)cl[e]]) { gcl.push_back(cl[e]); gvl.push_back(vl[e]); }
+            grp[(size_t)r + 1] = (int64_t)gcl.size();
+        }
+        rc = upload_sparse(ctx, st.sub_off, grp, gcl, gvl, p.o_growptr, p.o_gecv, p.o_gfin, p.o_gitems, ctx->Ag, part_t);
+        if (rc != GAD_OK) return rc;
+        ctx->use_loss_rows = true;
+        ctx->nnz_loss_rows = (int64_t)gcl.size();
     }
     if ((rc = upload(ctx, p.o_sub_off, st.sub_off)) || (rc = upload(ctx, p.o_gid, st.gid)) || (rc = upload(ctx, p.o_deg, st.deg)) ||
         (rc = upload(ctx, p.o_label, label)) || (rc = upload(ctx, p.o_train, train)) || (rc = upload(ctx, p.o_deg_sum, deg_sum)) ||
@@ -1123,6 +1161,8 @@ int gad_check_store(gad_ctx* ctx, int64_t* violations) {
     GAD_CK(cudaMemcpyAsync(bad, init, 16, cudaMemcpyHostToDevice, ctx->stream));
     GAD_CK(launch_check_store(ctx->A, p.nnz, p.slots, ctx->at<int32_t>(p.o_sub_off), p.K, bad, ctx->stream));
     if (!ctx->symmetric) GAD_CK(launch_check_store(ctx->At, p.nnz, p.slots, ctx->at<int32_t>(p.o_sub_off), p.K, bad, ctx->stream));
+    if (ctx->use_loss_rows)
+        GAD_CK(launch_check_store(ctx->Ag, ctx->nnz_loss_rows, p.slots, ctx->at<int32_t>(p.o_sub_off), p.K, bad, ctx->stream));
     unsigned long long out[2] = {0, 0};
     GAD_CK(cudaMemcpyAsync(out, bad, 16, cudaMemcpyDeviceToHost, ctx->stream));
     GAD_CK(cudaStreamSynchronize(ctx->stream));

@@ -62,7 +62,8 @@ struct RowWork {
     int64_t slots = 0, part_entries = kMinPart;
 };
 int64_t part_entries_for(const std::vector<int64_t>& rowptr);
-void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& sub_off, RowWork& out);
+// forced_part > 0: cut rows into parts of that many entries instead of the length part_entries_for would choose
+void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& sub_off, RowWork& out, int64_t forced_part = 0);
 // Scratch slots bin_rows would use, from the row lengths alone.
 int64_t count_slots(const std::vector<int64_t>& rowptr);
 

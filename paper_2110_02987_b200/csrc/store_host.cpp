@@ -263,9 +263,9 @@ int64_t count_slots(const std::vector<int64_t>& rowptr) {
     return slots;
 }
 
-void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& sub_off, RowWork& out) {
+void bin_rows(const std::vector<int64_t>& rowptr, const std::vector<int32_t>& sub_off, RowWork& out, int64_t forced_part) {
     const int64_t Np = (int64_t)rowptr.size() - 1;
-    const int64_t part = part_entries_for(rowptr);
+    const int64_t part = forced_part > 0 ? forced_part : part_entries_for(rowptr);
     out.perm.clear(); out.parts.clear(); out.fin.clear(); out.items.clear(); out.slots = 0; out.part_entries = part;
     std::vector<int64_t> count(64, 0);
     auto bin_of = [](int64_t len) { int b = 0; while (len > 1) { len >>= 1; ++b; } return b; };

@@ -360,6 +360,51 @@ def test_hub_rows_and_wide_features():
         check_epoch(g, ref)
 
 
+@pytest.mark.parametrize("directed,weighted,dims", [(False, False, (24, 40, 5)), (True, True, (24, 40, 70)), (True, False, (16, 6))])
+def test_last_backward_aggregation_over_the_rows_that_carry_loss(directed, weighted, dims):
+    """d loss / d logits is zero on replicated rows and on core rows outside the training split, so by default the last
+    layer's backward aggregation runs over a store without the entries that read such rows.  Same gradients as the
+    full store (flag bit 6) up to the grouping of a cut row's partial sums, and as the oracle; subgraph 1 has no
+    training node at all, subgraph 0 holds a hub row that is cut into parts."""
+    n, rowptr, col, w, core, halo = small_random_case(31, n=1500, K=3, p=0.004, directed=directed, weighted=weighted)
+    # a hub: node core[0][0] gains an edge from and to every other node of its subgraph
+    hub, others = int(core[0][0]), [int(v) for v in core[0][1:]]
+    src = np.repeat(np.arange(n, dtype=np.int64), np.diff(rowptr))
+    pairs = set(zip(src.tolist(), col.tolist()))
+    extra = [(hub, v) for v in others if (hub, v) not in pairs] + [(v, hub) for v in others if (v, hub) not in pairs]
+    es = np.concatenate([src, np.array([e[0] for e in extra], dtype=np.int64)])
+    ed = np.concatenate([col.astype(np.int64), np.array([e[1] for e in extra], dtype=np.int64)])
+    ew = None if w is None else np.concatenate([w, np.ones(len(extra), dtype=np.float32)])
+    order = np.lexsort((ed, es))
+    es, ed = es[order], ed[order]
+    ew = None if ew is None else ew[order]
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(np.bincount(es, minlength=n), out=rowptr[1:])
+    col = ed.astype(np.int32)
+    rng = np.random.default_rng(77)
+    X = rng.standard_normal((n, dims[0])).astype(np.float32)
+    y = rng.integers(0, dims[-1], size=n).astype(np.int32)
+    split = rng.integers(0, 3, size=n).astype(np.uint8)
+    split[core[1]] = 1 + (split[core[1]] & 1)          # no training node in subgraph 1
+    theta = glorot_params(dims, rng, bias_scale=0.2)
+    cp, cn = flat(core)
+    hp, hn = flat(halo)
+    st = orc().Store(n, rowptr, col, cp, cn, hp, hn, weights=ew)
+    ref = orc().Model(st, X, y, split, dims, theta, lr=0.05)
+    a = pkg().Gad(n, rowptr, col, cp, cn, hp, hn, X, y, split, dims, init_params=theta, weights=ew, lr=0.05)
+    b = pkg().Gad(n, rowptr, col, cp, cn, hp, hn, X, y, split, dims, init_params=theta, weights=ew, lr=0.05, flags=64)
+    with a, b:
+        assert a.check_store() == 0 and b.check_store() == 0
+        assert a.ntrain()[1] == 0
+        for _ in range(2):
+            b.train_epoch()
+            check_epoch(a, ref)
+            assert np.array_equal(a.get_activation(len(dims) - 1), b.get_activation(len(dims) - 1))   # the forward pass does not differ
+            for k in range(a.K):
+                assert rel_err(a.get_grads(k), b.get_grads(k)) <= 1e-6
+                assert rel_err(a.get_params(k), b.get_params(k)) <= 1e-6
+
+
 def test_runs_are_bitwise_reproducible_and_resume_is_exact(tiny_signal):
     w = tiny_signal
     theta = glorot_params(w.dims, np.random.default_rng(5))
